@@ -1,0 +1,246 @@
+/*
+ * ppo_b200.h -- C ABI of the per-token PPO-for-RLHF hot path (arXiv 2403.17031) for NVIDIA
+ * B200 (sm_100a).
+ *
+ * The path, in the order a PPO iteration runs it:
+ *   1. ppo_logprob_entropy      log-prob of each sampled response token and entropy of the
+ *                               temperature-scaled distribution, for the policy and again for
+ *                               the frozen SFT reference
+ *   2. ppo_truncate_and_score   the "EOS trick": cut at the first EOS, fill [PAD], -1 score
+ *   3. ppo_kl_rewards           per-token KL penalty, reward-model score on the last token
+ *   4. ppo_gae                  reverse-time generalised advantage estimation
+ *   5. ppo_whiten               masked mean/variance normalisation of the advantages
+ *   6. ppo_loss_fwd_bwd         clipped policy loss + clipped value loss and their gradients
+ *   7. ppo_lmhead_logprob_entropy  step 1 with the LM-head GEMM fused in (logits never stored)
+ *
+ * General rules
+ *   - Every pointer is a DEVICE pointer owned by the caller unless a comment says "host".
+ *     The library allocates nothing; scratch lives in a caller-provided workspace.
+ *   - Work is enqueued on the caller's stream (`stream` is a cudaStream_t passed as void*;
+ *     NULL is the default stream) and the call returns without synchronising, except
+ *     ppo_last_device_status and the *_host entry points.
+ *   - Return value: 0 on success; a negative PPO_ERR_* code for an argument error found on
+ *     the host before anything is launched; a positive value is a cudaError_t reported by
+ *     the CUDA runtime.  Nothing traps, aborts or falls back to a CPU path.
+ *   - Outputs are completely overwritten (positions with mask 0 receive 0); inputs are never
+ *     modified; outputs must not alias inputs unless stated.
+ *   - Data-dependent soft errors (a token id outside [0,V), an all-zero mask, a bounded wait
+ *     that ran out) set bits in a status word inside the workspace; the affected outputs are
+ *     NaN.  Read it with ppo_last_device_status.
+ *   - Logits: row-major [rows, V], dtype PPO_F32 or PPO_BF16.  The fast kernels need the base
+ *     address and the row pitch to be multiples of 16 bytes and V a multiple of 16/sizeof(elt);
+ *     anything else takes a slower element-wise kernel with the same results.
+ */
+#ifndef PPO_B200_H
+#define PPO_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* logits storage types */
+#define PPO_F32 0
+#define PPO_BF16 1
+
+/* host-side argument errors (returned, never thrown) */
+#define PPO_OK 0
+#define PPO_ERR_NULL (-1)        /* a required pointer is NULL */
+#define PPO_ERR_SHAPE (-2)       /* a size is <= 0, too large, or inconsistent */
+#define PPO_ERR_PARAM (-3)       /* temperature <= 0, negative clip range, eos_id == pad_id, non-finite */
+#define PPO_ERR_ALIGN (-4)       /* pointer alignment below the element size / documented minimum */
+#define PPO_ERR_DTYPE (-5)       /* unknown dtype code */
+#define PPO_ERR_UNSUPPORTED (-6) /* shape outside what the kernel handles (documented per call) */
+
+/* bits of the device status word */
+#define PPO_DEV_BAD_TOKEN 1      /* a token id was outside [0, V): that row's outputs are NaN */
+#define PPO_DEV_EMPTY_MASK 2     /* mask selected no element: statistics / losses are 0 */
+#define PPO_DEV_TIMEOUT 4        /* a bounded wait inside a kernel gave up; outputs are invalid */
+
+/* indices into the losses[8] output of ppo_loss_fwd_bwd */
+enum { PPO_LOSS_PG = 0, PPO_LOSS_VF = 1, PPO_LOSS_TOTAL = 2, PPO_LOSS_APPROX_KL = 3,
+       PPO_LOSS_PG_CLIPFRAC = 4, PPO_LOSS_VF_CLIPFRAC = 5, PPO_LOSS_ENTROPY = 6, PPO_LOSS_N = 7 };
+
+/*
+ * Hyper-parameters of the path.  Defaults (ppo_default_params) are the paper's Table "PPO
+ * hyperparameters": temperature 0.7, kl_coef (beta) 0.05, gamma 1.0, lam 0.95, cliprange
+ * (epsilon) 0.2, cliprange_value (epsilon-hat) 0.2, vf_coef (c1) 0.1; no_eos_score -1 from the
+ * "EOS trick"; whiten_eps 1e-8 from the whiten() listing; eos_id 0 (Pythia <|endoftext|>);
+ * pad_id must be set by the caller to a [PAD] id different from eos_id (section "Dataset ->
+ * ... do not use EOS synonymously as [PAD]"); the default 1 is only a placeholder.
+ */
+typedef struct ppo_params {
+    float temperature, kl_coef, gamma, lam, cliprange, cliprange_value, vf_coef, no_eos_score,
+        whiten_eps;
+    int32_t eos_id, pad_id;
+} ppo_params;
+
+void ppo_default_params(ppo_params *p /* host */);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int ppo_version(void);
+
+/*
+ * Process-wide tuning switches; every setting computes the same results.  Returns 0, or
+ * PPO_ERR_PARAM for an unknown key/value.  Not thread-safe against concurrent launches.
+ *   PPO_OPT_LOSS_ROW_CACHE  how ppo_loss_fwd_bwd keeps a row between its statistics pass and its
+ *                           gradient pass: 0 = choose by row size (default), 1 = in shared memory
+ *                           whenever the row fits one block, 2 = re-read it from global memory/L2
+ */
+#define PPO_OPT_LOSS_ROW_CACHE 1
+int ppo_set_option(int key, int value);
+
+/*
+ * Workspace.  ppo_workspace_bytes gives the size (a multiple of 256) that serves every call
+ * below for batches up to B x T tokens (V is accepted for future use); the fused LM-head call
+ * needs ppo_lmhead_workspace_bytes(M, K, V) instead (use the larger of the two to share one
+ * buffer).  The buffer must be 256-byte aligned and must be cleared once with
+ * ppo_workspace_init before its first use.  One workspace serves one stream at a time.
+ */
+size_t ppo_workspace_bytes(int32_t B, int32_t T, int64_t V);
+size_t ppo_lmhead_workspace_bytes(int64_t M, int64_t K, int64_t V);
+int ppo_workspace_init(void *workspace, size_t bytes, void *stream);
+
+/*
+ * Waits for `stream`, copies the status word to *status (host), clears it on the device, and
+ * returns 0 (or a CUDA error).  The word accumulates PPO_DEV_* bits from every call that was
+ * given this workspace since the last read.
+ */
+int ppo_last_device_status(void *workspace, void *stream, int *status /* host */);
+
+/*
+ * Step 1.  For every row r of logits [rows, V] (row pitch `row_stride` elements):
+ *     z = logits[r, :] / temperature,   lse = log sum_j exp(z_j),
+ *     logprob[r] = z[tokens[r]] - lse,  entropy[r] = -sum_j softmax(z)_j * log softmax(z)_j.
+ * The paper fixes the temperature (Table "PPO hyperparameters": 0.7) and requires policy and
+ * SFT reference to be scored identically (Eq. "RL"; section "Disable dropout ...": ratios
+ * are 1 in the first epoch); call once per model.  Row [b,t] must be the distribution that
+ * response token t was sampled from (the caller has already shifted/sliced the sequence
+ * logits).  -inf logits are allowed and carry zero probability.
+ *   mask     nullable [rows] u8: rows with 0 are not read and output 0.
+ *   entropy, lse   nullable [rows] f32.
+ *   workspace      nullable; without it out-of-range tokens still give NaN but set no status.
+ * Errors: PPO_ERR_NULL, PPO_ERR_SHAPE (rows < 0, V <= 0, row_stride < V, V >= 2^31),
+ * PPO_ERR_PARAM (temperature), PPO_ERR_DTYPE, PPO_ERR_ALIGN (base not element-aligned).
+ * rows == 0 is a successful no-op.
+ */
+int ppo_logprob_entropy(const void *logits, int dtype, int64_t rows, int64_t V, int64_t row_stride,
+                        const int32_t *tokens, const uint8_t *mask, float temperature,
+                        float *logprob, float *entropy, float *lse, void *workspace, void *stream);
+
+/*
+ * Step 2, the "EOS trick" (section "PPO Training -> EOS trick"): responses always have T
+ * sampled tokens; the response is cut at its first eos_id, later positions become pad_id, and
+ * a response without EOS has its score REPLACED by no_eos_score (-1).  The EOS token itself
+ * stays a real token (the reward model's score is read on it).
+ *   responses      [B,T] i32 in;  scores [B] f32 in (nullable together with scores_out)
+ *   responses_out  [B,T] i32 (nullable; may alias responses)
+ *   eos_index      [B] i32, -1 when absent (nullable)
+ *   seq_len        [B] i32 = eos_index+1, or T (nullable)
+ *   mask           [B,T] u8 = (t < seq_len) (nullable)
+ *   scores_out     [B] f32 (nullable)
+ * Integer outputs are exact.  Errors: PPO_ERR_NULL, PPO_ERR_SHAPE, PPO_ERR_PARAM (eos_id ==
+ * pad_id).
+ */
+int ppo_truncate_and_score(const int32_t *responses, int32_t B, int32_t T, int32_t eos_id,
+                           int32_t pad_id, const float *scores, float no_eos_score,
+                           int32_t *responses_out, int32_t *eos_index, int32_t *seq_len,
+                           uint8_t *mask, float *scores_out, void *stream);
+
+/*
+ * Step 3 (Eq. "RL": R = r_phi - beta * KL[pi_theta || pi_SFT]; figure "reward vs value": the
+ * reward vector holds a KL penalty per token and the reward-model score on the EOS token):
+ *     kl[b,t] = mask * (logprob - ref_logprob)         (the k1 estimator at the sampled token)
+ *     rewards[b,t] = -kl_coef * kl[b,t];  rewards[b, seq_len[b]-1] += scores[b]
+ * All arrays [B,T] f32 except seq_len [B] i32, scores [B] f32 (already passed through step 2).
+ * kl and rewards are nullable (at least one required).
+ */
+int ppo_kl_rewards(const float *logprob, const float *ref_logprob, const uint8_t *mask,
+                   const int32_t *seq_len, const float *scores, int32_t B, int32_t T,
+                   float kl_coef, float *kl, float *rewards, void *stream);
+
+/*
+ * Step 4, GAE with the table's gamma and lambda.  The episode ends after the last real token
+ * (the value function predicts the end-of-episode return, section "Value model initializes
+ * from the reward model"), so nothing is bootstrapped beyond seq_len-1:
+ *     delta_t = r_t + gamma * V_{t+1} - V_t,   A_t = delta_t + gamma * lam * A_{t+1},
+ *     returns_t = A_t + V_t;   V_t = A_t = 0 for t >= seq_len;  zeros are written there.
+ * One warp per sequence runs a segmented reverse scan of affine maps in fp64 and rounds once.
+ * Any T >= 1 is supported.
+ */
+int ppo_gae(const float *rewards, const float *values, const int32_t *seq_len, int32_t B, int32_t T,
+            float gamma, float lam, float *advantages, float *returns, void *stream);
+
+/*
+ * Step 5, the paper's whiten() (listing in section "Reward whitening"; applied to advantages
+ * in section "Advantage whitening") over the entries with mask 1 of one flat array:
+ *     mean = sum(m*x)/n,  var = sum(m*(x-mean)^2)/n  (biased),
+ *     out = (x - mean) * rsqrt(var + eps);  if (!shift_mean) out += mean;  out = 0 where m == 0.
+ * shift_mean != 0 (the listing's default, used for advantages) leaves zero mean.
+ *   mask nullable (all ones); out may alias x; stats3 nullable [3] f32 = {mean, var, n}.
+ * One thread block computes the statistics in fp64 in a fixed order (bit-reproducible).
+ * n == 0 writes zeros and sets PPO_DEV_EMPTY_MASK (when a workspace is given).
+ */
+int ppo_whiten(const float *x, const uint8_t *mask, int64_t n_elems, int shift_mean, float eps,
+               float *out, float *stats3, void *workspace, void *stream);
+
+/*
+ * Step 6.  With lp_new computed from `logits` as in step 1 (temperature from *p),
+ * rho = exp(lp_new - old_logprob), A = advantages, v = values_new:
+ *     pg = max(-A*rho, -A*clip(rho, 1-cliprange, 1+cliprange))
+ *     vc = clip(v, values_old - cliprange_value, values_old + cliprange_value)
+ *     vf = max((v - returns)^2, (vc - returns)^2)
+ *     losses[PG] = sum(m*pg)/n,  losses[VF] = 0.5*sum(m*vf)/n,  losses[TOTAL] = PG + vf_coef*VF
+ * (Table "PPO hyperparameters": cliprange 0.2, cliprange_value 0.2, vf_coef 0.1, value-loss
+ * clipping on, one minibatch so n counts the whole call's real tokens), and the gradients of
+ * losses[TOTAL]:
+ *     dlogits[b,t,j] = g * (1[j == token] - softmax(z)_j) / temperature,
+ *         g = (m/n) * (-A*rho) unless the clipped branch is strictly larger (then 0)
+ *     dvalues[b,t]   = vf_coef * (m/n) * (v - returns) unless the clipped branch is strictly larger
+ * Also losses[APPROX_KL] = 0.5*mean((lp_new-old_logprob)^2), the two clip fractions, the mean
+ * entropy and n.  Rows with mask 0 are not read; their dlogits rows are zero-filled.
+ *   logits   [B,T,V] contiguous (pitch V);   dlogits same shape and dtype (nullable: forward
+ *            statistics and dlogprob only);  must not alias logits
+ *   tokens, mask(u8), old_logprob, advantages, values_new, values_old, returns: [B,T]
+ *   losses   [8] f32;  dvalues [B,T] f32;  new_logprob, entropy, dlogprob: nullable [B,T] f32
+ *   workspace required (ppo_workspace_bytes(B,T,V)).
+ * Per-row partial sums are reduced in a fixed order in fp64, so results are bit-reproducible.
+ */
+int ppo_loss_fwd_bwd(const void *logits, int dtype, int32_t B, int32_t T, int64_t V,
+                     const int32_t *tokens, const uint8_t *mask, const float *old_logprob,
+                     const float *advantages, const float *values_new, const float *values_old,
+                     const float *returns, const ppo_params *p /* host */, float *losses,
+                     void *dlogits, float *dvalues, float *new_logprob, float *entropy,
+                     float *dlogprob, void *workspace, void *stream);
+
+/*
+ * Step 6 when the logits were never materialised (fused LM head): same losses and dvalues from
+ * a given new_logprob [B,T]; dlogprob [B,T] receives g.  entropy nullable [B,T] (averaged into
+ * losses[ENTROPY] when given, else 0).
+ */
+int ppo_loss_from_logprob(const float *new_logprob, const float *entropy, int32_t B, int32_t T,
+                          const uint8_t *mask, const float *old_logprob, const float *advantages,
+                          const float *values_new, const float *values_old, const float *returns,
+                          const ppo_params *p /* host */, float *losses, float *dlogprob,
+                          float *dvalues, void *workspace, void *stream);
+
+/*
+ * Step 7 (fused LM head): logits[r, :] = H[r, :] . W are formed tile by tile on the tensor
+ * cores (bf16 inputs, fp32 accumulation in tensor memory) and consumed by step 1's reduction
+ * in the epilogue; they are never written to memory.
+ *   H [M,K] bf16 row-major;  W [K,V] bf16 row-major;  tokens [M];  mask nullable [M]
+ *   logprob [M] f32;  entropy, lse nullable [M] f32
+ * Requirements: K % 64 == 0, V % 8 == 0, H and W 16-byte aligned; otherwise
+ * PPO_ERR_UNSUPPORTED.  workspace required (ppo_lmhead_workspace_bytes).
+ */
+int ppo_lmhead_logprob_entropy(const void *H, const void *W, int64_t M, int64_t K, int64_t V,
+                               const int32_t *tokens, const uint8_t *mask, float temperature,
+                               float *logprob, float *entropy, float *lse, void *workspace,
+                               void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PPO_B200_H */

@@ -1,0 +1,200 @@
+// Shared device/host helpers of the PPO hot-path kernels (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+#include "ppo_b200.h"
+
+namespace ppo {
+
+// ---------------------------------------------------------------- workspace layout
+// [0, 256)                      WorkspaceHeader
+// [256, 256 + rows*8*4)         per-token loss partials, 8 floats per token
+struct WorkspaceHeader {
+    int status;      // PPO_DEV_* bits, sticky until read
+    int n_tokens;    // number of mask==1 tokens of the loss call in flight
+    int reserved[62];
+};
+static_assert(sizeof(WorkspaceHeader) == 256, "header is one 256-byte block");
+
+constexpr int kPartialsPerToken = 8;   // pg, vf, kl, pg_clipped, vf_clipped, entropy, unused, unused
+constexpr size_t kHeaderBytes = 256;
+
+inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+
+__host__ __device__ inline WorkspaceHeader *ws_header(void *ws) { return reinterpret_cast<WorkspaceHeader *>(ws); }
+__host__ __device__ inline float *ws_partials(void *ws)
+{
+    return reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(ws) + kHeaderBytes);
+}
+
+inline bool finite_f(float x) { return isfinite(x); }
+
+#define PPO_RETURN_IF_CUDA(expr)                      \
+    do {                                              \
+        cudaError_t e__ = (expr);                     \
+        if (e__ != cudaSuccess) return (int)e__;      \
+    } while (0)
+
+inline int launch_status()
+{
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? PPO_OK : (int)e;
+}
+
+// ---------------------------------------------------------------- small device helpers
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kNegBig = -1.0e30f;   // stands in for -inf: exp2 of it is 0 and 0 * it is 0
+
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Running softmax statistics of a set of scaled logits y (base-2 units, y = logit*log2(e)/tau):
+//   m = reference (>= every y seen),  s = sum 2^(y-m),  u = sum 2^(y-m) * (y-m).
+// log2-sum-exp = m + log2 s;  entropy = ln2 * (log2 s - u/s).
+struct SoftmaxState {
+    float m, s, u;
+    __device__ __forceinline__ void init() { m = kNegBig; s = 0.f; u = 0.f; }
+    // move the reference up to nm >= m
+    __device__ __forceinline__ void rebase(float nm)
+    {
+        float d = m - nm;
+        float a = ex2(d);
+        u = a * fmaf(d, s, u);
+        s *= a;
+        m = nm;
+    }
+    __device__ __forceinline__ void add(float t /* = y - m, <= ~0 */)
+    {
+        float e = ex2(t);
+        s += e;
+        u = fmaf(e, t, u);
+    }
+};
+
+__device__ __forceinline__ SoftmaxState merge(const SoftmaxState &a, const SoftmaxState &b)
+{
+    SoftmaxState r;
+    r.m = fmaxf(a.m, b.m);
+    float da = a.m - r.m, db = b.m - r.m;
+    float ea = ex2(da), eb = ex2(db);
+    r.s = fmaf(a.s, ea, b.s * eb);
+    r.u = fmaf(ea, fmaf(da, a.s, a.u), eb * fmaf(db, b.s, b.u));
+    return r;
+}
+
+__device__ __forceinline__ SoftmaxState warp_merge(SoftmaxState st)
+{
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        SoftmaxState o;
+        o.m = __shfl_xor_sync(0xffffffffu, st.m, off);
+        o.s = __shfl_xor_sync(0xffffffffu, st.s, off);
+        o.u = __shfl_xor_sync(0xffffffffu, st.u, off);
+        st = merge(st, o);
+    }
+    return st;
+}
+
+// Block-wide merge; `red` holds 3*32 floats. Result is returned to every thread.
+template <int THREADS>
+__device__ __forceinline__ SoftmaxState block_merge(SoftmaxState st, float *red)
+{
+    constexpr int WARPS = THREADS / 32;
+    st = warp_merge(st);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (WARPS > 1) {
+        if (lane == 0) {
+            red[warp] = st.m;
+            red[32 + warp] = st.s;
+            red[64 + warp] = st.u;
+        }
+        __syncthreads();
+        SoftmaxState t;
+        if (lane < WARPS) {
+            t.m = red[lane];
+            t.s = red[32 + lane];
+            t.u = red[64 + lane];
+        } else {
+            t.init();
+        }
+        st = warp_merge(t);
+        __syncthreads();   // red may be reused by the caller's next row
+    }
+    return st;
+}
+
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    return v;
+}
+
+// Block-wide fp64 sum in a fixed order; `red` holds 32 doubles. Result to every thread.
+template <int THREADS>
+__device__ __forceinline__ double block_sum(double v, double *red)
+{
+    constexpr int WARPS = THREADS / 32;
+    v = warp_sum(v);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    double t = (lane < WARPS) ? red[lane] : 0.0;
+    t = warp_sum(t);
+    __syncthreads();
+    return t;
+}
+
+// ---------------------------------------------------------------- per-token PPO loss terms
+struct TokenLoss {
+    float g;        // d loss / d new_logprob
+    float dvalue;   // d loss / d value
+    float pg, vf, kl, pg_clipped, vf_clipped;
+};
+
+// Clipped surrogate and clipped value loss of one real token (Table "PPO hyperparameters":
+// epsilon, epsilon-hat, c1, value-loss clipping on). Evaluated in fp64 from the fp32 inputs so
+// that the branch decisions do not depend on fp32 rounding of intermediate products.
+__device__ __forceinline__ TokenLoss token_loss(float lp_new, float lp_old, float adv, float v, float v_old,
+                                               float ret, float eps, float eps_v, float c1, double n)
+{
+    TokenLoss o;
+    const double A = adv;
+    const double lr = (double)lp_new - (double)lp_old;
+    const double rho = exp(lr);
+    const double lo = 1.0 - (double)eps, hi = 1.0 + (double)eps;
+    const double rc = rho < lo ? lo : (rho > hi ? hi : rho);
+    const double l1 = -A * rho, l2 = -A * rc;
+    const bool pclip = l2 > l1;
+    o.pg = (float)(pclip ? l2 : l1);
+    o.g = pclip ? 0.f : (float)(l1 / n);
+    o.pg_clipped = pclip ? 1.f : 0.f;
+    o.kl = (float)(0.5 * lr * lr);
+    const double dv = v, dvo = v_old, dr = ret;
+    const double vlo = dvo - (double)eps_v, vhi = dvo + (double)eps_v;
+    const double vc = dv < vlo ? vlo : (dv > vhi ? vhi : dv);
+    const double e1 = (dv - dr) * (dv - dr), e2 = (vc - dr) * (vc - dr);
+    const bool vclip = e2 > e1;
+    o.vf = (float)(vclip ? e2 : e1);
+    o.vf_clipped = vclip ? 1.f : 0.f;
+    o.dvalue = vclip ? 0.f : (float)((double)c1 * (dv - dr) / n);
+    return o;
+}
+
+// launchers shared between translation units
+int launch_count_mask(const uint8_t *mask, int64_t n_elems, void *workspace, cudaStream_t s);
+int launch_loss_finalize(int64_t rows, float vf_coef, float *losses, void *workspace, cudaStream_t s);
+
+// tuning options (ppo_set_option)
+int option_value(int key);
+
+}   // namespace ppo

@@ -1,0 +1,444 @@
+// Row kernels: the two steps that stream the [rows, V] logits.
+//   ppo_logprob_entropy  -- one read of every row (single-pass online softmax statistics)
+//   ppo_loss_fwd_bwd     -- one read and one write of every real row: the row is parked in
+//                           shared memory between the statistics pass and the gradient pass
+// One thread block owns one row at a time; 128-bit coalesced loads/stores; fp32 accumulation
+// in base-2 units (one ex2 per element); warp-shuffle + shared-memory merge of the running
+// (max, sum, sum*log) states; per-token scalar math in fp64 by one thread.
+#include "ppo_common.cuh"
+
+namespace ppo {
+
+// ---------------------------------------------------------------- element packs
+// A "pack" is one 16-byte vector: 8 bf16 or 4 fp32 logits.
+template <typename T> struct Pack;
+
+template <> struct Pack<float> {
+    static constexpr int N = 4;
+    static __device__ __forceinline__ float clampf(float x) { return (x != x) ? x : fmaxf(x, kNegBig); }
+    static __device__ __forceinline__ void unpack(const uint4 &v, float (&x)[4], float &xmax)
+    {
+        // fmaxf drops NaN; clampf keeps it so a NaN logit poisons the row as documented
+        x[0] = clampf(__uint_as_float(v.x));
+        x[1] = clampf(__uint_as_float(v.y));
+        x[2] = clampf(__uint_as_float(v.z));
+        x[3] = clampf(__uint_as_float(v.w));
+        xmax = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+    }
+    static __device__ __forceinline__ uint4 pack(const float (&d)[4])
+    {
+        return make_uint4(__float_as_uint(d[0]), __float_as_uint(d[1]), __float_as_uint(d[2]),
+                          __float_as_uint(d[3]));
+    }
+    static __device__ __forceinline__ float load1(const float *p) { return *p; }
+    static __device__ __forceinline__ void store1(float *p, float v) { *p = v; }
+};
+
+template <> struct Pack<__nv_bfloat16> {
+    static constexpr int N = 8;
+    static __device__ __forceinline__ __nv_bfloat162 as2(uint32_t w)
+    {
+        return *reinterpret_cast<__nv_bfloat162 *>(&w);
+    }
+    static __device__ __forceinline__ uint32_t bits(__nv_bfloat162 h) { return *reinterpret_cast<uint32_t *>(&h); }
+    static __device__ __forceinline__ void unpack(const uint4 &v, float (&x)[8], float &xmax)
+    {
+        const __nv_bfloat162 lim = __float2bfloat162_rn(kNegBig);
+        const __nv_bfloat162 h0 = __hmax2_nan(as2(v.x), lim), h1 = __hmax2_nan(as2(v.y), lim),
+                             h2 = __hmax2_nan(as2(v.z), lim), h3 = __hmax2_nan(as2(v.w), lim);
+        const __nv_bfloat162 hm = __hmax2(__hmax2(h0, h1), __hmax2(h2, h3));
+        xmax = fmaxf(__low2float(hm), __high2float(hm));
+        const uint32_t w0 = bits(h0), w1 = bits(h1), w2 = bits(h2), w3 = bits(h3);
+        x[0] = __uint_as_float(w0 << 16); x[1] = __uint_as_float(w0 & 0xffff0000u);
+        x[2] = __uint_as_float(w1 << 16); x[3] = __uint_as_float(w1 & 0xffff0000u);
+        x[4] = __uint_as_float(w2 << 16); x[5] = __uint_as_float(w2 & 0xffff0000u);
+        x[6] = __uint_as_float(w3 << 16); x[7] = __uint_as_float(w3 & 0xffff0000u);
+    }
+    static __device__ __forceinline__ uint4 pack(const float (&d)[8])
+    {
+        return make_uint4(bits(__floats2bfloat162_rn(d[0], d[1])), bits(__floats2bfloat162_rn(d[2], d[3])),
+                          bits(__floats2bfloat162_rn(d[4], d[5])), bits(__floats2bfloat162_rn(d[6], d[7])));
+    }
+    static __device__ __forceinline__ float load1(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
+    static __device__ __forceinline__ void store1(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
+};
+
+// streaming 16-byte global accesses (data is touched once: evict-first)
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p) { return __ldcs(p); }
+__device__ __forceinline__ void st_stream(uint4 *p, const uint4 &v) { __stcs(p, v); }
+
+// fold one pack into the running state
+template <typename T>
+__device__ __forceinline__ void accumulate(const uint4 &v, float c, SoftmaxState &st)
+{
+    float x[Pack<T>::N], xmax;
+    Pack<T>::unpack(v, x, xmax);
+    const float ymax = xmax * c;
+    if (ymax > st.m) st.rebase(ymax);
+    const float nm = -st.m;
+    float s1 = 0.f, u1 = 0.f;   // second accumulator pair: two independent add chains
+#pragma unroll
+    for (int k = 0; k < Pack<T>::N; k += 2) {
+        const float t0 = fmaf(x[k], c, nm), t1 = fmaf(x[k + 1], c, nm);
+        const float e0 = ex2(t0), e1 = ex2(t1);
+        st.s += e0;
+        st.u = fmaf(e0, t0, st.u);
+        s1 += e1;
+        u1 = fmaf(e1, t1, u1);
+    }
+    st.s += s1;
+    st.u += u1;
+}
+
+// Statistics pass over one row. VECTOR: 16-byte packs (row base 16-byte aligned, V % N == 0);
+// otherwise element by element. STAGE: also park the raw packs / elements in shared memory.
+template <typename T, bool VECTOR, bool STAGE, int THREADS, int UNROLL>
+__device__ __forceinline__ SoftmaxState row_statistics(const T *__restrict__ src, int V, float c, void *stage)
+{
+    SoftmaxState st;
+    st.init();
+    if (VECTOR) {
+        constexpr int N = Pack<T>::N;
+        const uint4 *src4 = reinterpret_cast<const uint4 *>(src);
+        uint4 *stage4 = reinterpret_cast<uint4 *>(stage);
+        const int nvec = V / N;
+        int i = threadIdx.x;
+        for (; i + (UNROLL - 1) * THREADS < nvec; i += UNROLL * THREADS) {
+            uint4 v[UNROLL];
+#pragma unroll
+            for (int k = 0; k < UNROLL; ++k) v[k] = ld_stream(src4 + i + k * THREADS);
+#pragma unroll
+            for (int k = 0; k < UNROLL; ++k) {
+                if (STAGE) stage4[i + k * THREADS] = v[k];
+                accumulate<T>(v[k], c, st);
+            }
+        }
+        for (; i < nvec; i += THREADS) {
+            const uint4 v = ld_stream(src4 + i);
+            if (STAGE) stage4[i] = v;
+            accumulate<T>(v, c, st);
+        }
+    } else {
+        T *stage1 = reinterpret_cast<T *>(stage);
+        for (int j = threadIdx.x; j < V; j += THREADS) {
+            const T raw = src[j];
+            if (STAGE) stage1[j] = raw;
+            float x = Pack<T>::load1(&raw);
+            x = (x != x) ? x : fmaxf(x, kNegBig);
+            const float y = x * c;
+            if (y > st.m) st.rebase(y);
+            st.add(fmaf(x, c, -st.m));
+        }
+    }
+    return st;
+}
+
+// ---------------------------------------------------------------- step 1 kernel
+template <typename T, bool VECTOR, int THREADS>
+__global__ void __launch_bounds__(THREADS)
+logprob_entropy_kernel(const T *__restrict__ logits, int64_t rows, int V, int64_t row_stride,
+                       const int32_t *__restrict__ tokens, const uint8_t *__restrict__ mask, float c,
+                       float *__restrict__ logprob, float *__restrict__ entropy, float *__restrict__ lse,
+                       int *status)
+{
+    __shared__ float red[96];
+    for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
+        if (mask && !mask[row]) {
+            if (threadIdx.x == 0) {
+                logprob[row] = 0.f;
+                if (entropy) entropy[row] = 0.f;
+                if (lse) lse[row] = 0.f;
+            }
+            continue;
+        }
+        const T *src = logits + row * row_stride;
+        const int tok = tokens[row];
+        const bool bad = tok < 0 || tok >= V;
+        float xtok = 0.f;
+        if (threadIdx.x == 0 && !bad) xtok = Pack<T>::load1(src + tok);
+        SoftmaxState st = row_statistics<T, VECTOR, false, THREADS, 4>(src, V, c, nullptr);
+        st = block_merge<THREADS>(st, red);
+        if (threadIdx.x == 0) {
+            const float l2s = log2f(st.s);
+            float lp = (fmaf(xtok, c, -st.m) - l2s) * kLn2;
+            float H = (l2s - st.u / st.s) * kLn2;
+            float L = (st.m + l2s) * kLn2;
+            if (bad) {
+                lp = H = L = __int_as_float(0x7fc00000);
+                if (status) atomicOr(status, PPO_DEV_BAD_TOKEN);
+            }
+            logprob[row] = lp;
+            if (entropy) entropy[row] = H;
+            if (lse) lse[row] = L;
+        }
+    }
+}
+
+// ---------------------------------------------------------------- step 6 kernel
+struct LossArgs {
+    const void *logits;
+    void *dlogits;
+    int64_t rows;
+    int V;
+    const int32_t *tokens;
+    const uint8_t *mask;
+    const float *old_logprob, *advantages, *values_new, *values_old, *returns;
+    float *dvalues, *new_logprob, *entropy, *dlogprob;
+    float *partials;
+    const int *n_tokens;
+    int *status;
+    float c;        // log2(e) / temperature
+    float inv_tau;  // 1 / temperature
+    float eps, eps_v, c1;
+};
+
+template <typename T, bool VECTOR, int THREADS>
+__device__ __forceinline__ void fill_row_zero(T *dst, int V)
+{
+    if (VECTOR) {
+        uint4 *d4 = reinterpret_cast<uint4 *>(dst);
+        const int nvec = V / Pack<T>::N;
+        const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+        for (int i = threadIdx.x; i < nvec; i += THREADS) st_stream(d4 + i, z);
+    } else {
+        for (int j = threadIdx.x; j < V; j += THREADS) Pack<T>::store1(dst + j, 0.f);
+    }
+}
+
+// ROW_IN_SMEM: pass 2 reads the row back from shared memory (every thread re-reads exactly the
+// packs it parked itself); otherwise it re-reads global memory (served by L2 when the row is
+// still resident there).
+template <typename T, bool VECTOR, bool ROW_IN_SMEM, int THREADS>
+__global__ void __launch_bounds__(THREADS)
+loss_rows_kernel(const LossArgs a)
+{
+    extern __shared__ uint4 row_stage[];
+    __shared__ float red[96];
+    __shared__ float bc[2];
+    const T *logits = reinterpret_cast<const T *>(a.logits);
+    T *dlogits = reinterpret_cast<T *>(a.dlogits);
+    const int V = a.V;
+    const double n = (double)(*a.n_tokens);
+
+    for (int64_t row = blockIdx.x; row < a.rows; row += gridDim.x) {
+        T *dst = dlogits ? dlogits + row * (int64_t)V : nullptr;
+        float *part = a.partials + row * kPartialsPerToken;
+        if (!a.mask[row]) {
+            if (dst) fill_row_zero<T, VECTOR, THREADS>(dst, V);
+            if (threadIdx.x == 0) {
+                a.dvalues[row] = 0.f;
+                if (a.new_logprob) a.new_logprob[row] = 0.f;
+                if (a.entropy) a.entropy[row] = 0.f;
+                if (a.dlogprob) a.dlogprob[row] = 0.f;
+                float4 *p4 = reinterpret_cast<float4 *>(part);
+                p4[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+                p4[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            continue;
+        }
+        const T *src = logits + row * (int64_t)V;
+        const int tok = a.tokens[row];
+        const bool bad = tok < 0 || tok >= V;
+        float xtok = 0.f;
+        if (threadIdx.x == 0 && !bad) xtok = Pack<T>::load1(src + tok);
+        SoftmaxState st = row_statistics<T, VECTOR, ROW_IN_SMEM, THREADS, 4>(src, V, a.c, row_stage);
+        st = block_merge<THREADS>(st, red);
+        if (threadIdx.x == 0) {
+            const float l2s = log2f(st.s);
+            float lp = (fmaf(xtok, a.c, -st.m) - l2s) * kLn2;
+            float H = (l2s - st.u / st.s) * kLn2;
+            if (bad) {
+                lp = H = __int_as_float(0x7fc00000);
+                if (a.status) atomicOr(a.status, PPO_DEV_BAD_TOKEN);
+            }
+            const TokenLoss tl = token_loss(lp, a.old_logprob[row], a.advantages[row], a.values_new[row],
+                                            a.values_old[row], a.returns[row], a.eps, a.eps_v, a.c1, n);
+            a.dvalues[row] = tl.dvalue;
+            if (a.new_logprob) a.new_logprob[row] = lp;
+            if (a.entropy) a.entropy[row] = H;
+            if (a.dlogprob) a.dlogprob[row] = tl.g;
+            float4 *p4 = reinterpret_cast<float4 *>(part);
+            p4[0] = make_float4(tl.pg, tl.vf, tl.kl, tl.pg_clipped);
+            p4[1] = make_float4(tl.vf_clipped, H, 0.f, 0.f);
+            bc[0] = st.m + l2s;          // log2-sum-exp
+            bc[1] = tl.g * a.inv_tau;    // gradient scale
+        }
+        __syncthreads();
+        const float Y = bc[0], gs = bc[1];
+        if (dst) {
+            if (gs == 0.f) {
+                fill_row_zero<T, VECTOR, THREADS>(dst, V);
+            } else {
+                const float ngs = -gs;
+                if (VECTOR) {
+                    constexpr int N = Pack<T>::N;
+                    const uint4 *src4 = ROW_IN_SMEM ? row_stage : reinterpret_cast<const uint4 *>(src);
+                    uint4 *dst4 = reinterpret_cast<uint4 *>(dst);
+                    const int nvec = V / N;
+                    const float nY = -Y;
+#pragma unroll 2
+                    for (int i = threadIdx.x; i < nvec; i += THREADS) {
+                        const uint4 v = src4[i];
+                        float x[N], xmax, d[N];
+                        Pack<T>::unpack(v, x, xmax);
+#pragma unroll
+                        for (int k = 0; k < N; ++k) d[k] = ngs * ex2(fmaf(x[k], a.c, nY));
+                        st_stream(dst4 + i, Pack<T>::pack(d));
+                    }
+                    // the thread that wrote the pack holding the sampled token adds the one-hot term
+                    if (!bad && threadIdx.x == (tok / N) % THREADS) {
+                        const float xt = Pack<T>::load1(src + tok);
+                        Pack<T>::store1(dst + tok, fmaf(ngs, ex2(fmaf(xt, a.c, nY)), gs));
+                    }
+                } else {
+                    const T *src1 = ROW_IN_SMEM ? reinterpret_cast<const T *>(row_stage) : src;
+                    for (int j = threadIdx.x; j < V; j += THREADS) {
+                        float x = Pack<T>::load1(src1 + j);
+                        x = (x != x) ? x : fmaxf(x, kNegBig);
+                        float d = ngs * ex2(fmaf(x, a.c, -Y));
+                        if (j == tok) d += gs;
+                        Pack<T>::store1(dst + j, d);
+                    }
+                }
+            }
+        }
+        __syncthreads();   // bc and the staged row are reused by the next row
+    }
+}
+
+// ---------------------------------------------------------------- host side
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+template <typename T>
+static int launch_logprob(const void *logits, int64_t rows, int V, int64_t row_stride, const int32_t *tokens,
+                          const uint8_t *mask, float c, float *logprob, float *entropy, float *lse, int *status,
+                          cudaStream_t s)
+{
+    constexpr int THREADS = 256;
+    const bool vec = aligned16(logits) && (row_stride * sizeof(T)) % 16 == 0 && V % Pack<T>::N == 0;
+    const unsigned grid = (unsigned)(rows < (int64_t)1 << 30 ? rows : (int64_t)1 << 30);
+    const T *lg = reinterpret_cast<const T *>(logits);
+    if (vec)
+        logprob_entropy_kernel<T, true, THREADS><<<grid, THREADS, 0, s>>>(lg, rows, V, row_stride, tokens, mask, c,
+                                                                           logprob, entropy, lse, status);
+    else
+        logprob_entropy_kernel<T, false, THREADS><<<grid, THREADS, 0, s>>>(lg, rows, V, row_stride, tokens, mask, c,
+                                                                            logprob, entropy, lse, status);
+    return launch_status();
+}
+
+constexpr size_t kMaxDynSmem = 227 * 1024;
+
+template <typename T, bool VECTOR, bool ROW_IN_SMEM, int THREADS>
+static int launch_loss_variant(const LossArgs &a, size_t smem, cudaStream_t s)
+{
+    auto kern = loss_rows_kernel<T, VECTOR, ROW_IN_SMEM, THREADS>;
+    if (smem > 48 * 1024)
+        PPO_RETURN_IF_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const unsigned grid = (unsigned)(a.rows < (int64_t)1 << 30 ? a.rows : (int64_t)1 << 30);
+    kern<<<grid, THREADS, smem, s>>>(a);
+    return launch_status();
+}
+
+template <typename T>
+static int launch_loss(const LossArgs &a, cudaStream_t s)
+{
+    const bool vec = aligned16(a.logits) && (a.dlogits == nullptr || aligned16(a.dlogits)) &&
+                     a.V % Pack<T>::N == 0;
+    const size_t row_bytes = (size_t)a.V * sizeof(T);
+    // Two blocks per SM when the row is small enough (they overlap each other's load, compute
+    // and store phases); one big block per SM while the row still fits; else re-read via L2.
+    const int mode = option_value(PPO_OPT_LOSS_ROW_CACHE);
+    const bool fits2 = row_bytes <= 112 * 1024, fits1 = row_bytes + 1024 <= kMaxDynSmem;
+    bool in_smem = a.dlogits != nullptr && (fits2 || fits1);
+    if (mode == 1) in_smem = fits1;
+    if (mode == 2) in_smem = false;
+    if (in_smem) {
+        if (fits2) {
+            return vec ? launch_loss_variant<T, true, true, 512>(a, row_bytes, s)
+                       : launch_loss_variant<T, false, true, 512>(a, row_bytes, s);
+        }
+        return vec ? launch_loss_variant<T, true, true, 1024>(a, row_bytes, s)
+                   : launch_loss_variant<T, false, true, 1024>(a, row_bytes, s);
+    }
+    return vec ? launch_loss_variant<T, true, false, 512>(a, 0, s)
+               : launch_loss_variant<T, false, false, 512>(a, 0, s);
+}
+
+}   // namespace ppo
+
+using namespace ppo;
+
+extern "C" int ppo_logprob_entropy(const void *logits, int dtype, int64_t rows, int64_t V, int64_t row_stride,
+                                   const int32_t *tokens, const uint8_t *mask, float temperature,
+                                   float *logprob, float *entropy, float *lse, void *workspace, void *stream)
+{
+    if (dtype != PPO_F32 && dtype != PPO_BF16) return PPO_ERR_DTYPE;
+    if (rows < 0 || V <= 0 || V >= ((int64_t)1 << 31) || row_stride < V) return PPO_ERR_SHAPE;
+    if (!(temperature > 0.f) || !finite_f(temperature)) return PPO_ERR_PARAM;
+    if (rows == 0) return PPO_OK;
+    if (!logits || !tokens || !logprob) return PPO_ERR_NULL;
+    const size_t es = dtype == PPO_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(logits) % es) return PPO_ERR_ALIGN;
+    int *status = workspace ? &ws_header(workspace)->status : nullptr;
+    const float c = kLog2e / temperature;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    if (dtype == PPO_F32)
+        return launch_logprob<float>(logits, rows, (int)V, row_stride, tokens, mask, c, logprob, entropy, lse,
+                                     status, s);
+    return launch_logprob<__nv_bfloat16>(logits, rows, (int)V, row_stride, tokens, mask, c, logprob, entropy, lse,
+                                         status, s);
+}
+
+extern "C" int ppo_loss_fwd_bwd(const void *logits, int dtype, int32_t B, int32_t T, int64_t V,
+                                const int32_t *tokens, const uint8_t *mask, const float *old_logprob,
+                                const float *advantages, const float *values_new, const float *values_old,
+                                const float *returns, const ppo_params *p, float *losses, void *dlogits,
+                                float *dvalues, float *new_logprob, float *entropy, float *dlogprob,
+                                void *workspace, void *stream)
+{
+    if (dtype != PPO_F32 && dtype != PPO_BF16) return PPO_ERR_DTYPE;
+    if (B <= 0 || T <= 0 || V <= 0 || V >= ((int64_t)1 << 31)) return PPO_ERR_SHAPE;
+    if (!logits || !tokens || !mask || !old_logprob || !advantages || !values_new || !values_old || !returns ||
+        !p || !losses || !dvalues || !workspace)
+        return PPO_ERR_NULL;
+    if (!(p->temperature > 0.f) || !finite_f(p->temperature) || !(p->cliprange >= 0.f) ||
+        !(p->cliprange_value >= 0.f) || !finite_f(p->vf_coef))
+        return PPO_ERR_PARAM;
+    const size_t es = dtype == PPO_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(logits) % es || reinterpret_cast<uintptr_t>(dlogits) % es ||
+        reinterpret_cast<uintptr_t>(workspace) % 256)
+        return PPO_ERR_ALIGN;
+    if (dlogits == logits) return PPO_ERR_PARAM;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const int64_t rows = (int64_t)B * T;
+    int rc = launch_count_mask(mask, rows, workspace, s);
+    if (rc) return rc;
+    LossArgs a;
+    a.logits = logits;
+    a.dlogits = dlogits;
+    a.rows = rows;
+    a.V = (int)V;
+    a.tokens = tokens;
+    a.mask = mask;
+    a.old_logprob = old_logprob;
+    a.advantages = advantages;
+    a.values_new = values_new;
+    a.values_old = values_old;
+    a.returns = returns;
+    a.dvalues = dvalues;
+    a.new_logprob = new_logprob;
+    a.entropy = entropy;
+    a.dlogprob = dlogprob;
+    a.partials = ws_partials(workspace);
+    a.n_tokens = &ws_header(workspace)->n_tokens;
+    a.status = &ws_header(workspace)->status;
+    a.c = kLog2e / p->temperature;
+    a.inv_tau = 1.0f / p->temperature;
+    a.eps = p->cliprange;
+    a.eps_v = p->cliprange_value;
+    a.c1 = p->vf_coef;
+    rc = dtype == PPO_F32 ? launch_loss<float>(a, s) : launch_loss<__nv_bfloat16>(a, s);
+    if (rc) return rc;
+    return launch_loss_finalize(rows, p->vf_coef, losses, workspace, s);
+}

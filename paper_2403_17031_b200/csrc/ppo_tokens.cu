@@ -1,0 +1,380 @@
+// Token-level kernels: everything that touches only [B,T]-sized arrays (steps 2-5, the loss
+// reductions, workspace and status plumbing). These move <0.1% of the path's bytes and are
+// bound by launch latency; each is a single small launch.
+#include "ppo_common.cuh"
+
+namespace ppo {
+
+static int g_options[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+int option_value(int key) { return (key >= 0 && key < 8) ? g_options[key] : 0; }
+
+// ---------------------------------------------------------------- step 2: EOS trick
+// One warp per response: lanes stride over t, a warp-wide min finds the first EOS.
+__global__ void __launch_bounds__(128)
+truncate_kernel(const int32_t *responses, int B, int T, int eos_id, int pad_id,
+                const float *__restrict__ scores, float no_eos_score, int32_t *responses_out,
+                int32_t *__restrict__ eos_index, int32_t *__restrict__ seq_len, uint8_t *__restrict__ mask,
+                float *__restrict__ scores_out)
+{
+    const int b = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
+    const int lane = threadIdx.x & 31;
+    if (b >= B) return;
+    const int32_t *r = responses + (int64_t)b * T;
+    int first = T;
+    for (int t = lane; t < T; t += 32)
+        if (r[t] == eos_id) { first = t; break; }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) first = min(first, __shfl_xor_sync(0xffffffffu, first, off));
+    const int e = first < T ? first : -1;
+    const int L = first < T ? first + 1 : T;
+    for (int t = lane; t < T; t += 32) {
+        const int64_t i = (int64_t)b * T + t;
+        const int32_t tok = r[t];
+        if (responses_out) responses_out[i] = t < L ? tok : pad_id;
+        if (mask) mask[i] = (uint8_t)(t < L);
+    }
+    if (lane == 0) {
+        if (eos_index) eos_index[b] = e;
+        if (seq_len) seq_len[b] = L;
+        if (scores_out) scores_out[b] = e >= 0 ? scores[b] : no_eos_score;
+    }
+}
+
+// ---------------------------------------------------------------- step 3: KL rewards
+__global__ void __launch_bounds__(256)
+kl_rewards_kernel(const float *__restrict__ logprob, const float *__restrict__ ref_logprob,
+                  const uint8_t *__restrict__ mask, const int32_t *__restrict__ seq_len,
+                  const float *__restrict__ scores, int B, int T, float kl_coef, float *__restrict__ kl,
+                  float *__restrict__ rewards)
+{
+    const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (i >= (int64_t)B * T) return;
+    const int b = (int)(i / T), t = (int)(i - (int64_t)b * T);
+    const float k = mask[i] ? logprob[i] - ref_logprob[i] : 0.f;
+    if (kl) kl[i] = k;
+    if (rewards) {
+        float r = mask[i] ? -kl_coef * k : 0.f;
+        if (t == seq_len[b] - 1) r += scores[b];
+        rewards[i] = r;
+    }
+}
+
+// ---------------------------------------------------------------- step 4: GAE
+// One warp per sequence. Lane l owns the contiguous time segment [l*S, (l+1)*S); running the
+// recurrence A_t = delta_t + c*A_{t+1} over a segment is an affine map of the incoming A, so
+// (1) each lane folds its segment into (a, b), (2) a reverse inclusive warp scan composes the
+// maps, (3) each lane replays its segment from the correct incoming value. fp64 throughout.
+__global__ void __launch_bounds__(128)
+gae_kernel(const float *__restrict__ rewards, const float *__restrict__ values,
+           const int32_t *__restrict__ seq_len, int B, int T, double gamma, double c /* gamma*lam */,
+           float *__restrict__ advantages, float *__restrict__ returns)
+{
+    const int b = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
+    const int lane = threadIdx.x & 31;
+    if (b >= B) return;
+    int L = seq_len[b];
+    L = L < 0 ? 0 : (L > T ? T : L);
+    const float *r = rewards + (int64_t)b * T;
+    const float *v = values + (int64_t)b * T;
+    const int S = (T + 31) / 32;
+    const int s0 = min(lane * S, T), s1 = min(s0 + S, T);
+
+    double a = 1.0, bb = 0.0;
+    for (int t = s1 - 1; t >= s0; --t) {
+        double d = 0.0;
+        if (t < L) {
+            const double vn = (t + 1 < L) ? (double)v[t + 1] : 0.0;
+            d = ((double)r[t] + gamma * vn) - (double)v[t];
+        }
+        bb = d + c * bb;
+        a = c * a;
+    }
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const double aj = __shfl_down_sync(0xffffffffu, a, off);
+        const double bj = __shfl_down_sync(0xffffffffu, bb, off);
+        if (lane + off < 32) {
+            bb = bb + a * bj;
+            a = a * aj;
+        }
+    }
+    double A = __shfl_down_sync(0xffffffffu, bb, 1);
+    if (lane == 31) A = 0.0;
+    for (int t = s1 - 1; t >= s0; --t) {
+        const int64_t i = (int64_t)b * T + t;
+        if (t < L) {
+            const double vn = (t + 1 < L) ? (double)v[t + 1] : 0.0;
+            const double d = ((double)r[t] + gamma * vn) - (double)v[t];
+            A = d + c * A;
+            advantages[i] = (float)A;
+            returns[i] = (float)(A + (double)v[t]);
+        } else {
+            A = c * A;
+            advantages[i] = 0.f;
+            returns[i] = 0.f;
+        }
+    }
+}
+
+// ---------------------------------------------------------------- step 5: masked whitening
+// One block: three passes over the (L1/L2-resident) array, fp64 sums in a fixed order.
+constexpr int kWhitenThreads = 1024;
+__global__ void __launch_bounds__(kWhitenThreads)
+whiten_kernel(const float *x, const uint8_t *__restrict__ mask, int64_t n_elems, int shift_mean, float eps,
+              float *out, float *__restrict__ stats3, int *status)
+{
+    __shared__ double red[32];
+    double sum = 0.0, cnt = 0.0;
+    for (int64_t i = threadIdx.x; i < n_elems; i += kWhitenThreads)
+        if (!mask || mask[i]) { sum += (double)x[i]; cnt += 1.0; }
+    sum = block_sum<kWhitenThreads>(sum, red);
+    cnt = block_sum<kWhitenThreads>(cnt, red);
+    const double mean = cnt > 0.0 ? sum / cnt : 0.0;
+    double ss = 0.0;
+    for (int64_t i = threadIdx.x; i < n_elems; i += kWhitenThreads)
+        if (!mask || mask[i]) { const double d = (double)x[i] - mean; ss += d * d; }
+    ss = block_sum<kWhitenThreads>(ss, red);
+    const double var = cnt > 0.0 ? ss / cnt : 0.0;
+    const double inv = 1.0 / sqrt(var + (double)eps);
+    const double back = shift_mean ? 0.0 : mean;
+    for (int64_t i = threadIdx.x; i < n_elems; i += kWhitenThreads) {
+        float y = 0.f;
+        if (!mask || mask[i]) y = (float)(((double)x[i] - mean) * inv + back);
+        out[i] = y;
+    }
+    if (threadIdx.x == 0) {
+        if (stats3) { stats3[0] = (float)mean; stats3[1] = (float)var; stats3[2] = (float)cnt; }
+        if (cnt == 0.0 && status) atomicOr(status, PPO_DEV_EMPTY_MASK);
+    }
+}
+
+// ---------------------------------------------------------------- loss plumbing
+constexpr int kReduceThreads = 1024;
+
+__global__ void __launch_bounds__(kReduceThreads)
+count_mask_kernel(const uint8_t *__restrict__ mask, int64_t n_elems, WorkspaceHeader *hdr)
+{
+    __shared__ int red[32];
+    int c = 0;
+    for (int64_t i = threadIdx.x; i < n_elems; i += kReduceThreads) c += mask[i] ? 1 : 0;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) c += __shfl_xor_sync(0xffffffffu, c, off);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = c;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        c = red[threadIdx.x];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) c += __shfl_xor_sync(0xffffffffu, c, off);
+        if (threadIdx.x == 0) {
+            hdr->n_tokens = c;
+            if (c == 0) atomicOr(&hdr->status, PPO_DEV_EMPTY_MASK);
+        }
+    }
+}
+
+// Sum the per-token partials (fixed thread assignment, fp64) and write the eight loss scalars.
+__global__ void __launch_bounds__(kReduceThreads)
+loss_finalize_kernel(const float *__restrict__ partials, int64_t rows, const WorkspaceHeader *hdr, float vf_coef,
+                     float *__restrict__ losses)
+{
+    __shared__ double red[32];
+    double acc[6] = {0, 0, 0, 0, 0, 0};
+    for (int64_t r = threadIdx.x; r < rows; r += kReduceThreads) {
+        const float4 p0 = reinterpret_cast<const float4 *>(partials + r * kPartialsPerToken)[0];
+        const float4 p1 = reinterpret_cast<const float4 *>(partials + r * kPartialsPerToken)[1];
+        acc[0] += p0.x; acc[1] += p0.y; acc[2] += p0.z; acc[3] += p0.w; acc[4] += p1.x; acc[5] += p1.y;
+    }
+#pragma unroll
+    for (int k = 0; k < 6; ++k) acc[k] = block_sum<kReduceThreads>(acc[k], red);
+    if (threadIdx.x == 0) {
+        const double n = (double)hdr->n_tokens;
+        const double inv = n > 0.0 ? 1.0 / n : 0.0;
+        const double pg = acc[0] * inv, vf = 0.5 * acc[1] * inv;
+        losses[PPO_LOSS_PG] = (float)pg;
+        losses[PPO_LOSS_VF] = (float)vf;
+        losses[PPO_LOSS_TOTAL] = (float)(pg + (double)vf_coef * vf);
+        losses[PPO_LOSS_APPROX_KL] = (float)(acc[2] * inv);
+        losses[PPO_LOSS_PG_CLIPFRAC] = (float)(acc[3] * inv);
+        losses[PPO_LOSS_VF_CLIPFRAC] = (float)(acc[4] * inv);
+        losses[PPO_LOSS_ENTROPY] = (float)(acc[5] * inv);
+        losses[PPO_LOSS_N] = (float)n;
+    }
+}
+
+// Step 6 at log-prob level (the logits were never materialised): one thread per token.
+__global__ void __launch_bounds__(256)
+loss_from_logprob_kernel(const float *__restrict__ new_logprob, const float *__restrict__ entropy, int64_t rows,
+                         const uint8_t *__restrict__ mask, const float *__restrict__ old_logprob,
+                         const float *__restrict__ advantages, const float *__restrict__ values_new,
+                         const float *__restrict__ values_old, const float *__restrict__ returns, float eps,
+                         float eps_v, float c1, const WorkspaceHeader *hdr, float *__restrict__ partials,
+                         float *__restrict__ dlogprob, float *__restrict__ dvalues)
+{
+    const int64_t r = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (r >= rows) return;
+    float4 p0 = make_float4(0.f, 0.f, 0.f, 0.f), p1 = make_float4(0.f, 0.f, 0.f, 0.f);
+    float g = 0.f, dv = 0.f;
+    if (mask[r]) {
+        const TokenLoss tl = token_loss(new_logprob[r], old_logprob[r], advantages[r], values_new[r],
+                                        values_old[r], returns[r], eps, eps_v, c1, (double)hdr->n_tokens);
+        p0 = make_float4(tl.pg, tl.vf, tl.kl, tl.pg_clipped);
+        p1 = make_float4(tl.vf_clipped, entropy ? entropy[r] : 0.f, 0.f, 0.f);
+        g = tl.g;
+        dv = tl.dvalue;
+    }
+    reinterpret_cast<float4 *>(partials + r * kPartialsPerToken)[0] = p0;
+    reinterpret_cast<float4 *>(partials + r * kPartialsPerToken)[1] = p1;
+    if (dlogprob) dlogprob[r] = g;
+    dvalues[r] = dv;
+}
+
+int launch_count_mask(const uint8_t *mask, int64_t n_elems, void *workspace, cudaStream_t s)
+{
+    count_mask_kernel<<<1, kReduceThreads, 0, s>>>(mask, n_elems, ws_header(workspace));
+    return launch_status();
+}
+
+int launch_loss_finalize(int64_t rows, float vf_coef, float *losses, void *workspace, cudaStream_t s)
+{
+    loss_finalize_kernel<<<1, kReduceThreads, 0, s>>>(ws_partials(workspace), rows, ws_header(workspace), vf_coef,
+                                                      losses);
+    return launch_status();
+}
+
+}   // namespace ppo
+
+using namespace ppo;
+
+extern "C" void ppo_default_params(ppo_params *p)
+{
+    if (!p) return;
+    p->temperature = 0.7f;
+    p->kl_coef = 0.05f;
+    p->gamma = 1.0f;
+    p->lam = 0.95f;
+    p->cliprange = 0.2f;
+    p->cliprange_value = 0.2f;
+    p->vf_coef = 0.1f;
+    p->no_eos_score = -1.0f;
+    p->whiten_eps = 1e-8f;
+    p->eos_id = 0;
+    p->pad_id = 1;
+}
+
+extern "C" int ppo_version(void) { return 100; }
+
+extern "C" int ppo_set_option(int key, int value)
+{
+    if (key == PPO_OPT_LOSS_ROW_CACHE && value >= 0 && value <= 2) {
+        g_options[key] = value;
+        return PPO_OK;
+    }
+    return PPO_ERR_PARAM;
+}
+
+extern "C" size_t ppo_workspace_bytes(int32_t B, int32_t T, int64_t V)
+{
+    (void)V;
+    if (B <= 0 || T <= 0) return kHeaderBytes;
+    return kHeaderBytes + align256((size_t)B * (size_t)T * kPartialsPerToken * sizeof(float));
+}
+
+extern "C" int ppo_workspace_init(void *workspace, size_t bytes, void *stream)
+{
+    if (!workspace) return PPO_ERR_NULL;
+    if (bytes < kHeaderBytes) return PPO_ERR_SHAPE;
+    if (reinterpret_cast<uintptr_t>(workspace) % 256) return PPO_ERR_ALIGN;
+    PPO_RETURN_IF_CUDA(cudaMemsetAsync(workspace, 0, kHeaderBytes, reinterpret_cast<cudaStream_t>(stream)));
+    return PPO_OK;
+}
+
+extern "C" int ppo_last_device_status(void *workspace, void *stream, int *status)
+{
+    if (!workspace || !status) return PPO_ERR_NULL;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    PPO_RETURN_IF_CUDA(cudaMemcpyAsync(status, &ws_header(workspace)->status, sizeof(int), cudaMemcpyDeviceToHost, s));
+    PPO_RETURN_IF_CUDA(cudaMemsetAsync(&ws_header(workspace)->status, 0, sizeof(int), s));
+    PPO_RETURN_IF_CUDA(cudaStreamSynchronize(s));
+    return PPO_OK;
+}
+
+extern "C" int ppo_truncate_and_score(const int32_t *responses, int32_t B, int32_t T, int32_t eos_id,
+                                      int32_t pad_id, const float *scores, float no_eos_score,
+                                      int32_t *responses_out, int32_t *eos_index, int32_t *seq_len,
+                                      uint8_t *mask, float *scores_out, void *stream)
+{
+    if (B < 0 || T <= 0) return PPO_ERR_SHAPE;
+    if (eos_id == pad_id) return PPO_ERR_PARAM;
+    if (B == 0) return PPO_OK;
+    if (!responses || (scores_out && !scores)) return PPO_ERR_NULL;
+    const int warps_per_block = 4;
+    const unsigned grid = (unsigned)((B + warps_per_block - 1) / warps_per_block);
+    truncate_kernel<<<grid, 128, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+        responses, B, T, eos_id, pad_id, scores, no_eos_score, responses_out, eos_index, seq_len, mask, scores_out);
+    return launch_status();
+}
+
+extern "C" int ppo_kl_rewards(const float *logprob, const float *ref_logprob, const uint8_t *mask,
+                              const int32_t *seq_len, const float *scores, int32_t B, int32_t T,
+                              float kl_coef, float *kl, float *rewards, void *stream)
+{
+    if (B < 0 || T <= 0) return PPO_ERR_SHAPE;
+    if (!finite_f(kl_coef)) return PPO_ERR_PARAM;
+    if (B == 0) return PPO_OK;
+    if (!logprob || !ref_logprob || !mask || (!kl && !rewards) || (rewards && (!seq_len || !scores)))
+        return PPO_ERR_NULL;
+    const int64_t n = (int64_t)B * T;
+    kl_rewards_kernel<<<(unsigned)((n + 255) / 256), 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+        logprob, ref_logprob, mask, seq_len, scores, B, T, kl_coef, kl, rewards);
+    return launch_status();
+}
+
+extern "C" int ppo_gae(const float *rewards, const float *values, const int32_t *seq_len, int32_t B, int32_t T,
+                       float gamma, float lam, float *advantages, float *returns, void *stream)
+{
+    if (B < 0 || T <= 0) return PPO_ERR_SHAPE;
+    if (!finite_f(gamma) || !finite_f(lam)) return PPO_ERR_PARAM;
+    if (B == 0) return PPO_OK;
+    if (!rewards || !values || !seq_len || !advantages || !returns) return PPO_ERR_NULL;
+    const unsigned grid = (unsigned)((B + 3) / 4);
+    gae_kernel<<<grid, 128, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+        rewards, values, seq_len, B, T, (double)gamma, (double)gamma * (double)lam, advantages, returns);
+    return launch_status();
+}
+
+extern "C" int ppo_whiten(const float *x, const uint8_t *mask, int64_t n_elems, int shift_mean, float eps,
+                          float *out, float *stats3, void *workspace, void *stream)
+{
+    if (n_elems < 0) return PPO_ERR_SHAPE;
+    if (!(eps >= 0.f) || !finite_f(eps)) return PPO_ERR_PARAM;
+    if (n_elems == 0) return PPO_OK;
+    if (!x || !out) return PPO_ERR_NULL;
+    int *status = workspace ? &ws_header(workspace)->status : nullptr;
+    whiten_kernel<<<1, kWhitenThreads, 0, reinterpret_cast<cudaStream_t>(stream)>>>(x, mask, n_elems, shift_mean, eps,
+                                                                                    out, stats3, status);
+    return launch_status();
+}
+
+extern "C" int ppo_loss_from_logprob(const float *new_logprob, const float *entropy, int32_t B, int32_t T,
+                                     const uint8_t *mask, const float *old_logprob, const float *advantages,
+                                     const float *values_new, const float *values_old, const float *returns,
+                                     const ppo_params *p, float *losses, float *dlogprob, float *dvalues,
+                                     void *workspace, void *stream)
+{
+    if (B <= 0 || T <= 0) return PPO_ERR_SHAPE;
+    if (!new_logprob || !mask || !old_logprob || !advantages || !values_new || !values_old || !returns || !p ||
+        !losses || !dvalues || !workspace)
+        return PPO_ERR_NULL;
+    if (!(p->cliprange >= 0.f) || !(p->cliprange_value >= 0.f) || !finite_f(p->vf_coef)) return PPO_ERR_PARAM;
+    if (reinterpret_cast<uintptr_t>(workspace) % 256) return PPO_ERR_ALIGN;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const int64_t rows = (int64_t)B * T;
+    int rc = launch_count_mask(mask, rows, workspace, s);
+    if (rc) return rc;
+    loss_from_logprob_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, s>>>(
+        new_logprob, entropy, rows, mask, old_logprob, advantages, values_new, values_old, returns, p->cliprange,
+        p->cliprange_value, p->vf_coef, ws_header(workspace), ws_partials(workspace), dlogprob, dvalues);
+    rc = launch_status();
+    if (rc) return rc;
+    return launch_loss_finalize(rows, p->vf_coef, losses, workspace, s);
+}
