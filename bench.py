@@ -1,0 +1,393 @@
+#!/usr/bin/env python
+"""Benchmark of the per-token PPO hot path (arXiv 2403.17031) on B200.
+
+One "step" = one pass of the whole path over one synthetic batch: EOS trick, log-prob/entropy of
+policy and reference logits, KL rewards, GAE, advantage whitening, clipped losses + gradients
+(9 kernel launches). Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1|2|3] [--impl ours|reference]
+
+N > 1: launch with torch.distributed.run (one rank per GPU, NCCL); every rank runs the same
+per-GPU batch shape on its own seeded batch (weak scaling, no data-path collective); the time is
+the max over ranks of the device-timed region.
+
+--impl reference times the fp64 CPU oracle (the only "reference" this work has) on the host
+cores, on a bounded sample of the same workload per step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+LAUNCHES_PER_STEP = 9   # truncate, 2x logprob, kl_rewards, gae, whiten, count_mask, loss_rows, loss_finalize
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            d = json.load(open(path))
+            return float(d["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, device_index: int, period_s: float = 0.01):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._period = period_s
+        self._h = None
+        try:
+            import pynvml
+            self._nv = pynvml
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            h = None
+            for cand in ("GPU-" + uuid, uuid):
+                try:
+                    h = pynvml.nvmlDeviceGetHandleByUUID(cand.encode() if isinstance(cand, str) else cand)
+                    break
+                except Exception:
+                    try:
+                        h = pynvml.nvmlDeviceGetHandleByUUID(cand)
+                        break
+                    except Exception:
+                        h = None
+            if h is None:
+                h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self._h = h
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+
+    def _reason_names(self, bits: int):
+        nv = self._nv
+        table = {
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "hw_power_brake_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80),
+        }
+        return [k for k, v in table.items() if bits & v]
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                try:
+                    bits = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                except Exception:
+                    bits = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                self.reasons.update(self._reason_names(bits))
+            except Exception:
+                pass
+            self._stop.wait(self._period)
+
+    def __enter__(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+
+    def summary(self):
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def _dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def _oracle_inputs(cfg, B_sample: int, seed: int):
+    """Host copies of a B_sample-sequence batch of cfg's shape, in the oracle's input types."""
+    import numpy as np
+    from paper_2403_17031_b200.synthetic import make_batch
+    batch = make_batch(cfg, "cpu", B=B_sample, seed=seed)
+
+    def host(t):
+        t = t.contiguous()
+        return t.view(torch.int16).numpy().view(np.uint16) if t.dtype == torch.bfloat16 else t.numpy()
+    return {k: host(v) for k, v in batch.items()}
+
+
+def _oracle_chain_time(cfg, inp):
+    """One pass of the whole path on the oracle; returns (seconds, tokens)."""
+    import numpy as np
+    from oracle import ppo_oracle as O
+    h = cfg.hyper
+    V = cfg.V
+    pl, rl, resp = inp["policy_logits"], inp["ref_logits"], inp["responses"]
+    tau = np.float32(h.temperature)
+    f32 = lambda a: np.asarray(a, np.float64).astype(np.float32)
+    t0 = time.perf_counter()
+    _, _, L, m, so = O.truncate_and_score(resp, h.eos_id, h.pad_id, inp["scores"], np.float32(h.no_eos_score))
+    lp, _, _ = O.logprob_entropy(pl.reshape(-1, V), resp, tau)
+    rlp, _, _ = O.logprob_entropy(rl.reshape(-1, V), resp, tau)
+    lp, rlp = lp.reshape(resp.shape), rlp.reshape(resp.shape)
+    _, rew = O.kl_rewards(f32(lp), f32(rlp), m, L, f32(so), np.float32(h.kl_coef))
+    adv, ret = O.gae(f32(rew), inp["values"], L, np.float32(h.gamma), np.float32(h.lam))
+    aw, _ = O.whiten(f32(adv), m, True, np.float32(h.whiten_eps))
+    old = f32(lp) + inp["old_logprob_noise"]
+    O.loss_fwd_bwd(pl, resp, m, old, f32(aw), inp["values_new"], inp["values"], f32(ret), tau,
+                   np.float32(h.cliprange), np.float32(h.cliprange_value), np.float32(h.vf_coef), want_dlogits=True)
+    return time.perf_counter() - t0, resp.size
+
+
+def run_reference(args, cfg):
+    """The reference arm: the fp64 CPU oracle, as it stands, on the host cores."""
+    rank, world, _ = _dist_env()
+    if rank != 0:
+        return
+    from oracle import ppo_oracle as O
+    O.build()
+    cores = O.num_threads()
+    # size the per-step sample so that the whole run stays within a few minutes
+    probe_s, _ = _oracle_chain_time(cfg, _oracle_inputs(cfg, 1, cfg.seed + 99))
+    budget = args.ref_seconds / max(args.steps + args.warmup, 1)
+    B_s = int(max(1, min(cfg.B, args.ref_sample, budget / max(probe_s, 1e-6))))
+    inp = _oracle_inputs(cfg, B_s, cfg.seed + 100)
+    for i in range(args.warmup):
+        _oracle_chain_time(cfg, inp)
+    total_s, total_tok = 0.0, 0
+    for i in range(args.steps):
+        s, tok = _oracle_chain_time(cfg, inp)
+        total_s += s
+        total_tok += tok
+    value = total_tok / total_s
+    sample = "%d of %d sequences per step (%d tokens, V=%d), oracle chain incl. dlogits" % (B_s, cfg.B, B_s * cfg.T, cfg.V)
+    line = {
+        "impl": "reference", "metric": "response tokens/s", "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_s / max(args.steps, 1),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "config%d %s" % (cfg.index, cfg.name), "B": cfg.B, "T": cfg.T, "V": cfg.V,
+                   "logits_dtype": cfg.dtype, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, cfg):
+    rank, world, local = _dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    distributed = world > 1
+    if distributed:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    from paper_2403_17031_b200 import binding, build
+    from paper_2403_17031_b200.pipeline import PPOHotPath
+    from paper_2403_17031_b200.synthetic import make_batch
+    if rank == 0:
+        build.build()
+    if distributed:
+        dist.barrier()
+    binding.lib()
+
+    h = cfg.hyper
+    B, T, V = cfg.B, cfg.T, cfg.V
+    batch = make_batch(cfg, dev, seed=cfg.seed + 1000 * rank)
+    hp = PPOHotPath(B, T, V, cfg.torch_dtype, binding.params_from(h), device=dev)
+    # stored rollout log-probs + noise: PPO ratios straddle the clip range (data, prepared untimed)
+    o = hp.rollout_stats(batch["policy_logits"], batch["ref_logits"], batch["responses"], batch["scores"],
+                         batch["values"])
+    old_logprob = (o["logprob"] + batch["old_logprob_noise"]).contiguous()
+    n_real = int(o["mask"].sum().item())
+    torch.cuda.synchronize()
+    esize = 2 if cfg.dtype == "bf16" else 4
+    R = B * T * V * esize
+
+    def step():
+        hp.step(batch["policy_logits"], batch["ref_logits"], batch["responses"], batch["scores"], batch["values"],
+                batch["values_new"], old_logprob=old_logprob)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+
+    # ---- timed region: K steps, device-timed; per-call events give the dominant kernel's duration
+    K = args.steps
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    loss_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    lp_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    if distributed:
+        dist.barrier()
+    torch.cuda.synchronize()
+    with ClockSampler(local) as clk:
+        ev0.record()
+        for i in range(K):
+            o = hp.out
+            p = hp.params
+            binding.truncate_and_score(batch["responses"], batch["scores"], p.eos_id, p.pad_id, p.no_eos_score,
+                                       out=(o["responses_out"], o["eos_index"], o["seq_len"], o["mask"], o["scores_out"]))
+            lp_ev[i][0].record()
+            binding.logprob_entropy(batch["policy_logits"], batch["responses"], p.temperature, workspace=hp.workspace,
+                                    out=(o["logprob"], o["entropy"], None))
+            lp_ev[i][1].record()
+            binding.logprob_entropy(batch["ref_logits"], batch["responses"], p.temperature, workspace=hp.workspace,
+                                    out=(o["ref_logprob"], None, None))
+            binding.kl_rewards(o["logprob"], o["ref_logprob"], o["mask"], o["seq_len"], o["scores_out"], p.kl_coef,
+                               out=(o["kl"], o["rewards"]))
+            binding.gae(o["rewards"], batch["values"], o["seq_len"], p.gamma, p.lam, out=(o["advantages"], o["returns"]))
+            binding.whiten(o["advantages"], o["mask"], True, p.whiten_eps, workspace=hp.workspace,
+                           out=o["advantages_whitened"], stats=o["whiten_stats"])
+            loss_ev[i][0].record()
+            hp.loss(batch["policy_logits"], batch["responses"], old_logprob, batch["values_new"], batch["values"])
+            loss_ev[i][1].record()
+        ev1.record()
+        torch.cuda.synchronize()
+    total_ms = ev0.elapsed_time(ev1)
+    if distributed:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+        dist.barrier()
+    ms_per_step = total_ms / K
+    tokens_per_step = B * T * world
+    value = tokens_per_step / (ms_per_step * 1e-3)
+    loss_ms = statistics.mean(a.elapsed_time(b) for a, b in loss_ev)
+    lp_ms = statistics.mean(a.elapsed_time(b) for a, b in lp_ev)
+    status = hp.device_status()
+
+    # ---- roofline of the dominant kernel (loss forward+backward): algorithmic bytes per launch =
+    # V*s read per real token + V*s written per token (zeros on masked rows)
+    peak, peak_kind = _peaks()
+    loss_bytes = n_real * V * esize + B * T * V * esize
+    loss_gbs = loss_bytes / (loss_ms * 1e-3) / 1e9
+    lp_gbs = R / (lp_ms * 1e-3) / 1e9
+    path_bytes = 2 * R + loss_bytes
+
+    # ---- end to end: inputs start in pinned host memory, results are read back to the host
+    e2e = None
+    if not args.no_e2e:
+        names = ["policy_logits", "ref_logits", "responses", "scores", "values", "values_new"]
+        host = {k: batch[k].cpu().pin_memory() for k in names}
+        host["old_logprob"] = old_logprob.cpu().pin_memory()
+        devbuf = {k: torch.empty_like(v, device=dev) for k, v in host.items()}
+        res_names = ["losses", "dvalues", "advantages_whitened", "returns", "logprob", "ref_logprob"]
+        host_res = {k: torch.empty_like(hp.out[k], device="cpu").pin_memory() for k in res_names}
+        h2d = sum(v.numel() * v.element_size() for v in host.values())
+        d2h = sum(v.numel() * v.element_size() for v in host_res.values())
+
+        def e2e_step():
+            for k, v in host.items():
+                devbuf[k].copy_(v, non_blocking=True)
+            hp.step(devbuf["policy_logits"], devbuf["ref_logits"], devbuf["responses"], devbuf["scores"],
+                    devbuf["values"], devbuf["values_new"], old_logprob=devbuf["old_logprob"])
+            for k, v in host_res.items():
+                v.copy_(hp.out[k], non_blocking=True)
+        Ke = max(3, min(K, args.e2e_steps))
+        for _ in range(2):
+            e2e_step()
+        torch.cuda.synchronize()
+        if distributed:
+            dist.barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(Ke):
+            e2e_step()
+        b.record()
+        torch.cuda.synchronize()
+        e_ms = a.elapsed_time(b)
+        if distributed:
+            t = torch.tensor([e_ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        e2e = {"value": tokens_per_step / (e_ms / Ke * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": Ke}
+        del host, devbuf
+
+    # ---- CPU baseline: the oracle on a bounded sample, rank 0, N = 1 only
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import ppo_oracle as O
+        O.build()
+        per_seq, _ = _oracle_chain_time(cfg, _oracle_inputs(cfg, 1, cfg.seed + 300))   # size probe
+        B_s = int(max(1, min(cfg.B, args.cpu_seconds / max(per_seq, 1e-6))))
+        s, tok = _oracle_chain_time(cfg, _oracle_inputs(cfg, B_s, cfg.seed + 301))
+        cpu = {"value": tok / s, "unit": "tokens/s", "cores": O.num_threads(), "kind": "oracle",
+               "sample": "%d of %d sequences (%d tokens, V=%d), whole chain incl. dlogits, %.1f s" %
+                         (B_s, cfg.B, tok, V, s)}
+
+    if rank == 0:
+        line = {
+            "metric": "response tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "config%d %s" % (cfg.index, cfg.name), "B_per_gpu": B, "T": T, "V": V,
+                       "logits_dtype": cfg.dtype, "real_tokens": n_real,
+                       "l2": "inputs larger than L2 (%.0f MB of logits read + %.0f MB written per step)" %
+                             (2 * R / 1e6, R / 1e6),
+                       "path_hbm_gbs": path_bytes / (ms_per_step * 1e-3) / 1e9,
+                       "path_hbm_frac_of_8tbs": path_bytes / (ms_per_step * 1e-3) / 8e12,
+                       "logprob_entropy_ms": lp_ms, "logprob_entropy_gbs": lp_gbs,
+                       "logprob_entropy_frac_of_peak": lp_gbs / peak, "loss_fwd_bwd_ms": loss_ms,
+                       "device_status": status},
+            "roofline": {"bound": "hbm", "kernel": "loss_rows_kernel (ppo_loss_fwd_bwd)", "achieved": loss_gbs,
+                         "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": loss_gbs / peak,
+                         "frac_of_8tbs": loss_gbs / 8000.0, "traffic": None,
+                         "timing": "CUDA events around the C-ABI call (3 launches: count, rows, finalize)"},
+            "clocks": clk.summary(),
+            "e2e": e2e,
+            "cpu_baseline": cpu,
+            "gpu_launches": LAUNCHES_PER_STEP * K,
+        }
+        print(json.dumps(line), flush=True)
+    if distributed:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--config", type=int, default=1, choices=[1, 2, 3])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--ref-sample", type=int, default=16, help="max sequences per step of the reference arm")
+    ap.add_argument("--ref-seconds", type=float, default=150.0, help="time budget of the reference arm")
+    args = ap.parse_args()
+    from paper_2403_17031_b200.synthetic import CONFIGS
+    cfg = CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

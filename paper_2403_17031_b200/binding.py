@@ -1,0 +1,308 @@
+"""ctypes binding of libppo_b200.so. Every function here only marshals arguments: it checks
+that tensors are CUDA, contiguous and of the documented dtype, allocates outputs with torch,
+passes raw device pointers and the current CUDA stream to the C ABI, and raises PPOError on a
+non-zero status. No step of the path is computed in Python or by torch kernels."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libppo_b200.so")
+
+PPO_F32, PPO_BF16 = 0, 1
+OPT_LOSS_ROW_CACHE = 1
+LOSS_NAMES = ("pg_loss", "vf_loss", "loss", "approx_kl", "pg_clipfrac", "vf_clipfrac", "entropy", "n")
+DEV_BAD_TOKEN, DEV_EMPTY_MASK, DEV_TIMEOUT = 1, 2, 4
+
+_ERR = {-1: "PPO_ERR_NULL", -2: "PPO_ERR_SHAPE", -3: "PPO_ERR_PARAM", -4: "PPO_ERR_ALIGN", -5: "PPO_ERR_DTYPE",
+        -6: "PPO_ERR_UNSUPPORTED"}
+
+
+class PPOError(RuntimeError):
+    def __init__(self, fn: str, code: int):
+        self.code = code
+        what = _ERR.get(code, "cudaError %d" % code if code > 0 else "status %d" % code)
+        super().__init__("%s failed: %s" % (fn, what))
+
+
+class PPOParams(C.Structure):
+    _fields_ = [("temperature", C.c_float), ("kl_coef", C.c_float), ("gamma", C.c_float), ("lam", C.c_float),
+                ("cliprange", C.c_float), ("cliprange_value", C.c_float), ("vf_coef", C.c_float),
+                ("no_eos_score", C.c_float), ("whiten_eps", C.c_float), ("eos_id", C.c_int32),
+                ("pad_id", C.c_int32)]
+
+
+_lib = None
+
+_SIGS = {
+    "ppo_default_params": (None, [C.POINTER(PPOParams)]),
+    "ppo_version": (C.c_int, []),
+    "ppo_set_option": (C.c_int, [C.c_int, C.c_int]),
+    "ppo_workspace_bytes": (C.c_size_t, [C.c_int32, C.c_int32, C.c_int64]),
+    "ppo_lmhead_workspace_bytes": (C.c_size_t, [C.c_int64, C.c_int64, C.c_int64]),
+    "ppo_workspace_init": (C.c_int, [C.c_void_p, C.c_size_t, C.c_void_p]),
+    "ppo_last_device_status": (C.c_int, [C.c_void_p, C.c_void_p, C.POINTER(C.c_int)]),
+    "ppo_logprob_entropy": (C.c_int, [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
+                                      C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "ppo_truncate_and_score": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
+                                         C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                         C.c_void_p]),
+    "ppo_kl_rewards": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
+                                 C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "ppo_gae": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float, C.c_float,
+                          C.c_void_p, C.c_void_p, C.c_void_p]),
+    "ppo_whiten": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_float, C.c_void_p, C.c_void_p,
+                             C.c_void_p, C.c_void_p]),
+    "ppo_loss_fwd_bwd": (C.c_int, [C.c_void_p, C.c_int, C.c_int32, C.c_int32, C.c_int64] + [C.c_void_p] * 7 +
+                         [C.POINTER(PPOParams)] + [C.c_void_p] * 8),
+    "ppo_loss_from_logprob": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32] + [C.c_void_p] * 6 +
+                              [C.POINTER(PPOParams)] + [C.c_void_p] * 5),
+    "ppo_lmhead_logprob_entropy": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p,
+                                             C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                             C.c_void_p]),
+}
+
+
+def lib():
+    """Load the CUDA library (built in-tree by paper_2403_17031_b200/build.py)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError("%s is missing: run `python -m paper_2403_17031_b200.build` (nvcc, sm_100a). "
+                              "There is no fallback path." % _LIB_PATH)
+        L = C.CDLL(_LIB_PATH)
+        for name, (res, args) in _SIGS.items():
+            fn = getattr(L, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = L
+    return _lib
+
+
+def exported_symbols():
+    return tuple(_SIGS.keys())
+
+
+# ---------------------------------------------------------------- helpers
+def _stream() -> C.c_void_p:
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None, name="tensor"):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise TypeError("%s must be a CUDA tensor" % name)
+    if not t.is_contiguous():
+        raise TypeError("%s must be contiguous" % name)
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError("%s must have dtype %s, got %s" % (name, dtype, t.dtype))
+    return C.c_void_p(t.data_ptr())
+
+
+def _logits_dtype(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return PPO_F32
+    if t.dtype == torch.bfloat16:
+        return PPO_BF16
+    raise TypeError("logits must be float32 or bfloat16, got %s" % t.dtype)
+
+
+def _check(fn: str, rc: int):
+    if rc != 0:
+        raise PPOError(fn, rc)
+
+
+def version() -> int:
+    return int(lib().ppo_version())
+
+
+def default_params(pad_id: Optional[int] = None, **overrides) -> PPOParams:
+    p = PPOParams()
+    lib().ppo_default_params(C.byref(p))
+    if pad_id is not None:
+        p.pad_id = pad_id
+    for k, v in overrides.items():
+        setattr(p, k, v)
+    return p
+
+
+def params_from(h) -> PPOParams:
+    """PPOParams from any object with the same attribute names (e.g. synthetic.PPOHyper)."""
+    p = PPOParams()
+    for name, _ in PPOParams._fields_:
+        setattr(p, name, getattr(h, name))
+    return p
+
+
+def set_option(key: int, value: int) -> None:
+    _check("ppo_set_option", lib().ppo_set_option(key, value))
+
+
+def workspace_bytes(B: int, T: int, V: int) -> int:
+    return int(lib().ppo_workspace_bytes(B, T, V))
+
+
+def lmhead_workspace_bytes(M: int, K: int, V: int) -> int:
+    return int(lib().ppo_lmhead_workspace_bytes(M, K, V))
+
+
+def new_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    """Allocate (torch) and clear a workspace of at least `nbytes`."""
+    ws = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+    assert ws.data_ptr() % 256 == 0
+    _check("ppo_workspace_init", lib().ppo_workspace_init(_ptr(ws), ws.numel(), _stream()))
+    return ws
+
+
+def last_device_status(workspace: torch.Tensor) -> int:
+    st = C.c_int(0)
+    _check("ppo_last_device_status", lib().ppo_last_device_status(_ptr(workspace), _stream(), C.byref(st)))
+    return int(st.value)
+
+
+# ---------------------------------------------------------------- the path
+def logprob_entropy(logits: torch.Tensor, tokens: torch.Tensor, temperature: float,
+                    mask: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                    want_entropy: bool = True, want_lse: bool = False, out=None):
+    """logits [..., V] (last dim contiguous rows), tokens [...] int32. Returns (logprob, entropy, lse)."""
+    V = logits.shape[-1]
+    rows = logits.numel() // V if V else 0
+    lg2 = logits.reshape(rows, V) if logits.is_contiguous() else logits
+    if lg2.dim() != 2 or lg2.stride(1) != 1:
+        raise TypeError("logits rows must be contiguous")
+    stride = lg2.stride(0) if rows > 1 else V
+    shape = tokens.shape
+    if out is None:
+        lp = torch.empty(shape, dtype=torch.float32, device=logits.device)
+        ent = torch.empty(shape, dtype=torch.float32, device=logits.device) if want_entropy else None
+        lse = torch.empty(shape, dtype=torch.float32, device=logits.device) if want_lse else None
+    else:
+        lp, ent, lse = out
+    if not lg2.is_cuda:
+        raise TypeError("logits must be a CUDA tensor")
+    rc = lib().ppo_logprob_entropy(C.c_void_p(lg2.data_ptr()), _logits_dtype(lg2), rows, V, stride,
+                                   _ptr(tokens, torch.int32, "tokens"), _ptr(mask, torch.uint8, "mask"),
+                                   float(temperature), _ptr(lp, torch.float32), _ptr(ent, torch.float32),
+                                   _ptr(lse, torch.float32), _ptr(workspace), _stream())
+    _check("ppo_logprob_entropy", rc)
+    return lp, ent, lse
+
+
+def truncate_and_score(responses: torch.Tensor, scores: torch.Tensor, eos_id: int, pad_id: int,
+                       no_eos_score: float, out=None):
+    """Returns (responses_out, eos_index, seq_len, mask, scores_out)."""
+    B, T = responses.shape
+    dev = responses.device
+    if out is None:
+        out = (torch.empty((B, T), dtype=torch.int32, device=dev), torch.empty((B,), dtype=torch.int32, device=dev),
+               torch.empty((B,), dtype=torch.int32, device=dev), torch.empty((B, T), dtype=torch.uint8, device=dev),
+               torch.empty((B,), dtype=torch.float32, device=dev))
+    ro, ei, sl, m, so = out
+    rc = lib().ppo_truncate_and_score(_ptr(responses, torch.int32, "responses"), B, T, eos_id, pad_id,
+                                      _ptr(scores, torch.float32, "scores"), float(no_eos_score),
+                                      _ptr(ro, torch.int32), _ptr(ei, torch.int32), _ptr(sl, torch.int32),
+                                      _ptr(m, torch.uint8), _ptr(so, torch.float32), _stream())
+    _check("ppo_truncate_and_score", rc)
+    return out
+
+
+def kl_rewards(logprob, ref_logprob, mask, seq_len, scores, kl_coef: float, out=None):
+    B, T = logprob.shape
+    if out is None:
+        out = (torch.empty_like(logprob), torch.empty_like(logprob))
+    kl, rew = out
+    rc = lib().ppo_kl_rewards(_ptr(logprob, torch.float32), _ptr(ref_logprob, torch.float32),
+                              _ptr(mask, torch.uint8), _ptr(seq_len, torch.int32), _ptr(scores, torch.float32),
+                              B, T, float(kl_coef), _ptr(kl, torch.float32), _ptr(rew, torch.float32), _stream())
+    _check("ppo_kl_rewards", rc)
+    return out
+
+
+def gae(rewards, values, seq_len, gamma: float, lam: float, out=None):
+    B, T = rewards.shape
+    if out is None:
+        out = (torch.empty_like(rewards), torch.empty_like(rewards))
+    adv, ret = out
+    rc = lib().ppo_gae(_ptr(rewards, torch.float32), _ptr(values, torch.float32), _ptr(seq_len, torch.int32), B, T,
+                       float(gamma), float(lam), _ptr(adv, torch.float32), _ptr(ret, torch.float32), _stream())
+    _check("ppo_gae", rc)
+    return out
+
+
+def whiten(x, mask=None, shift_mean: bool = True, eps: float = 1e-8, workspace=None, out=None, stats=None):
+    if out is None:
+        out = torch.empty_like(x)
+    if stats is None:
+        stats = torch.empty(3, dtype=torch.float32, device=x.device)
+    rc = lib().ppo_whiten(_ptr(x, torch.float32), _ptr(mask, torch.uint8), x.numel(), 1 if shift_mean else 0,
+                          float(eps), _ptr(out, torch.float32), _ptr(stats, torch.float32), _ptr(workspace),
+                          _stream())
+    _check("ppo_whiten", rc)
+    return out, stats
+
+
+def loss_fwd_bwd(logits, tokens, mask, old_logprob, advantages, values_new, values_old, returns,
+                 params: PPOParams, workspace, want_dlogits: bool = True, want_aux: bool = True, out=None):
+    """Returns dict(losses[8], dlogits, dvalues, new_logprob, entropy, dlogprob)."""
+    B, T, V = logits.shape
+    dev = logits.device
+    if out is None:
+        out = {
+            "losses": torch.empty(8, dtype=torch.float32, device=dev),
+            "dlogits": torch.empty_like(logits) if want_dlogits else None,
+            "dvalues": torch.empty((B, T), dtype=torch.float32, device=dev),
+            "new_logprob": torch.empty((B, T), dtype=torch.float32, device=dev) if want_aux else None,
+            "entropy": torch.empty((B, T), dtype=torch.float32, device=dev) if want_aux else None,
+            "dlogprob": torch.empty((B, T), dtype=torch.float32, device=dev) if want_aux else None,
+        }
+    f32 = torch.float32
+    rc = lib().ppo_loss_fwd_bwd(_ptr(logits, None, "logits"), _logits_dtype(logits), B, T, V,
+                                _ptr(tokens, torch.int32, "tokens"), _ptr(mask, torch.uint8, "mask"),
+                                _ptr(old_logprob, f32), _ptr(advantages, f32), _ptr(values_new, f32),
+                                _ptr(values_old, f32), _ptr(returns, f32), C.byref(params),
+                                _ptr(out["losses"], f32), _ptr(out["dlogits"], logits.dtype),
+                                _ptr(out["dvalues"], f32), _ptr(out["new_logprob"], f32), _ptr(out["entropy"], f32),
+                                _ptr(out["dlogprob"], f32), _ptr(workspace), _stream())
+    _check("ppo_loss_fwd_bwd", rc)
+    return out
+
+
+def loss_from_logprob(new_logprob, entropy, mask, old_logprob, advantages, values_new, values_old, returns,
+                      params: PPOParams, workspace, out=None):
+    B, T = new_logprob.shape
+    dev = new_logprob.device
+    f32 = torch.float32
+    if out is None:
+        out = {"losses": torch.empty(8, dtype=f32, device=dev), "dlogprob": torch.empty((B, T), dtype=f32, device=dev),
+               "dvalues": torch.empty((B, T), dtype=f32, device=dev)}
+    rc = lib().ppo_loss_from_logprob(_ptr(new_logprob, f32), _ptr(entropy, f32), B, T, _ptr(mask, torch.uint8),
+                                     _ptr(old_logprob, f32), _ptr(advantages, f32), _ptr(values_new, f32),
+                                     _ptr(values_old, f32), _ptr(returns, f32), C.byref(params),
+                                     _ptr(out["losses"], f32), _ptr(out["dlogprob"], f32), _ptr(out["dvalues"], f32),
+                                     _ptr(workspace), _stream())
+    _check("ppo_loss_from_logprob", rc)
+    return out
+
+
+def lmhead_logprob_entropy(H, W, tokens, temperature: float, workspace, mask=None, want_lse: bool = True,
+                           out=None):
+    M, K = H.shape
+    K2, V = W.shape
+    if K != K2:
+        raise ValueError("H [M,K] and W [K,V] disagree on K")
+    dev = H.device
+    if out is None:
+        out = (torch.empty(M, dtype=torch.float32, device=dev), torch.empty(M, dtype=torch.float32, device=dev),
+               torch.empty(M, dtype=torch.float32, device=dev) if want_lse else None)
+    lp, ent, lse = out
+    rc = lib().ppo_lmhead_logprob_entropy(_ptr(H, torch.bfloat16, "H"), _ptr(W, torch.bfloat16, "W"), M, K, V,
+                                          _ptr(tokens, torch.int32, "tokens"), _ptr(mask, torch.uint8),
+                                          float(temperature), _ptr(lp, torch.float32), _ptr(ent, torch.float32),
+                                          _ptr(lse, torch.float32), _ptr(workspace), _stream())
+    _check("ppo_lmhead_logprob_entropy", rc)
+    return out

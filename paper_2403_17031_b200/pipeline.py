@@ -1,0 +1,77 @@
+"""The whole per-token path as one object: preallocated outputs + the chain of C-ABI calls in
+the order a PPO iteration runs them. Pure call sequencing; every step runs in the CUDA library."""
+from __future__ import annotations
+
+from typing import Dict, Optional
+
+import torch
+
+from . import binding as _b
+
+
+class PPOHotPath:
+    """Buffers and call chain for a batch of B responses x T tokens over a vocabulary of V.
+
+    step(...) runs: EOS trick -> log-prob/entropy of policy and reference -> KL rewards -> GAE ->
+    advantage whitening -> clipped losses + gradients, all on the current CUDA stream, and
+    returns the dict of output tensors (owned by this object, overwritten by the next step).
+    """
+
+    def __init__(self, B: int, T: int, V: int, logits_dtype: torch.dtype, params: _b.PPOParams,
+                 device="cuda", want_dlogits: bool = True):
+        self.B, self.T, self.V = B, T, V
+        self.params = params
+        self.device = torch.device(device)
+        f32, i32, u8 = torch.float32, torch.int32, torch.uint8
+        dev = self.device
+        bt = lambda dt: torch.empty((B, T), dtype=dt, device=dev)
+        self.workspace = _b.new_workspace(_b.workspace_bytes(B, T, V), dev)
+        self.out: Dict[str, Optional[torch.Tensor]] = {
+            "responses_out": bt(i32), "eos_index": torch.empty(B, dtype=i32, device=dev),
+            "seq_len": torch.empty(B, dtype=i32, device=dev), "mask": bt(u8),
+            "scores_out": torch.empty(B, dtype=f32, device=dev),
+            "logprob": bt(f32), "entropy": bt(f32), "ref_logprob": bt(f32),
+            "kl": bt(f32), "rewards": bt(f32), "advantages": bt(f32), "returns": bt(f32),
+            "advantages_whitened": bt(f32), "whiten_stats": torch.empty(3, dtype=f32, device=dev),
+            "losses": torch.empty(8, dtype=f32, device=dev),
+            "dlogits": torch.empty((B, T, V), dtype=logits_dtype, device=dev) if want_dlogits else None,
+            "dvalues": bt(f32), "new_logprob": bt(f32), "new_entropy": bt(f32), "dlogprob": bt(f32),
+        }
+        self._loss_out = {"losses": self.out["losses"], "dlogits": self.out["dlogits"],
+                          "dvalues": self.out["dvalues"], "new_logprob": self.out["new_logprob"],
+                          "entropy": self.out["new_entropy"], "dlogprob": self.out["dlogprob"]}
+
+    def rollout_stats(self, policy_logits, ref_logits, responses, scores, values, skip_masked_rows=False):
+        """Steps 1-5: everything between sampling and the first PPO epoch."""
+        o, p = self.out, self.params
+        _b.truncate_and_score(responses, scores, p.eos_id, p.pad_id, p.no_eos_score,
+                              out=(o["responses_out"], o["eos_index"], o["seq_len"], o["mask"], o["scores_out"]))
+        m = o["mask"] if skip_masked_rows else None
+        _b.logprob_entropy(policy_logits, responses, p.temperature, mask=m, workspace=self.workspace,
+                           out=(o["logprob"], o["entropy"], None))
+        _b.logprob_entropy(ref_logits, responses, p.temperature, mask=m, workspace=self.workspace,
+                           out=(o["ref_logprob"], None, None))
+        _b.kl_rewards(o["logprob"], o["ref_logprob"], o["mask"], o["seq_len"], o["scores_out"], p.kl_coef,
+                      out=(o["kl"], o["rewards"]))
+        _b.gae(o["rewards"], values, o["seq_len"], p.gamma, p.lam, out=(o["advantages"], o["returns"]))
+        _b.whiten(o["advantages"], o["mask"], True, p.whiten_eps, workspace=self.workspace,
+                  out=o["advantages_whitened"], stats=o["whiten_stats"])
+        return o
+
+    def loss(self, logits, responses, old_logprob, values_new, values_old):
+        """Step 6 on the loss-time logits, using the advantages/returns of rollout_stats."""
+        o = self.out
+        _b.loss_fwd_bwd(logits, responses, o["mask"], old_logprob, o["advantages_whitened"], values_new,
+                        values_old, o["returns"], self.params, self.workspace, out=self._loss_out)
+        return o
+
+    def step(self, policy_logits, ref_logits, responses, scores, values, values_new, old_logprob=None,
+             loss_logits=None, skip_masked_rows=False):
+        """One pass of the whole path. old_logprob defaults to the rollout log-probs just computed
+        (first PPO epoch: ratio = 1); loss_logits defaults to policy_logits."""
+        o = self.rollout_stats(policy_logits, ref_logits, responses, scores, values, skip_masked_rows)
+        return self.loss(policy_logits if loss_logits is None else loss_logits, responses,
+                         o["logprob"] if old_logprob is None else old_logprob, values_new, values)
+
+    def device_status(self) -> int:
+        return _b.last_device_status(self.workspace)
