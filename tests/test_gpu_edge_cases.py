@@ -184,11 +184,12 @@ def test_loss_kernel_variants(P, oracle, dtype, V, mode):
     assert_abs(n * npy(o["dlogprob"]), n * ref["dlogprob"], 1e-4, "n*dlogprob")
     assert_grad(n * o["dlogits"].float().cpu().numpy().reshape(-1, V), n * ref["dlogits"],
                 dtype == torch.bfloat16, "n*dlogits")
-    # bit-reproducible from run to run; forward-only call agrees on everything it returns
+    # bit-reproducible from run to run
     for k in ("losses", "dlogits", "dvalues", "new_logprob", "entropy", "dlogprob"):
         assert torch.equal(o[k], o_b[k]), k
+    # the forward-only call may run a differently shaped block (other summation order)
     for k in ("losses", "dvalues", "new_logprob", "entropy", "dlogprob"):
-        assert torch.equal(o[k], o_n[k]), k
+        assert torch.allclose(o[k], o_n[k], rtol=1e-5, atol=1e-6), k
 
 
 def test_loss_from_logprob_matches_oracle(P, oracle):
@@ -196,7 +197,7 @@ def test_loss_from_logprob_matches_oracle(P, oracle):
     rng = np.random.default_rng(21)
     L = rng.integers(1, T + 1, B)
     m = (np.arange(T)[None] < L[:, None]).astype(np.uint8)
-    nlp = rng.normal(-3, 1, (B, T)).astype(np.float32)
+    nlp = (-0.05 - np.abs(rng.normal(3, 1, (B, T)))).astype(np.float32)     # log-probs are negative
     old = (nlp + rng.normal(0, 0.15, (B, T))).astype(np.float32)
     adv, vo, ret = (rng.normal(size=(B, T)).astype(np.float32) for _ in range(3))
     vn = (vo + rng.normal(0, 0.2, (B, T))).astype(np.float32)
