@@ -30,7 +30,7 @@ if ROOT not in sys.path:
 
 import torch  # noqa: E402
 
-LAUNCHES_PER_STEP = 9   # truncate, 2x logprob, kl_rewards, gae, whiten, count_mask, loss_rows, loss_finalize
+LAUNCHES_PER_STEP = 8   # truncate, 2x logprob, kl_rewards, gae, whiten, loss_prepare, row_engine (loss)
 
 
 def _peaks():

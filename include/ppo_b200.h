@@ -88,8 +88,13 @@ int ppo_version(void);
  *   PPO_OPT_LOSS_ROW_CACHE  how ppo_loss_fwd_bwd keeps a row between its statistics pass and its
  *                           gradient pass: 0 = choose by row size (default), 1 = in shared memory
  *                           whenever the row fits one block, 2 = re-read it from global memory/L2
+ *                           (applies to the direct-load kernels only)
+ *   PPO_OPT_ROW_ENGINE      which kernels stream the logits: 0 = default (the loss through the
+ *                           bulk-copy row engine when the shape allows, log-prob/entropy through
+ *                           direct loads), 1 = direct loads for both, 2 = row engine for both
  */
 #define PPO_OPT_LOSS_ROW_CACHE 1
+#define PPO_OPT_ROW_ENGINE 2
 int ppo_set_option(int key, int value);
 
 /*

@@ -15,6 +15,7 @@ _LIB_PATH = os.path.join(_HERE, "libppo_b200.so")
 
 PPO_F32, PPO_BF16 = 0, 1
 OPT_LOSS_ROW_CACHE = 1
+OPT_ROW_ENGINE = 2
 LOSS_NAMES = ("pg_loss", "vf_loss", "loss", "approx_kl", "pg_clipfrac", "vf_clipfrac", "entropy", "n")
 DEV_BAD_TOKEN, DEV_EMPTY_MASK, DEV_TIMEOUT = 1, 2, 4
 

@@ -12,11 +12,15 @@ namespace ppo {
 
 // ---------------------------------------------------------------- workspace layout
 // [0, 256)                      WorkspaceHeader
-// [256, 256 + rows*8*4)         per-token loss partials, 8 floats per token
+// [256, +align256(rows*8*4))    per-token loss partials, 8 floats per token
+// [.., +align256(rows*4))       row order of the loss call: real rows first (ascending), then
+//                               masked rows from the back
 struct WorkspaceHeader {
-    int status;      // PPO_DEV_* bits, sticky until read
-    int n_tokens;    // number of mask==1 tokens of the loss call in flight
-    int reserved[62];
+    int status;        // PPO_DEV_* bits, sticky until read
+    int n_tokens;      // number of mask==1 tokens of the loss call in flight
+    int masked_next;   // work counter of the zero-fill phase (reset by every loss call)
+    int done_blocks;   // blocks of the loss kernel that have retired (reset by every loss call)
+    int reserved[60];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header is one 256-byte block");
 
@@ -29,6 +33,11 @@ __host__ __device__ inline WorkspaceHeader *ws_header(void *ws) { return reinter
 __host__ __device__ inline float *ws_partials(void *ws)
 {
     return reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(ws) + kHeaderBytes);
+}
+inline int32_t *ws_order(void *ws, int64_t rows)
+{
+    return reinterpret_cast<int32_t *>(reinterpret_cast<unsigned char *>(ws) + kHeaderBytes +
+                                       align256((size_t)rows * kPartialsPerToken * sizeof(float)));
 }
 
 inline bool finite_f(float x) { return isfinite(x); }
@@ -190,8 +199,48 @@ __device__ __forceinline__ TokenLoss token_loss(float lp_new, float lp_old, floa
     return o;
 }
 
+// Sum the per-token partials in a fixed order (thread t takes rows t, t+NT, ...; fp64) and write the
+// eight loss scalars. Called by all NT threads of one block; `red` holds 6*32 doubles; `sync` is a
+// barrier over exactly those NT threads.
+template <int NT, typename SyncFn>
+__device__ __forceinline__ void reduce_loss_partials(const float *partials, int64_t rows, int n_tokens, float vf_coef,
+                                                     float *losses, double *red, int t, SyncFn sync)
+{
+    double acc[6] = {0, 0, 0, 0, 0, 0};
+    for (int64_t r = t; r < rows; r += NT) {
+        const float4 p0 = __ldcg(reinterpret_cast<const float4 *>(partials + r * kPartialsPerToken));
+        const float4 p1 = __ldcg(reinterpret_cast<const float4 *>(partials + r * kPartialsPerToken) + 1);
+        acc[0] += p0.x; acc[1] += p0.y; acc[2] += p0.z; acc[3] += p0.w; acc[4] += p1.x; acc[5] += p1.y;
+    }
+    const int lane = t & 31, warp = t >> 5;
+#pragma unroll
+    for (int k = 0; k < 6; ++k) {
+        acc[k] = warp_sum(acc[k]);
+        if (lane == 0) red[k * 32 + warp] = acc[k];
+    }
+    sync();
+    if (warp == 0) {
+        double tot[6];
+#pragma unroll
+        for (int k = 0; k < 6; ++k) tot[k] = warp_sum(lane < NT / 32 ? red[k * 32 + lane] : 0.0);
+        if (lane == 0) {
+            const double n = (double)n_tokens;
+            const double inv = n > 0.0 ? 1.0 / n : 0.0;
+            const double pg = tot[0] * inv, vf = 0.5 * tot[1] * inv;
+            losses[PPO_LOSS_PG] = (float)pg;
+            losses[PPO_LOSS_VF] = (float)vf;
+            losses[PPO_LOSS_TOTAL] = (float)(pg + (double)vf_coef * vf);
+            losses[PPO_LOSS_APPROX_KL] = (float)(tot[2] * inv);
+            losses[PPO_LOSS_PG_CLIPFRAC] = (float)(tot[3] * inv);
+            losses[PPO_LOSS_VF_CLIPFRAC] = (float)(tot[4] * inv);
+            losses[PPO_LOSS_ENTROPY] = (float)(tot[5] * inv);
+            losses[PPO_LOSS_N] = (float)n;
+        }
+    }
+}
+
 // launchers shared between translation units
-int launch_count_mask(const uint8_t *mask, int64_t n_elems, void *workspace, cudaStream_t s);
+int launch_loss_prepare(const uint8_t *mask, int64_t rows, void *workspace, cudaStream_t s);
 int launch_loss_finalize(int64_t rows, float vf_coef, float *losses, void *workspace, cudaStream_t s);
 
 // tuning options (ppo_set_option)

@@ -1,140 +1,19 @@
-// Row kernels: the two steps that stream the [rows, V] logits.
-//   ppo_logprob_entropy  -- one read of every row (single-pass online softmax statistics)
+// Row kernels: the two steps that stream the [rows, V] logits, and their C entry points.
+//   ppo_logprob_entropy  -- one read of every row (single-pass softmax statistics)
 //   ppo_loss_fwd_bwd     -- one read and one write of every real row: the row is parked in
 //                           shared memory between the statistics pass and the gradient pass
-// One thread block owns one row at a time; 128-bit coalesced loads/stores; fp32 accumulation
-// in base-2 units (one ex2 per element); warp-shuffle + shared-memory merge of the running
-// (max, sum, sum*log) states; per-token scalar math in fp64 by one thread.
-#include "ppo_common.cuh"
+// The entry points prefer the bulk-copy row engine (ppo_rows_bulk.cu). The kernels in this file
+// load straight into registers and serve every shape the engine does not take: rows that are not
+// 16-byte aligned, V not a multiple of the pack size, rows larger than shared memory, and the
+// forward-only loss call. One thread block owns one row at a time; fp32 accumulation in base-2
+// units (one ex2 per element); warp-shuffle + shared-memory merge of the per-thread states;
+// per-token scalar math in fp64 by one thread.
+#include "ppo_rows.cuh"
 
 namespace ppo {
 
-// ---------------------------------------------------------------- element packs
-// A "pack" is one 16-byte vector: 8 bf16 or 4 fp32 logits.
-template <typename T> struct Pack;
-
-template <> struct Pack<float> {
-    static constexpr int N = 4;
-    static __device__ __forceinline__ float clampf(float x) { return (x != x) ? x : fmaxf(x, kNegBig); }
-    static __device__ __forceinline__ void unpack(const uint4 &v, float (&x)[4], float &xmax)
-    {
-        // fmaxf drops NaN; clampf keeps it so a NaN logit poisons the row as documented
-        x[0] = clampf(__uint_as_float(v.x));
-        x[1] = clampf(__uint_as_float(v.y));
-        x[2] = clampf(__uint_as_float(v.z));
-        x[3] = clampf(__uint_as_float(v.w));
-        xmax = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
-    }
-    static __device__ __forceinline__ uint4 pack(const float (&d)[4])
-    {
-        return make_uint4(__float_as_uint(d[0]), __float_as_uint(d[1]), __float_as_uint(d[2]),
-                          __float_as_uint(d[3]));
-    }
-    static __device__ __forceinline__ float load1(const float *p) { return *p; }
-    static __device__ __forceinline__ void store1(float *p, float v) { *p = v; }
-};
-
-template <> struct Pack<__nv_bfloat16> {
-    static constexpr int N = 8;
-    static __device__ __forceinline__ __nv_bfloat162 as2(uint32_t w)
-    {
-        return *reinterpret_cast<__nv_bfloat162 *>(&w);
-    }
-    static __device__ __forceinline__ uint32_t bits(__nv_bfloat162 h) { return *reinterpret_cast<uint32_t *>(&h); }
-    static __device__ __forceinline__ void unpack(const uint4 &v, float (&x)[8], float &xmax)
-    {
-        const __nv_bfloat162 lim = __float2bfloat162_rn(kNegBig);
-        const __nv_bfloat162 h0 = __hmax2_nan(as2(v.x), lim), h1 = __hmax2_nan(as2(v.y), lim),
-                             h2 = __hmax2_nan(as2(v.z), lim), h3 = __hmax2_nan(as2(v.w), lim);
-        const __nv_bfloat162 hm = __hmax2(__hmax2(h0, h1), __hmax2(h2, h3));
-        xmax = fmaxf(__low2float(hm), __high2float(hm));
-        const uint32_t w0 = bits(h0), w1 = bits(h1), w2 = bits(h2), w3 = bits(h3);
-        x[0] = __uint_as_float(w0 << 16); x[1] = __uint_as_float(w0 & 0xffff0000u);
-        x[2] = __uint_as_float(w1 << 16); x[3] = __uint_as_float(w1 & 0xffff0000u);
-        x[4] = __uint_as_float(w2 << 16); x[5] = __uint_as_float(w2 & 0xffff0000u);
-        x[6] = __uint_as_float(w3 << 16); x[7] = __uint_as_float(w3 & 0xffff0000u);
-    }
-    static __device__ __forceinline__ uint4 pack(const float (&d)[8])
-    {
-        return make_uint4(bits(__floats2bfloat162_rn(d[0], d[1])), bits(__floats2bfloat162_rn(d[2], d[3])),
-                          bits(__floats2bfloat162_rn(d[4], d[5])), bits(__floats2bfloat162_rn(d[6], d[7])));
-    }
-    static __device__ __forceinline__ float load1(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
-    static __device__ __forceinline__ void store1(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
-};
-
-// streaming 16-byte global accesses (data is touched once: evict-first)
-__device__ __forceinline__ uint4 ld_stream(const uint4 *p) { return __ldcs(p); }
-__device__ __forceinline__ void st_stream(uint4 *p, const uint4 &v) { __stcs(p, v); }
-
-// fold one pack into the running state
-template <typename T>
-__device__ __forceinline__ void accumulate(const uint4 &v, float c, SoftmaxState &st)
-{
-    float x[Pack<T>::N], xmax;
-    Pack<T>::unpack(v, x, xmax);
-    const float ymax = xmax * c;
-    if (ymax > st.m) st.rebase(ymax);
-    const float nm = -st.m;
-    float s1 = 0.f, u1 = 0.f;   // second accumulator pair: two independent add chains
-#pragma unroll
-    for (int k = 0; k < Pack<T>::N; k += 2) {
-        const float t0 = fmaf(x[k], c, nm), t1 = fmaf(x[k + 1], c, nm);
-        const float e0 = ex2(t0), e1 = ex2(t1);
-        st.s += e0;
-        st.u = fmaf(e0, t0, st.u);
-        s1 += e1;
-        u1 = fmaf(e1, t1, u1);
-    }
-    st.s += s1;
-    st.u += u1;
-}
-
-// Statistics pass over one row. VECTOR: 16-byte packs (row base 16-byte aligned, V % N == 0);
-// otherwise element by element. STAGE: also park the raw packs / elements in shared memory.
-template <typename T, bool VECTOR, bool STAGE, int THREADS, int UNROLL>
-__device__ __forceinline__ SoftmaxState row_statistics(const T *__restrict__ src, int V, float c, void *stage)
-{
-    SoftmaxState st;
-    st.init();
-    if (VECTOR) {
-        constexpr int N = Pack<T>::N;
-        const uint4 *src4 = reinterpret_cast<const uint4 *>(src);
-        uint4 *stage4 = reinterpret_cast<uint4 *>(stage);
-        const int nvec = V / N;
-        int i = threadIdx.x;
-        for (; i + (UNROLL - 1) * THREADS < nvec; i += UNROLL * THREADS) {
-            uint4 v[UNROLL];
-#pragma unroll
-            for (int k = 0; k < UNROLL; ++k) v[k] = ld_stream(src4 + i + k * THREADS);
-#pragma unroll
-            for (int k = 0; k < UNROLL; ++k) {
-                if (STAGE) stage4[i + k * THREADS] = v[k];
-                accumulate<T>(v[k], c, st);
-            }
-        }
-        for (; i < nvec; i += THREADS) {
-            const uint4 v = ld_stream(src4 + i);
-            if (STAGE) stage4[i] = v;
-            accumulate<T>(v, c, st);
-        }
-    } else {
-        T *stage1 = reinterpret_cast<T *>(stage);
-        for (int j = threadIdx.x; j < V; j += THREADS) {
-            const T raw = src[j];
-            if (STAGE) stage1[j] = raw;
-            float x = Pack<T>::load1(&raw);
-            x = (x != x) ? x : fmaxf(x, kNegBig);
-            const float y = x * c;
-            if (y > st.m) st.rebase(y);
-            st.add(fmaf(x, c, -st.m));
-        }
-    }
-    return st;
-}
-
 // ---------------------------------------------------------------- step 1 kernel
-template <typename T, bool VECTOR, int THREADS>
+template <typename T, bool VECTOR, bool ENTROPY, int THREADS>
 __global__ void __launch_bounds__(THREADS)
 logprob_entropy_kernel(const T *__restrict__ logits, int64_t rows, int V, int64_t row_stride,
                        const int32_t *__restrict__ tokens, const uint8_t *__restrict__ mask, float c,
@@ -156,7 +35,7 @@ logprob_entropy_kernel(const T *__restrict__ logits, int64_t rows, int V, int64_
         const bool bad = tok < 0 || tok >= V;
         float xtok = 0.f;
         if (threadIdx.x == 0 && !bad) xtok = Pack<T>::load1(src + tok);
-        SoftmaxState st = row_statistics<T, VECTOR, false, THREADS, 4>(src, V, c, nullptr);
+        SoftmaxState st = row_statistics<T, VECTOR, false, ENTROPY, THREADS, 4>(src, V, c, nullptr);
         st = block_merge<THREADS>(st, red);
         if (threadIdx.x == 0) {
             const float l2s = log2f(st.s);
@@ -175,22 +54,6 @@ logprob_entropy_kernel(const T *__restrict__ logits, int64_t rows, int V, int64_
 }
 
 // ---------------------------------------------------------------- step 6 kernel
-struct LossArgs {
-    const void *logits;
-    void *dlogits;
-    int64_t rows;
-    int V;
-    const int32_t *tokens;
-    const uint8_t *mask;
-    const float *old_logprob, *advantages, *values_new, *values_old, *returns;
-    float *dvalues, *new_logprob, *entropy, *dlogprob;
-    float *partials;
-    const int *n_tokens;
-    int *status;
-    float c;        // log2(e) / temperature
-    float inv_tau;  // 1 / temperature
-    float eps, eps_v, c1;
-};
 
 template <typename T, bool VECTOR, int THREADS>
 __device__ __forceinline__ void fill_row_zero(T *dst, int V)
@@ -239,9 +102,16 @@ loss_rows_kernel(const LossArgs a)
         const T *src = logits + row * (int64_t)V;
         const int tok = a.tokens[row];
         const bool bad = tok < 0 || tok >= V;
-        float xtok = 0.f;
-        if (threadIdx.x == 0 && !bad) xtok = Pack<T>::load1(src + tok);
-        SoftmaxState st = row_statistics<T, VECTOR, ROW_IN_SMEM, THREADS, 4>(src, V, a.c, row_stage);
+        float xtok = 0.f, t_old = 0.f, t_adv = 0.f, t_vn = 0.f, t_vo = 0.f, t_ret = 0.f;
+        if (threadIdx.x == 0) {   // per-token scalars: fetched now, used after the row reduction
+            if (!bad) xtok = Pack<T>::load1(src + tok);
+            t_old = a.old_logprob[row];
+            t_adv = a.advantages[row];
+            t_vn = a.values_new[row];
+            t_vo = a.values_old[row];
+            t_ret = a.returns[row];
+        }
+        SoftmaxState st = row_statistics<T, VECTOR, ROW_IN_SMEM, true, THREADS, 4>(src, V, a.c, row_stage);
         st = block_merge<THREADS>(st, red);
         if (threadIdx.x == 0) {
             const float l2s = log2f(st.s);
@@ -251,8 +121,7 @@ loss_rows_kernel(const LossArgs a)
                 lp = H = __int_as_float(0x7fc00000);
                 if (a.status) atomicOr(a.status, PPO_DEV_BAD_TOKEN);
             }
-            const TokenLoss tl = token_loss(lp, a.old_logprob[row], a.advantages[row], a.values_new[row],
-                                            a.values_old[row], a.returns[row], a.eps, a.eps_v, a.c1, n);
+            const TokenLoss tl = token_loss(lp, t_old, t_adv, t_vn, t_vo, t_ret, a.eps, a.eps_v, a.c1, n);
             a.dvalues[row] = tl.dvalue;
             if (a.new_logprob) a.new_logprob[row] = lp;
             if (a.entropy) a.entropy[row] = H;
@@ -269,33 +138,43 @@ loss_rows_kernel(const LossArgs a)
             if (gs == 0.f) {
                 fill_row_zero<T, VECTOR, THREADS>(dst, V);
             } else {
-                const float ngs = -gs;
+                // -gs * 2^(y - Y) = -+ 2^(y - Y + log2|gs|): the scale rides in the exponent
+                const float off = log2f(fabsf(gs)) - Y;
+                const bool neg = gs > 0.f;
                 if (VECTOR) {
                     constexpr int N = Pack<T>::N;
                     const uint4 *src4 = ROW_IN_SMEM ? row_stage : reinterpret_cast<const uint4 *>(src);
                     uint4 *dst4 = reinterpret_cast<uint4 *>(dst);
                     const int nvec = V / N;
-                    const float nY = -Y;
+                    if (neg) {
 #pragma unroll 2
-                    for (int i = threadIdx.x; i < nvec; i += THREADS) {
-                        const uint4 v = src4[i];
-                        float x[N], xmax, d[N];
-                        Pack<T>::unpack(v, x, xmax);
+                        for (int i = threadIdx.x; i < nvec; i += THREADS) {
+                            float x[N], d[N];
+                            Pack<T>::unpack_raw(src4[i], x);
 #pragma unroll
-                        for (int k = 0; k < N; ++k) d[k] = ngs * ex2(fmaf(x[k], a.c, nY));
-                        st_stream(dst4 + i, Pack<T>::pack(d));
+                            for (int k = 0; k < N; ++k) d[k] = -ex2(fmaf(x[k], a.c, off));
+                            st_stream(dst4 + i, Pack<T>::pack(d));
+                        }
+                    } else {
+#pragma unroll 2
+                        for (int i = threadIdx.x; i < nvec; i += THREADS) {
+                            float x[N], d[N];
+                            Pack<T>::unpack_raw(src4[i], x);
+#pragma unroll
+                            for (int k = 0; k < N; ++k) d[k] = ex2(fmaf(x[k], a.c, off));
+                            st_stream(dst4 + i, Pack<T>::pack(d));
+                        }
                     }
                     // the thread that wrote the pack holding the sampled token adds the one-hot term
                     if (!bad && threadIdx.x == (tok / N) % THREADS) {
-                        const float xt = Pack<T>::load1(src + tok);
-                        Pack<T>::store1(dst + tok, fmaf(ngs, ex2(fmaf(xt, a.c, nY)), gs));
+                        const float e = ex2(fmaf(Pack<T>::load1(src + tok), a.c, off));
+                        Pack<T>::store1(dst + tok, gs + (neg ? -e : e));
                     }
                 } else {
                     const T *src1 = ROW_IN_SMEM ? reinterpret_cast<const T *>(row_stage) : src;
                     for (int j = threadIdx.x; j < V; j += THREADS) {
-                        float x = Pack<T>::load1(src1 + j);
-                        x = (x != x) ? x : fmaxf(x, kNegBig);
-                        float d = ngs * ex2(fmaf(x, a.c, -Y));
+                        const float e = ex2(fmaf(Pack<T>::load1(src1 + j), a.c, off));
+                        float d = neg ? -e : e;
                         if (j == tok) d += gs;
                         Pack<T>::store1(dst + j, d);
                     }
@@ -307,7 +186,6 @@ loss_rows_kernel(const LossArgs a)
 }
 
 // ---------------------------------------------------------------- host side
-static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 template <typename T>
 static int launch_logprob(const void *logits, int64_t rows, int V, int64_t row_stride, const int32_t *tokens,
@@ -318,12 +196,15 @@ static int launch_logprob(const void *logits, int64_t rows, int V, int64_t row_s
     const bool vec = aligned16(logits) && (row_stride * sizeof(T)) % 16 == 0 && V % Pack<T>::N == 0;
     const unsigned grid = (unsigned)(rows < (int64_t)1 << 30 ? rows : (int64_t)1 << 30);
     const T *lg = reinterpret_cast<const T *>(logits);
-    if (vec)
-        logprob_entropy_kernel<T, true, THREADS><<<grid, THREADS, 0, s>>>(lg, rows, V, row_stride, tokens, mask, c,
-                                                                           logprob, entropy, lse, status);
-    else
-        logprob_entropy_kernel<T, false, THREADS><<<grid, THREADS, 0, s>>>(lg, rows, V, row_stride, tokens, mask, c,
-                                                                            logprob, entropy, lse, status);
+#define PPO_LAUNCH_LP(VEC, ENT)                                                                             \
+    logprob_entropy_kernel<T, VEC, ENT, THREADS><<<grid, THREADS, 0, s>>>(lg, rows, V, row_stride, tokens, mask, c, \
+                                                                          logprob, entropy, lse, status)
+    if (vec) {
+        if (entropy) PPO_LAUNCH_LP(true, true); else PPO_LAUNCH_LP(true, false);
+    } else {
+        if (entropy) PPO_LAUNCH_LP(false, true); else PPO_LAUNCH_LP(false, false);
+    }
+#undef PPO_LAUNCH_LP
     return launch_status();
 }
 
@@ -383,6 +264,11 @@ extern "C" int ppo_logprob_entropy(const void *logits, int dtype, int64_t rows, 
     int *status = workspace ? &ws_header(workspace)->status : nullptr;
     const float c = kLog2e / temperature;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    if (option_value(PPO_OPT_ROW_ENGINE) == 2) {
+        const int rc = launch_logprob_bulk(logits, dtype, rows, (int)V, row_stride, tokens, mask, c, logprob, entropy,
+                                           lse, status, s);
+        if (rc != PPO_ERR_UNSUPPORTED) return rc;
+    }
     if (dtype == PPO_F32)
         return launch_logprob<float>(logits, rows, (int)V, row_stride, tokens, mask, c, logprob, entropy, lse,
                                      status, s);
@@ -398,7 +284,8 @@ extern "C" int ppo_loss_fwd_bwd(const void *logits, int dtype, int32_t B, int32_
                                 void *workspace, void *stream)
 {
     if (dtype != PPO_F32 && dtype != PPO_BF16) return PPO_ERR_DTYPE;
-    if (B <= 0 || T <= 0 || V <= 0 || V >= ((int64_t)1 << 31)) return PPO_ERR_SHAPE;
+    if (B <= 0 || T <= 0 || V <= 0 || V >= ((int64_t)1 << 31) || (int64_t)B * T >= ((int64_t)1 << 31))
+        return PPO_ERR_SHAPE;
     if (!logits || !tokens || !mask || !old_logprob || !advantages || !values_new || !values_old || !returns ||
         !p || !losses || !dvalues || !workspace)
         return PPO_ERR_NULL;
@@ -412,7 +299,7 @@ extern "C" int ppo_loss_fwd_bwd(const void *logits, int dtype, int32_t B, int32_
     if (dlogits == logits) return PPO_ERR_PARAM;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     const int64_t rows = (int64_t)B * T;
-    int rc = launch_count_mask(mask, rows, workspace, s);
+    int rc = launch_loss_prepare(mask, rows, workspace, s);
     if (rc) return rc;
     LossArgs a;
     a.logits = logits;
@@ -438,6 +325,11 @@ extern "C" int ppo_loss_fwd_bwd(const void *logits, int dtype, int32_t B, int32_
     a.eps = p->cliprange;
     a.eps_v = p->cliprange_value;
     a.c1 = p->vf_coef;
+    rc = PPO_ERR_UNSUPPORTED;
+    if (option_value(PPO_OPT_ROW_ENGINE) != 1) {
+        rc = launch_loss_bulk(a, dtype, workspace, losses, p->vf_coef, s);
+        if (rc != PPO_ERR_UNSUPPORTED) return rc;      // the engine reduces the partials itself
+    }
     rc = dtype == PPO_F32 ? launch_loss<float>(a, s) : launch_loss<__nv_bfloat16>(a, s);
     if (rc) return rc;
     return launch_loss_finalize(rows, p->vf_coef, losses, workspace, s);

@@ -1,0 +1,566 @@
+// Row engine: persistent thread blocks that stream whole logits rows through shared memory with
+// bulk asynchronous copies (cp.async.bulk, completion counted on mbarriers).
+//
+//   * one producer thread per block issues the copies, 16 KB chunk by chunk, into a shared-memory
+//     buffer that holds exactly one row; 16 consumer warps read the chunks from shared memory;
+//   * every chunk has a "full" barrier (bytes have landed) and an "empty" barrier (all consumer
+//     warps are done with it). A chunk is released as soon as its last reader is done, so the
+//     next row's bytes stream in behind the pass that is still consuming the current row: the
+//     block never drains its loads at a row boundary;
+//   * step 1 (log-prob/entropy) makes one pass and releases chunks as it goes; step 6 (loss)
+//     keeps the row for a second pass that writes the gradient with 16-byte streaming stores and
+//     releases the chunks there. Rows whose mask is 0 are only zero-filled: a filler thread per
+//     block takes them from a shared work counter and writes them with bulk shared->global
+//     copies of a small block of zeros while the consumers work on real rows (the real-row
+//     phase alone leaves HBM bandwidth idle); consumers that run out of real rows join in;
+//   * two blocks per SM while a row is <= 112 KB (bf16, V = 50304), one otherwise.
+//
+// Every wait is bounded: when it runs out the block records PPO_DEV_TIMEOUT in the status word
+// and carries on with the same control flow (so no barrier is left short), which makes the
+// outputs invalid but lets the kernel end.
+#include "ppo_rows.cuh"
+
+namespace ppo {
+
+constexpr int kConsumers = 512;                     // 16 consumer warps
+constexpr int kConsumerWarps = kConsumers / 32;
+constexpr int kEngineThreads = kConsumers + 64;     // + one producer warp + one filler warp
+constexpr int kZeroBytes = 4096;                    // shared zeros, source of the bulk zero-fill stores
+constexpr int kChunkPacks = 2 * kConsumers;         // two packs per consumer thread and chunk
+constexpr int kChunkBytes = kChunkPacks * 16;       // 16 KB
+constexpr int kMaxChunks = 14;                      // 224 KB: the largest row one block can hold
+constexpr uint32_t kWaitTries = 1u << 20;           // x ~1 us per try
+
+struct EngineSmem {
+    unsigned long long full[kMaxChunks];
+    unsigned long long empty[kMaxChunks];
+    float red[96];
+    float bc[4];
+    int next_item;
+    int is_last;
+    double lred[6 * 32];
+    alignas(128) unsigned char zeros[kZeroBytes];
+};
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(unsigned long long *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(unsigned long long *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
+                 : "memory");
+}
+
+// Bounded wait for the phase with the given parity. Returns false (and sets the status bit) if
+// the phase did not complete in time.
+__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, uint32_t parity, int *status)
+{
+    const uint32_t addr = smem_addr(bar);
+    for (uint32_t it = 0; it < kWaitTries; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n"
+            ".reg .pred p;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+            "selp.u32 %0, 1, 0, p;\n"
+            "}\n"
+            : "=r"(ok)
+            : "r"(addr), "r"(parity), "r"(1000u)
+            : "memory");
+        if (ok) return true;
+    }
+    if (status) atomicOr(status, PPO_DEV_TIMEOUT);
+    return false;
+}
+
+// global -> shared bulk copy of `bytes` (multiple of 16; both addresses 16-byte aligned), read
+// once: L2 evict-first
+__device__ __forceinline__ void bulk_load(void *dst_smem, const void *src, uint32_t bytes, unsigned long long *bar,
+                                          uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+        ::"r"(smem_addr(dst_smem)), "l"(src), "r"(bytes), "r"(smem_addr(bar)), "l"(policy)
+        : "memory");
+}
+
+__device__ __forceinline__ uint64_t policy_evict_first()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory"); }
+
+// merge over the 16 consumer warps (named barrier 1); result to every consumer thread
+__device__ __forceinline__ SoftmaxState consumer_merge(SoftmaxState st, float *red, int ct)
+{
+    st = warp_merge(st);
+    const int lane = ct & 31, warp = ct >> 5;
+    if (lane == 0) {
+        red[warp] = st.m;
+        red[32 + warp] = st.s;
+        red[64 + warp] = st.u;
+    }
+    consumer_sync();
+    SoftmaxState t;
+    if (lane < kConsumerWarps) {
+        t.m = red[lane];
+        t.s = red[32 + lane];
+        t.u = red[64 + lane];
+    } else {
+        t.init();
+    }
+    st = warp_merge(t);
+    consumer_sync();
+    return st;
+}
+
+// per-thread statistics with a fixed reference that is only moved when a chunk overflows
+template <typename T, bool ENTROPY>
+struct ThreadStats {
+    float m;          // reference, base-2 units
+    FixedAcc acc;
+    bool have_ref;
+    __device__ __forceinline__ void init()
+    {
+        m = kNegBig;
+        acc.init();
+        have_ref = false;
+    }
+    __device__ __forceinline__ void rebase(float nm)
+    {
+        const float d = m - nm, a = ex2(d);
+        acc.u0 = a * fmaf(d, acc.s0, acc.u0);
+        acc.u1 = a * fmaf(d, acc.s1, acc.u1);
+        acc.s0 *= a;
+        acc.s1 *= a;
+        m = nm;
+    }
+    // fold up to two packs of one chunk
+    __device__ __forceinline__ void chunk(const uint4 &v0, bool h0, const uint4 &v1, bool h1, float c)
+    {
+        if (!h0) return;                      // h1 implies h0
+        if (!have_ref) {
+            float x[Pack<T>::N], xm0, xm1 = kNegBig;
+            Pack<T>::unpack(v0, x, xm0);
+            if (h1) Pack<T>::unpack(v1, x, xm1);
+            m = safe_reference(fmaxf(xm0, xm1), c);
+            have_ref = true;
+        }
+        const FixedAcc save = acc;
+        accumulate_fixed<T, ENTROPY>(v0, c, -m, acc);
+        if (h1) accumulate_fixed<T, ENTROPY>(v1, c, -m, acc);
+        if (!(acc.s0 + acc.s1 < 1.0e35f)) {   // overflow (or NaN): move the reference up and redo the chunk
+            acc = save;
+            float x[Pack<T>::N], xm0, xm1 = kNegBig;
+            Pack<T>::unpack(v0, x, xm0);
+            if (h1) Pack<T>::unpack(v1, x, xm1);
+            const float nm = safe_reference(fmaxf(xm0, xm1), c);
+            if (nm > m) rebase(nm);
+            accumulate_fixed<T, ENTROPY>(v0, c, -m, acc);
+            if (h1) accumulate_fixed<T, ENTROPY>(v1, c, -m, acc);
+        }
+    }
+    __device__ __forceinline__ SoftmaxState state() const
+    {
+        SoftmaxState st;
+        st.m = m;
+        st.s = acc.s0 + acc.s1;
+        st.u = ENTROPY ? acc.u0 + acc.u1 : 0.f;
+        return st;
+    }
+};
+
+struct EngineArgs {
+    // step 1 (MODE 0)
+    const void *logits;
+    int64_t rows;
+    int64_t row_stride;     // elements
+    int V;
+    const int32_t *tokens;
+    const uint8_t *mask;    // MODE 0: nullable
+    float c;
+    float *logprob, *entropy, *lse;
+    int *status;
+    // step 6 (MODE 1)
+    LossArgs loss;
+    const int32_t *order;
+    WorkspaceHeader *hdr;
+    float *losses;
+    float vf_coef;
+};
+
+__device__ __forceinline__ void block_sync_all() { asm volatile("bar.sync 2, %0;" ::"n"(kEngineThreads) : "memory"); }
+
+// End of the loss kernel, reached by every thread of the block once its role is finished: the
+// block takes a ticket; the block that draws the last one sums the per-token partials of the whole
+// batch in a fixed order and writes the loss scalars (so no separate reduction launch is needed
+// and the result does not depend on which block happens to be last).
+__device__ __forceinline__ void engine_epilogue(const EngineArgs &a, EngineSmem &sm)
+{
+    block_sync_all();                       // every partial of this block has been written
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const int ticket = atomicAdd(&a.hdr->done_blocks, 1);
+        sm.is_last = ticket == (int)gridDim.x - 1;
+    }
+    block_sync_all();
+    if (!sm.is_last) return;
+    __threadfence();
+    reduce_loss_partials<kEngineThreads>(a.loss.partials, a.loss.rows, a.hdr->n_tokens, a.vf_coef, a.losses, sm.lred,
+                                         (int)threadIdx.x, [] { block_sync_all(); });
+}
+
+// MODE 0: log-prob/entropy. MODE 1: loss forward + backward.
+template <typename T, int MODE, bool ENTROPY, int MIN_BLOCKS>
+__global__ void __launch_bounds__(kEngineThreads, MIN_BLOCKS)
+row_engine_kernel(const EngineArgs a)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ EngineSmem sm;
+    constexpr int N = Pack<T>::N;
+    const int V = a.V;
+    const int nvec = V / N;
+    const int nch = (nvec + kChunkPacks - 1) / kChunkPacks;
+    const T *logits = reinterpret_cast<const T *>(a.logits);
+    const int64_t stride = MODE == 0 ? a.row_stride : (int64_t)V;
+    // number of work items of the streaming phase and how an item maps to a row
+    const int64_t n_items = MODE == 0 ? a.rows : (int64_t)a.hdr->n_tokens;
+    int *status = a.status;
+
+    if (threadIdx.x == 0) {
+        for (int c = 0; c < nch; ++c) {
+            mbar_init(&sm.full[c], 1);
+            mbar_init(&sm.empty[c], kConsumerWarps);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (MODE == 1) {
+        for (int i = threadIdx.x; i < kZeroBytes / 16; i += kEngineThreads)
+            reinterpret_cast<uint4 *>(sm.zeros)[i] = make_uint4(0u, 0u, 0u, 0u);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // zeros are read by bulk copies
+    }
+    __syncthreads();
+
+    if (threadIdx.x >= kConsumers + 32) {
+        // ------------------------------------------------------------ filler (step 6 only)
+        if (MODE != 1) return;
+        if (threadIdx.x == kConsumers + 32) {
+        const LossArgs &la = a.loss;
+        const int64_t n_masked = la.rows - n_items;
+        const size_t row_bytes = (size_t)V * sizeof(T);
+        for (;;) {
+            const int64_t j = atomicAdd(&a.hdr->masked_next, 1);
+            if (j >= n_masked) break;
+            const int64_t row = a.order[la.rows - 1 - j];
+            unsigned char *dst = reinterpret_cast<unsigned char *>(reinterpret_cast<T *>(la.dlogits) + row * (int64_t)V);
+            for (size_t off = 0; off < row_bytes; off += kZeroBytes) {
+                const uint32_t bytes = (uint32_t)min((size_t)kZeroBytes, row_bytes - off);
+                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst + off),
+                             "r"(smem_addr(sm.zeros)), "r"(bytes)
+                             : "memory");
+            }
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            la.dvalues[row] = 0.f;
+            if (la.new_logprob) la.new_logprob[row] = 0.f;
+            if (la.entropy) la.entropy[row] = 0.f;
+            if (la.dlogprob) la.dlogprob[row] = 0.f;
+            float4 *p4 = reinterpret_cast<float4 *>(la.partials + row * kPartialsPerToken);
+            p4[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+            p4[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+            // keep a bounded number of row-sized groups in flight
+            asm volatile("cp.async.bulk.wait_group.read 4;" ::: "memory");
+        }
+        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all stores done before the block retires
+        }
+        __syncwarp();
+        engine_epilogue(a, sm);
+        return;
+    }
+
+    if (threadIdx.x >= kConsumers) {
+        // ------------------------------------------------------------ producer
+        if (threadIdx.x == kConsumers) {
+        const uint64_t policy = policy_evict_first();
+        uint32_t k = 0;
+        for (int64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+            int64_t row;
+            if (MODE == 0) {
+                row = item;
+                if (a.mask && !a.mask[row]) continue;
+            } else {
+                row = a.order[item];
+            }
+            const unsigned char *src = reinterpret_cast<const unsigned char *>(logits + row * stride);
+            for (int c = 0; c < nch; ++c) {
+                if (k > 0) mbar_wait(&sm.empty[c], (k - 1) & 1, status);
+                const int packs = min(kChunkPacks, nvec - c * kChunkPacks);
+                mbar_expect_tx(&sm.full[c], (uint32_t)packs * 16u);
+                bulk_load(smem_raw + (size_t)c * kChunkBytes, src + (size_t)c * kChunkBytes, (uint32_t)packs * 16u,
+                          &sm.full[c], policy);
+            }
+            ++k;
+        }
+        }
+        if (MODE == 1) {
+            __syncwarp();
+            engine_epilogue(a, sm);
+        }
+        return;
+    }
+
+    // ---------------------------------------------------------------- consumers
+    const int ct = threadIdx.x;
+    const uint4 *buf = reinterpret_cast<const uint4 *>(smem_raw);
+    const double n_tok = MODE == 1 ? (double)a.hdr->n_tokens : 0.0;
+    uint32_t k = 0;
+    for (int64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+        int64_t row;
+        if (MODE == 0) {
+            row = item;
+            if (a.mask && !a.mask[row]) {
+                if (ct == 0) {
+                    a.logprob[row] = 0.f;
+                    if (a.entropy) a.entropy[row] = 0.f;
+                    if (a.lse) a.lse[row] = 0.f;
+                }
+                continue;
+            }
+        } else {
+            row = a.order[item];
+        }
+        const T *src = logits + row * stride;
+        const int tok = a.tokens[row];
+        const bool bad = tok < 0 || tok >= V;
+        float xtok = 0.f, t_old = 0.f, t_adv = 0.f, t_vn = 0.f, t_vo = 0.f, t_ret = 0.f;
+        if (ct == 0) {   // per-token scalars: fetched now, used after the row reduction
+            if (!bad) xtok = Pack<T>::load1(src + tok);
+            if (MODE == 1) {
+                t_old = a.loss.old_logprob[row];
+                t_adv = a.loss.advantages[row];
+                t_vn = a.loss.values_new[row];
+                t_vo = a.loss.values_old[row];
+                t_ret = a.loss.returns[row];
+            }
+        }
+        // ---- pass 1: statistics, chunk by chunk as the bytes land
+        ThreadStats<T, ENTROPY> ts;
+        ts.init();
+        const uint32_t parity = k & 1;
+        for (int c = 0; c < nch; ++c) {
+            mbar_wait(&sm.full[c], parity, status);
+            const int i0 = c * kChunkPacks + ct, i1 = i0 + kConsumers;
+            const bool h0 = i0 < nvec, h1 = i1 < nvec;
+            uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
+            if (h0) v0 = buf[i0];
+            if (h1) v1 = buf[i1];
+            ts.chunk(v0, h0, v1, h1, a.c);
+            if (MODE == 0) {
+                __syncwarp();
+                if ((ct & 31) == 0) mbar_arrive(&sm.empty[c]);
+            }
+        }
+        SoftmaxState st = consumer_merge(ts.state(), sm.red, ct);
+        const float l2s = log2f(st.s);
+        if (MODE == 0) {
+            if (ct == 0) {
+                float lp = (fmaf(xtok, a.c, -st.m) - l2s) * kLn2;
+                float H = (l2s - st.u / st.s) * kLn2;
+                float L = (st.m + l2s) * kLn2;
+                if (bad) {
+                    lp = H = L = __int_as_float(0x7fc00000);
+                    if (status) atomicOr(status, PPO_DEV_BAD_TOKEN);
+                }
+                a.logprob[row] = lp;
+                if (a.entropy) a.entropy[row] = H;
+                if (a.lse) a.lse[row] = L;
+            }
+        } else {
+            const LossArgs &la = a.loss;
+            if (ct == 0) {
+                float lp = (fmaf(xtok, a.c, -st.m) - l2s) * kLn2;
+                float H = (l2s - st.u / st.s) * kLn2;
+                if (bad) {
+                    lp = H = __int_as_float(0x7fc00000);
+                    if (status) atomicOr(status, PPO_DEV_BAD_TOKEN);
+                }
+                const TokenLoss tl = token_loss(lp, t_old, t_adv, t_vn, t_vo, t_ret, la.eps, la.eps_v, la.c1, n_tok);
+                la.dvalues[row] = tl.dvalue;
+                if (la.new_logprob) la.new_logprob[row] = lp;
+                if (la.entropy) la.entropy[row] = H;
+                if (la.dlogprob) la.dlogprob[row] = tl.g;
+                float4 *p4 = reinterpret_cast<float4 *>(la.partials + row * kPartialsPerToken);
+                p4[0] = make_float4(tl.pg, tl.vf, tl.kl, tl.pg_clipped);
+                p4[1] = make_float4(tl.vf_clipped, H, 0.f, 0.f);
+                sm.bc[0] = st.m + l2s;          // log2-sum-exp
+                sm.bc[1] = tl.g * la.inv_tau;   // gradient scale
+            }
+            consumer_sync();
+            const float Y = sm.bc[0], gs = sm.bc[1];
+            // ---- pass 2: gradient row, chunk by chunk; each chunk is handed back to the producer
+            uint4 *dst4 = reinterpret_cast<uint4 *>(reinterpret_cast<T *>(la.dlogits) + row * (int64_t)V);
+            // -gs * 2^(y - Y) = -+ 2^(y - Y + log2|gs|): the scale rides in the exponent
+            const float off = log2f(fabsf(gs)) - Y;
+            const bool zero = gs == 0.f, neg = gs > 0.f;
+            for (int c = 0; c < nch; ++c) {
+                const int i0 = c * kChunkPacks + ct;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int i = i0 + h * kConsumers;
+                    if (i < nvec) {
+                        float x[N], d[N];
+                        Pack<T>::unpack_raw(buf[i], x);
+#pragma unroll
+                        for (int q = 0; q < N; ++q) {
+                            const float e = ex2(fmaf(x[q], a.c, off));
+                            d[q] = zero ? 0.f : (neg ? -e : e);
+                        }
+                        st_stream(dst4 + i, Pack<T>::pack(d));
+                    }
+                }
+                __syncwarp();
+                if ((ct & 31) == 0) mbar_arrive(&sm.empty[c]);
+            }
+            // the thread that wrote the pack holding the sampled token adds the one-hot term
+            if (!zero && !bad && ct == (tok / N) % kConsumers) {
+                const float e = ex2(fmaf(Pack<T>::load1(src + tok), a.c, off));
+                Pack<T>::store1(reinterpret_cast<T *>(dst4) + tok, gs + (neg ? -e : e));
+            }
+        }
+        ++k;
+    }
+
+    if (MODE == 1) {
+        // ---- zero-fill phase: rows with mask 0, handed out by a shared counter
+        const LossArgs &la = a.loss;
+        const int64_t n_masked = a.loss.rows - n_items;
+        const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+        for (;;) {
+            consumer_sync();
+            if (ct == 0) sm.next_item = atomicAdd(&a.hdr->masked_next, 1);
+            consumer_sync();
+            const int64_t j = sm.next_item;
+            if (j >= n_masked) break;
+            const int64_t row = a.order[a.loss.rows - 1 - j];
+            uint4 *dst4 = reinterpret_cast<uint4 *>(reinterpret_cast<T *>(la.dlogits) + row * (int64_t)V);
+            for (int i = ct; i < nvec; i += kConsumers) st_stream(dst4 + i, z);
+            if (ct == 0) {
+                la.dvalues[row] = 0.f;
+                if (la.new_logprob) la.new_logprob[row] = 0.f;
+                if (la.entropy) la.entropy[row] = 0.f;
+                if (la.dlogprob) la.dlogprob[row] = 0.f;
+                float4 *p4 = reinterpret_cast<float4 *>(la.partials + row * kPartialsPerToken);
+                p4[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+                p4[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+        engine_epilogue(a, sm);
+    }
+}
+
+// ---------------------------------------------------------------- host side
+static int sm_count()
+{
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (!cached[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+template <typename T, int MODE, bool ENTROPY>
+static int launch_engine(const EngineArgs &a, int64_t max_items, cudaStream_t s)
+{
+    const size_t row_bytes = (size_t)a.V * sizeof(T);
+    const int nch = (int)((row_bytes + kChunkBytes - 1) / kChunkBytes);
+    if (nch > kMaxChunks) return PPO_ERR_UNSUPPORTED;
+    const size_t smem = (row_bytes + 127) & ~size_t(127);   // the last chunk may be partial
+    const bool two = smem <= 110 * 1024;
+    int64_t grid = (int64_t)sm_count() * (two ? 2 : 1);
+    if (MODE == 0 && max_items < grid) grid = max_items;
+    if (grid < 1) grid = 1;
+    if (two) {
+        auto kern = row_engine_kernel<T, MODE, ENTROPY, 2>;
+        PPO_RETURN_IF_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        kern<<<(unsigned)grid, kEngineThreads, smem, s>>>(a);
+    } else {
+        auto kern = row_engine_kernel<T, MODE, ENTROPY, 1>;
+        PPO_RETURN_IF_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        kern<<<(unsigned)grid, kEngineThreads, smem, s>>>(a);
+    }
+    return launch_status();
+}
+
+template <typename T>
+static bool bulk_ok(const void *base, int64_t stride_elems, int V)
+{
+    return aligned16(base) && (stride_elems * (int64_t)sizeof(T)) % 16 == 0 && V % Pack<T>::N == 0 &&
+           (size_t)V * sizeof(T) <= (size_t)kMaxChunks * kChunkBytes;
+}
+
+int launch_logprob_bulk(const void *logits, int dtype, int64_t rows, int V, int64_t row_stride,
+                        const int32_t *tokens, const uint8_t *mask, float c, float *logprob, float *entropy,
+                        float *lse, int *status, cudaStream_t s)
+{
+    EngineArgs a = {};
+    a.logits = logits;
+    a.rows = rows;
+    a.row_stride = row_stride;
+    a.V = V;
+    a.tokens = tokens;
+    a.mask = mask;
+    a.c = c;
+    a.logprob = logprob;
+    a.entropy = entropy;
+    a.lse = lse;
+    a.status = status;
+    if (dtype == PPO_F32) {
+        if (!bulk_ok<float>(logits, row_stride, V)) return PPO_ERR_UNSUPPORTED;
+        return entropy ? launch_engine<float, 0, true>(a, rows, s) : launch_engine<float, 0, false>(a, rows, s);
+    }
+    if (!bulk_ok<__nv_bfloat16>(logits, row_stride, V)) return PPO_ERR_UNSUPPORTED;
+    return entropy ? launch_engine<__nv_bfloat16, 0, true>(a, rows, s)
+                   : launch_engine<__nv_bfloat16, 0, false>(a, rows, s);
+}
+
+int launch_loss_bulk(const LossArgs &la, int dtype, void *workspace, float *losses, float vf_coef, cudaStream_t s)
+{
+    if (!la.dlogits || !aligned16(la.dlogits)) return PPO_ERR_UNSUPPORTED;
+    EngineArgs a = {};
+    a.logits = la.logits;
+    a.rows = la.rows;
+    a.row_stride = la.V;
+    a.V = la.V;
+    a.tokens = la.tokens;
+    a.mask = la.mask;
+    a.c = la.c;
+    a.status = la.status;
+    a.loss = la;
+    a.order = ws_order(workspace, la.rows);
+    a.hdr = ws_header(workspace);
+    a.losses = losses;
+    a.vf_coef = vf_coef;
+    if (dtype == PPO_F32) {
+        if (!bulk_ok<float>(la.logits, la.V, la.V)) return PPO_ERR_UNSUPPORTED;
+        return launch_engine<float, 1, true>(a, la.rows, s);
+    }
+    if (!bulk_ok<__nv_bfloat16>(la.logits, la.V, la.V)) return PPO_ERR_UNSUPPORTED;
+    return launch_engine<__nv_bfloat16, 1, true>(a, la.rows, s);
+}
+
+}   // namespace ppo

@@ -151,24 +151,48 @@ whiten_kernel(const float *x, const uint8_t *__restrict__ mask, int64_t n_elems,
 // ---------------------------------------------------------------- loss plumbing
 constexpr int kReduceThreads = 1024;
 
+// Prologue of a loss call (one block): counts the real tokens, resets the zero-fill work counter
+// and writes the row order: indices of real rows ascending from the front, masked rows from the
+// back. Each thread owns one contiguous segment of rows, so the order is deterministic.
 __global__ void __launch_bounds__(kReduceThreads)
-count_mask_kernel(const uint8_t *__restrict__ mask, int64_t n_elems, WorkspaceHeader *hdr)
+loss_prepare_kernel(const uint8_t *__restrict__ mask, int64_t rows, WorkspaceHeader *hdr, int32_t *__restrict__ order)
 {
-    __shared__ int red[32];
+    __shared__ int warp_tot[32];
+    const int64_t seg = (rows + kReduceThreads - 1) / kReduceThreads;
+    const int64_t r0 = min(rows, (int64_t)threadIdx.x * seg), r1 = min(rows, r0 + seg);
     int c = 0;
-    for (int64_t i = threadIdx.x; i < n_elems; i += kReduceThreads) c += mask[i] ? 1 : 0;
+    for (int64_t r = r0; r < r1; ++r) c += mask[r] ? 1 : 0;
+    // block exclusive scan of c
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl = c;
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) c += __shfl_xor_sync(0xffffffffu, c, off);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = c;
+    for (int off = 1; off < 32; off <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += t;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
     __syncthreads();
-    if (threadIdx.x < 32) {
-        c = red[threadIdx.x];
+    if (warp == 0) {
+        int w = warp_tot[lane], wi = w;
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) c += __shfl_xor_sync(0xffffffffu, c, off);
-        if (threadIdx.x == 0) {
-            hdr->n_tokens = c;
-            if (c == 0) atomicOr(&hdr->status, PPO_DEV_EMPTY_MASK);
+        for (int off = 1; off < 32; off <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, wi, off);
+            if (lane >= off) wi += t;
         }
+        warp_tot[lane] = wi - w;   // exclusive prefix of the warp totals
+        if (lane == 31) {
+            hdr->n_tokens = wi;
+            hdr->masked_next = 0;
+            hdr->done_blocks = 0;
+            if (wi == 0) atomicOr(&hdr->status, PPO_DEV_EMPTY_MASK);
+        }
+    }
+    __syncthreads();
+    int real_pos = warp_tot[warp] + incl - c;            // real rows before this segment
+    int64_t masked_pos = r0 - real_pos;                   // masked rows before this segment
+    for (int64_t r = r0; r < r1; ++r) {
+        if (mask[r]) order[real_pos++] = (int32_t)r;
+        else order[rows - 1 - masked_pos++] = (int32_t)r;
     }
 }
 
@@ -177,28 +201,9 @@ __global__ void __launch_bounds__(kReduceThreads)
 loss_finalize_kernel(const float *__restrict__ partials, int64_t rows, const WorkspaceHeader *hdr, float vf_coef,
                      float *__restrict__ losses)
 {
-    __shared__ double red[32];
-    double acc[6] = {0, 0, 0, 0, 0, 0};
-    for (int64_t r = threadIdx.x; r < rows; r += kReduceThreads) {
-        const float4 p0 = reinterpret_cast<const float4 *>(partials + r * kPartialsPerToken)[0];
-        const float4 p1 = reinterpret_cast<const float4 *>(partials + r * kPartialsPerToken)[1];
-        acc[0] += p0.x; acc[1] += p0.y; acc[2] += p0.z; acc[3] += p0.w; acc[4] += p1.x; acc[5] += p1.y;
-    }
-#pragma unroll
-    for (int k = 0; k < 6; ++k) acc[k] = block_sum<kReduceThreads>(acc[k], red);
-    if (threadIdx.x == 0) {
-        const double n = (double)hdr->n_tokens;
-        const double inv = n > 0.0 ? 1.0 / n : 0.0;
-        const double pg = acc[0] * inv, vf = 0.5 * acc[1] * inv;
-        losses[PPO_LOSS_PG] = (float)pg;
-        losses[PPO_LOSS_VF] = (float)vf;
-        losses[PPO_LOSS_TOTAL] = (float)(pg + (double)vf_coef * vf);
-        losses[PPO_LOSS_APPROX_KL] = (float)(acc[2] * inv);
-        losses[PPO_LOSS_PG_CLIPFRAC] = (float)(acc[3] * inv);
-        losses[PPO_LOSS_VF_CLIPFRAC] = (float)(acc[4] * inv);
-        losses[PPO_LOSS_ENTROPY] = (float)(acc[5] * inv);
-        losses[PPO_LOSS_N] = (float)n;
-    }
+    __shared__ double red[6 * 32];
+    reduce_loss_partials<kReduceThreads>(partials, rows, hdr->n_tokens, vf_coef, losses, red, (int)threadIdx.x,
+                                         [] { __syncthreads(); });
 }
 
 // Step 6 at log-prob level (the logits were never materialised): one thread per token.
@@ -228,9 +233,9 @@ loss_from_logprob_kernel(const float *__restrict__ new_logprob, const float *__r
     dvalues[r] = dv;
 }
 
-int launch_count_mask(const uint8_t *mask, int64_t n_elems, void *workspace, cudaStream_t s)
+int launch_loss_prepare(const uint8_t *mask, int64_t rows, void *workspace, cudaStream_t s)
 {
-    count_mask_kernel<<<1, kReduceThreads, 0, s>>>(mask, n_elems, ws_header(workspace));
+    loss_prepare_kernel<<<1, kReduceThreads, 0, s>>>(mask, rows, ws_header(workspace), ws_order(workspace, rows));
     return launch_status();
 }
 
@@ -265,7 +270,8 @@ extern "C" int ppo_version(void) { return 100; }
 
 extern "C" int ppo_set_option(int key, int value)
 {
-    if (key == PPO_OPT_LOSS_ROW_CACHE && value >= 0 && value <= 2) {
+    if ((key == PPO_OPT_LOSS_ROW_CACHE && value >= 0 && value <= 2) ||
+        (key == PPO_OPT_ROW_ENGINE && value >= 0 && value <= 2)) {
         g_options[key] = value;
         return PPO_OK;
     }
@@ -276,7 +282,8 @@ extern "C" size_t ppo_workspace_bytes(int32_t B, int32_t T, int64_t V)
 {
     (void)V;
     if (B <= 0 || T <= 0) return kHeaderBytes;
-    return kHeaderBytes + align256((size_t)B * (size_t)T * kPartialsPerToken * sizeof(float));
+    const size_t rows = (size_t)B * (size_t)T;
+    return kHeaderBytes + align256(rows * kPartialsPerToken * sizeof(float)) + align256(rows * sizeof(int32_t));
 }
 
 extern "C" int ppo_workspace_init(void *workspace, size_t bytes, void *stream)
@@ -361,7 +368,7 @@ extern "C" int ppo_loss_from_logprob(const float *new_logprob, const float *entr
                                      const ppo_params *p, float *losses, float *dlogprob, float *dvalues,
                                      void *workspace, void *stream)
 {
-    if (B <= 0 || T <= 0) return PPO_ERR_SHAPE;
+    if (B <= 0 || T <= 0 || (int64_t)B * T >= ((int64_t)1 << 31)) return PPO_ERR_SHAPE;
     if (!new_logprob || !mask || !old_logprob || !advantages || !values_new || !values_old || !returns || !p ||
         !losses || !dvalues || !workspace)
         return PPO_ERR_NULL;
@@ -369,7 +376,7 @@ extern "C" int ppo_loss_from_logprob(const float *new_logprob, const float *entr
     if (reinterpret_cast<uintptr_t>(workspace) % 256) return PPO_ERR_ALIGN;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     const int64_t rows = (int64_t)B * T;
-    int rc = launch_count_mask(mask, rows, workspace, s);
+    int rc = launch_loss_prepare(mask, rows, workspace, s);
     if (rc) return rc;
     loss_from_logprob_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, s>>>(
         new_logprob, entropy, rows, mask, old_logprob, advantages, values_new, values_old, returns, p->cliprange,

@@ -24,10 +24,19 @@ def _rand_logits(rows, V, dtype, seed, std=2.0):
     return (std * torch.randn((rows, V), generator=g, device="cuda")).to(dtype)
 
 
+@pytest.fixture(params=[0, 2], ids=["direct", "engine"])
+def lp_engine(request, P):
+    """Run log-prob/entropy through the direct-load kernels (default) and through the row engine."""
+    from paper_2403_17031_b200 import binding
+    P.set_option(binding.OPT_ROW_ENGINE, request.param)
+    yield request.param
+    P.set_option(binding.OPT_ROW_ENGINE, 0)
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("V", [1, 7, 1000, 1001, 4099, 50304, 65536 + 24])
-def test_logprob_entropy_shapes(P, oracle, dtype, V):
-    rows = 37
+def test_logprob_entropy_shapes(P, oracle, dtype, V, lp_engine):
+    rows = 700 if (V == 50304 and dtype == torch.bfloat16) else 37   # more rows than blocks: several rows per block
     x = _rand_logits(rows, V, dtype, seed=V)
     tok = torch.randint(0, V, (rows,), device="cuda", dtype=torch.int32)
     lp, ent, lse = P.logprob_entropy(x, tok, 0.7, want_lse=True)
@@ -55,7 +64,7 @@ def test_logprob_entropy_strided_rows_and_unaligned_base(P, oracle):
     assert_abs(npy(ent), rent, TOL_LOGPROB, "entropy")
 
 
-def test_uniform_and_peaked_rows(P):
+def test_uniform_and_peaked_rows(P, lp_engine):
     V = 50304
     x = torch.full((3, V), 1.25, device="cuda", dtype=torch.bfloat16)
     x[1, 17] = 60.0                                   # one dominant logit
@@ -68,7 +77,27 @@ def test_uniform_and_peaked_rows(P):
     assert abs(float(lp[2]) + lnV) < 1e-4
 
 
-def test_neg_inf_logits_and_bad_tokens(P, oracle):
+def test_wide_range_rows_take_the_rebase_path(P, oracle, lp_engine):
+    """Rows whose later elements exceed the first ones by far more than 2^127 in base-2 units."""
+    V = 50304
+    x = torch.full((6, V), -300.0, device="cuda", dtype=torch.float32)
+    x[0, 40000] = 250.0
+    x[1, 5] = 100.0; x[1, 50000] = 320.0
+    x[2, ::977] = 90.0; x[2, 30011] = 400.0
+    x[3] = torch.linspace(-500, 500, V, device="cuda")
+    x[4] = torch.linspace(500, -500, V, device="cuda")
+    x[5, 123] = float("-inf")
+    for dt in (torch.float32, torch.bfloat16):
+        xx = x.to(dt)
+        tok = torch.tensor([40000, 5, 30011, V - 1, 3, 7], device="cuda", dtype=torch.int32)
+        lp, ent, lse = P.logprob_entropy(xx, tok, 0.7, want_lse=True)
+        rlp, rent, rlse = oracle.logprob_entropy(host_logits(xx), npy(tok), np.float32(0.7))
+        assert_abs(npy(lp), rlp, 2e-4, "logprob")          # |lse| reaches ~700: fp32 resolution there is 6e-5
+        assert_abs(npy(ent), rent, TOL_LOGPROB, "entropy")
+        assert_rel(npy(lse), rlse, 1e-6, "lse")
+
+
+def test_neg_inf_logits_and_bad_tokens(P, oracle, lp_engine):
     V = 4096
     x = _rand_logits(4, V, torch.float32, seed=7)
     x[0, 100:] = float("-inf")
@@ -170,6 +199,7 @@ def test_loss_kernel_variants(P, oracle, dtype, V, mode):
                               np.float32(0.2), np.float32(0.2), np.float32(0.1))
     ws = P.new_workspace(P.workspace_bytes(B, T, V))
     P.set_option(binding.OPT_LOSS_ROW_CACHE, mode)
+    P.set_option(binding.OPT_ROW_ENGINE, 1 if mode else 0)     # modes 1, 2 select among the direct-load kernels
     try:
         o = P.loss_fwd_bwd(lg, tok, dev(m), dev(old), dev(adv), dev(vn), dev(vo), dev(ret), P.default_params(), ws)
         o_b = P.loss_fwd_bwd(lg, tok, dev(m), dev(old), dev(adv), dev(vn), dev(vo), dev(ret), P.default_params(), ws)
@@ -177,6 +207,7 @@ def test_loss_kernel_variants(P, oracle, dtype, V, mode):
                              want_dlogits=False)
     finally:
         P.set_option(binding.OPT_LOSS_ROW_CACHE, 0)
+        P.set_option(binding.OPT_ROW_ENGINE, 0)
     n = ref["losses"][7]
     assert_abs(npy(o["losses"]), ref["losses"], TOL_LOGPROB, "losses")
     assert_abs(npy(o["new_logprob"]), ref["new_logprob"], TOL_LOGPROB, "new_logprob")

@@ -45,7 +45,7 @@ def test_defaults_are_the_papers_table(L):
 
 def test_workspace_sizes(L):
     from paper_2403_17031_b200 import binding
-    assert binding.workspace_bytes(64, 53, 50304) == 256 + ((64 * 53 * 32 + 255) // 256) * 256
+    assert binding.workspace_bytes(64, 53, 50304) == 256 + ((64 * 53 * 32 + 255) // 256) * 256 + ((64 * 53 * 4 + 255) // 256) * 256
     assert binding.workspace_bytes(0, 53, 50304) == 256
     assert binding.workspace_bytes(512, 53, 50304) % 256 == 0
     assert binding.lmhead_workspace_bytes(27136, 4096, 50304) % 256 == 0
