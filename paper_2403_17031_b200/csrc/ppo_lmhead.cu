@@ -1,15 +1,433 @@
-// Step 7: LM-head GEMM fused with the log-prob / entropy reduction (placeholder translation
-// unit; the tcgen05 kernel is added separately).
+// Step 7: LM-head GEMM fused with the log-prob / entropy reduction. The logits H.W are formed tile
+// by tile on the 5th-generation tensor cores and consumed straight out of tensor memory; they are
+// never written to global memory.
+//
+// One persistent block per SM, 192 threads in three roles:
+//   warp 0 (one lane)   TMA producer: 128x64 tiles of H (K-major) and 64x256 tiles of W (vocabulary-
+//                       major, as stored: W is [K,V] row-major) into a 4-stage shared-memory ring,
+//                       128-byte swizzle, completion counted on mbarriers
+//   warp 1 (one lane)   issues tcgen05.mma (M=128, N=256, K=16, bf16 x bf16 -> fp32) into one of two
+//                       256-column accumulators in tensor memory; tcgen05.commit releases the ring
+//                       slot and, after the last k-block, hands the accumulator to the epilogue
+//   warps 2-5           epilogue: thread r owns logits row r of the tile; tcgen05.ld 32 columns at a
+//                       time and fold them into that row's running softmax state (fixed reference,
+//                       one ex2 per logit), picking up the sampled token's logit on the way
+// While the epilogue drains one accumulator the tensor core fills the other.
+//
+// Work unit = (row tile of 128, chunk of 6 vocabulary tiles of 256). Units are ordered so that the
+// blocks running at the same time share the same W columns and a small set of H tiles (both stay
+// in L2); block b takes units b, b+grid, ... Each unit leaves one partial state per row in the
+// workspace; a second small kernel merges a row's partials in chunk order and writes log-prob,
+// entropy and lse.
+//
+// Every wait is bounded; a wait that runs out sets PPO_DEV_TIMEOUT and the block carries on with the
+// same control flow, so it still reaches the end, frees its tensor memory and returns.
+#include <cuda.h>
+
 #include "ppo_common.cuh"
+
+namespace ppo {
+
+constexpr int kBlockM = 128, kBlockN = 256, kBlockK = 64;
+constexpr int kStages = 4;
+constexpr int kABytes = kBlockM * kBlockK * 2;          // 16 KB
+constexpr int kBBoxBytes = 64 * kBlockK * 2;            // 8 KB: one 64(N) x 64(K) box of W
+constexpr int kBBytes = (kBlockN / 64) * kBBoxBytes;    // 32 KB
+constexpr int kStageBytes = kABytes + kBBytes;          // 48 KB
+constexpr int kLmThreads = 192;
+constexpr int kTilesPerChunk = 6;                       // vocabulary tiles per work unit
+constexpr int kRowGroup = 37;                           // row tiles that sweep the vocabulary together
+constexpr int kTmemCols = 512;
+constexpr uint32_t kLmWaitTries = 1u << 19;         // x up to ~2 us per try
+constexpr uint32_t kAbsentBits = 0xffffffffu;           // "this chunk does not hold the sampled token"
+
+struct LmSmem {
+    unsigned long long full[kStages], empty[kStages], tmem_full[2], tmem_empty[2];
+    uint32_t tmem_base;
+};
+
+__device__ __forceinline__ uint32_t lm_smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ bool lm_wait(unsigned long long *bar, uint32_t parity, int *status)
+{
+    const uint32_t addr = lm_smem_addr(bar);
+    for (uint32_t it = 0; it < kLmWaitTries; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n"
+            ".reg .pred p;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+            "selp.u32 %0, 1, 0, p;\n"
+            "}\n"
+            : "=r"(ok)
+            : "r"(addr), "r"(parity), "r"(2000u)
+            : "memory");
+        if (ok) return true;
+    }
+    atomicOr(status, PPO_DEV_TIMEOUT);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int x, int y, unsigned long long *bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(lm_smem_addr(dst)), "l"(map), "r"(x), "r"(y), "r"(lm_smem_addr(bar))
+        : "memory");
+}
+
+// shared-memory matrix descriptor: 128-byte swizzle, version 1; offsets in 16-byte units
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3fff);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3fff) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fff) << 32;
+    d |= (uint64_t)1 << 46;    // descriptor version (sm_100)
+    d |= (uint64_t)2 << 61;    // SWIZZLE_128B
+    return d;
+}
+
+// instruction descriptor: D fp32, A and B bf16, A K-major, B MN-major, M = 128, N = 256
+constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
+                                ((uint32_t)(kBlockN >> 3) << 17) | ((uint32_t)(kBlockM >> 4) << 24);
+
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n"
+        "}\n"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(kInstrDesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
+
+__device__ __forceinline__ void umma_commit(unsigned long long *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(lm_smem_addr(bar))
+                 : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+
+struct LmUnit {
+    int m_tile, chunk;
+};
+
+// unit index -> (row tile, vocabulary chunk): row tiles in groups of kRowGroup; inside a group the
+// chunk index moves slowest, so consecutive units share W columns
+__device__ __forceinline__ LmUnit lm_unit(int u, int m_tiles, int n_chunks)
+{
+    const int per_group = kRowGroup * n_chunks;
+    const int g = u / per_group;
+    const int gsize = min(kRowGroup, m_tiles - g * kRowGroup);
+    const int local = u - g * per_group;
+    LmUnit r;
+    r.chunk = local / gsize;
+    r.m_tile = g * kRowGroup + (local - r.chunk * gsize);
+    return r;
+}
+
+struct LmArgs {
+    int M, K, V;
+    int m_tiles, n_tiles, n_chunks, n_units;
+    const int32_t *tokens;
+    float c;
+    float4 *partials;     // [m_tiles*128][n_chunks]
+    int *status;
+};
+
+__global__ void __launch_bounds__(kLmThreads, 1)
+lmhead_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w, const LmArgs a)
+{
+    extern __shared__ __align__(1024) unsigned char lm_smem_raw[];
+    __shared__ LmSmem sm;
+    // the ring must start on a 1024-byte boundary (swizzle atoms)
+    unsigned char *ring = lm_smem_raw + ((1024u - (lm_smem_addr(lm_smem_raw) & 1023u)) & 1023u);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int k_blocks = a.K / kBlockK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(lm_smem_addr(&sm.full[s])) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(lm_smem_addr(&sm.empty[s])) : "memory");
+        }
+        for (int b = 0; b < 2; ++b) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(lm_smem_addr(&sm.tmem_full[b])) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 4;" ::"r"(lm_smem_addr(&sm.tmem_empty[b])) : "memory");
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {   // one warp allocates all 512 columns of tensor memory
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(lm_smem_addr(&sm.tmem_base)),
+                     "r"((uint32_t)kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = sm.tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            for (int u = blockIdx.x; u < a.n_units; u += gridDim.x) {
+                const LmUnit un = lm_unit(u, a.m_tiles, a.n_chunks);
+                const int t0 = un.chunk * kTilesPerChunk, t1 = min(t0 + kTilesPerChunk, a.n_tiles);
+                for (int t = t0; t < t1; ++t) {
+                    for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+                        const int s = it % kStages;
+                        if (it >= kStages) lm_wait(&sm.empty[s], ((it / kStages) - 1) & 1, a.status);
+                        unsigned char *stage = ring + (size_t)s * kStageBytes;
+                        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(lm_smem_addr(&sm.full[s])),
+                                     "r"((uint32_t)kStageBytes)
+                                     : "memory");
+                        tma_load_2d(stage, &map_h, kb * kBlockK, un.m_tile * kBlockM, &sm.full[s]);
+#pragma unroll
+                        for (int j = 0; j < kBlockN / 64; ++j)
+                            tma_load_2d(stage + kABytes + j * kBBoxBytes, &map_w, t * kBlockN + j * 64, kb * kBlockK,
+                                        &sm.full[s]);
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t it = 0, tc = 0;
+            for (int u = blockIdx.x; u < a.n_units; u += gridDim.x) {
+                const LmUnit un = lm_unit(u, a.m_tiles, a.n_chunks);
+                const int t0 = un.chunk * kTilesPerChunk, t1 = min(t0 + kTilesPerChunk, a.n_tiles);
+                for (int t = t0; t < t1; ++t, ++tc) {
+                    const uint32_t buf = tc & 1;
+                    if (tc >= 2) lm_wait(&sm.tmem_empty[buf], ((tc >> 1) - 1) & 1, a.status);
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t tmem_d = tmem_base + buf * kBlockN;
+                    for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+                        const int s = it % kStages;
+                        lm_wait(&sm.full[s], (it / kStages) & 1, a.status);
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        const uint32_t a_addr = lm_smem_addr(ring + (size_t)s * kStageBytes);
+                        const uint32_t b_addr = a_addr + kABytes;
+#pragma unroll
+                        for (int kk = 0; kk < kBlockK / 16; ++kk) {
+                            // A: K-major, 8-row groups 1024 B apart; 16 K-elements = 32 bytes further
+                            const uint64_t ad = smem_desc(a_addr + kk * 32, 16, 1024);
+                            // B: vocabulary-major; 64-column boxes 8192 B apart, 8 K-rows 1024 B apart;
+                            //    16 K-rows = 2048 bytes further
+                            const uint64_t bd = smem_desc(b_addr + kk * 2048, kBBoxBytes, 1024);
+                            umma(tmem_d, ad, bd, (kb | kk) ? 1u : 0u);
+                        }
+                        umma_commit(&sm.empty[s]);            // ring slot is free once these MMAs have read it
+                    }
+                    umma_commit(&sm.tmem_full[buf]);          // accumulator complete
+                }
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5)
+        const int q = warp & 3;                      // tensor-memory lane quarter this warp may read
+        const int row_in_tile = q * 32 + lane;
+        uint32_t tc = 0;
+        for (int u = blockIdx.x; u < a.n_units; u += gridDim.x) {
+            const LmUnit un = lm_unit(u, a.m_tiles, a.n_chunks);
+            const int t0 = un.chunk * kTilesPerChunk, t1 = min(t0 + kTilesPerChunk, a.n_tiles);
+            const int row = un.m_tile * kBlockM + row_in_tile;
+            const bool row_ok = row < a.M;
+            const int tok = row_ok ? a.tokens[row] : -1;
+            float m = 0.f, s0 = 0.f, s1 = 0.f, u0 = 0.f, u1 = 0.f;
+            bool have_ref = false;
+            uint32_t xtok_bits = kAbsentBits;
+            for (int t = t0; t < t1; ++t, ++tc) {
+                const uint32_t buf = tc & 1;
+                lm_wait(&sm.tmem_full[buf], (tc >> 1) & 1, a.status);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t taddr = tmem_base + buf * kBlockN + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+                for (int cc = 0; cc < kBlockN / 32; ++cc) {
+                    uint32_t r[32];
+                    __syncwarp();                            // the aligned tensor-memory load needs a converged warp
+                    tmem_ld32(taddr + cc * 32, r);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (cc == kBlockN / 32 - 1) {
+                        // all of this warp's reads of the accumulator are done: hand it back
+                        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                        __syncwarp();
+                        if (lane == 0)
+                            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(lm_smem_addr(&sm.tmem_empty[buf]))
+                                         : "memory");
+                    }
+                    const int col0 = t * kBlockN + cc * 32;
+                    if (col0 >= a.V) continue;
+                    const int ncol = min(32, a.V - col0);
+                    if ((unsigned)(tok - col0) < (unsigned)ncol) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (tok - col0 == j) xtok_bits = r[j];
+                    }
+                    if (!have_ref) {
+                        float mx = __uint_as_float(r[0]);
+#pragma unroll
+                        for (int j = 1; j < 32; ++j)
+                            if (j < ncol) mx = fmaxf(mx, __uint_as_float(r[j]));
+                        m = mx * a.c;
+                        have_ref = true;
+                    }
+                    for (int attempt = 0; attempt < 2; ++attempt) {
+                        const float nm = -m;
+                        float a0 = s0, a1 = s1, b0 = u0, b1 = u1;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 2) {
+                            const float ta = fmaf(__uint_as_float(r[j]), a.c, nm);
+                            const float tb = fmaf(__uint_as_float(r[j + 1]), a.c, nm);
+                            const float ea = j < ncol ? ex2(ta) : 0.f, eb = j + 1 < ncol ? ex2(tb) : 0.f;
+                            a0 += ea;
+                            a1 += eb;
+                            b0 = fmaf(ea, j < ncol ? ta : 0.f, b0);
+                            b1 = fmaf(eb, j + 1 < ncol ? tb : 0.f, b1);
+                        }
+                        if (a0 + a1 < 1.0e35f || attempt == 1) {
+                            s0 = a0; s1 = a1; u0 = b0; u1 = b1;
+                            break;
+                        }
+                        // overflow: move the reference up to this chunk's maximum and redo the chunk
+                        float mx = __uint_as_float(r[0]);
+#pragma unroll
+                        for (int j = 1; j < 32; ++j)
+                            if (j < ncol) mx = fmaxf(mx, __uint_as_float(r[j]));
+                        const float m2 = fmaxf(m, mx * a.c);
+                        const float d = m - m2, sc = ex2(d);
+                        u0 = sc * fmaf(d, s0, u0);
+                        u1 = sc * fmaf(d, s1, u1);
+                        s0 *= sc;
+                        s1 *= sc;
+                        m = m2;
+                    }
+                }
+            }
+            if (row_ok)
+                a.partials[(size_t)row * a.n_chunks + un.chunk] =
+                    make_float4(m, s0 + s1, u0 + u1, __uint_as_float(xtok_bits));
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols)
+                     : "memory");
+    }
+}
+
+// merge the chunk partials of each row in chunk order; one thread per row
+__global__ void __launch_bounds__(256)
+lmhead_finalize_kernel(const float4 *__restrict__ partials, int M, int V, int n_chunks, const int32_t *__restrict__ tokens,
+                       const uint8_t *__restrict__ mask, float c, float *__restrict__ logprob,
+                       float *__restrict__ entropy, float *__restrict__ lse, int *status)
+{
+    const int row = blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= M) return;
+    float lp = 0.f, H = 0.f, L = 0.f;
+    if (!mask || mask[row]) {
+        SoftmaxState st;
+        st.init();
+        uint32_t xbits = kAbsentBits;
+        for (int k = 0; k < n_chunks; ++k) {
+            const float4 p = partials[(size_t)row * n_chunks + k];
+            SoftmaxState o;
+            o.m = p.x;
+            o.s = p.y;
+            o.u = p.z;
+            st = merge(st, o);
+            if (__float_as_uint(p.w) != kAbsentBits) xbits = __float_as_uint(p.w);
+        }
+        const int tok = tokens[row];
+        const float l2s = log2f(st.s);
+        if (tok < 0 || tok >= V || xbits == kAbsentBits) {
+            lp = H = L = __int_as_float(0x7fc00000);
+            atomicOr(status, PPO_DEV_BAD_TOKEN);
+        } else {
+            lp = (fmaf(__uint_as_float(xbits), c, -st.m) - l2s) * kLn2;
+            H = (l2s - st.u / st.s) * kLn2;
+            L = (st.m + l2s) * kLn2;
+        }
+    }
+    logprob[row] = lp;
+    if (entropy) entropy[row] = H;
+    if (lse) lse[row] = L;
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2-D bf16 tensor [outer, inner] (inner contiguous), box [box_outer, 64], 128-byte swizzle
+static int make_map(CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint32_t box_outer)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return (int)cudaErrorNotSupported;
+    const cuuint64_t dims[2] = {inner, outer};
+    const cuuint64_t strides[1] = {inner * 2};
+    const cuuint32_t box[2] = {64, box_outer};
+    const cuuint32_t elem[2] = {1, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, elem,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? PPO_OK : (int)cudaErrorInvalidValue;
+}
+
+static void lm_shape(int64_t M, int64_t V, int *m_tiles, int *n_tiles, int *n_chunks)
+{
+    *m_tiles = (int)((M + kBlockM - 1) / kBlockM);
+    *n_tiles = (int)((V + kBlockN - 1) / kBlockN);
+    *n_chunks = (*n_tiles + kTilesPerChunk - 1) / kTilesPerChunk;
+}
+
+}   // namespace ppo
 
 using namespace ppo;
 
 extern "C" size_t ppo_lmhead_workspace_bytes(int64_t M, int64_t K, int64_t V)
 {
     (void)K;
-    (void)V;
-    if (M <= 0) return kHeaderBytes;
-    return kHeaderBytes + align256((size_t)M * 64);
+    if (M <= 0 || V <= 0) return kHeaderBytes;
+    int m_tiles, n_tiles, n_chunks;
+    lm_shape(M, V, &m_tiles, &n_tiles, &n_chunks);
+    return kHeaderBytes + align256((size_t)m_tiles * kBlockM * (size_t)n_chunks * sizeof(float4));
 }
 
 extern "C" int ppo_lmhead_logprob_entropy(const void *H, const void *W, int64_t M, int64_t K, int64_t V,
@@ -17,7 +435,47 @@ extern "C" int ppo_lmhead_logprob_entropy(const void *H, const void *W, int64_t 
                                           float *logprob, float *entropy, float *lse, void *workspace,
                                           void *stream)
 {
-    (void)H; (void)W; (void)M; (void)K; (void)V; (void)tokens; (void)mask; (void)temperature;
-    (void)logprob; (void)entropy; (void)lse; (void)workspace; (void)stream;
-    return PPO_ERR_UNSUPPORTED;
+    if (M < 0 || K <= 0 || V <= 0 || M >= ((int64_t)1 << 31) - kBlockM || V >= ((int64_t)1 << 31) - kBlockN ||
+        K >= ((int64_t)1 << 31))
+        return PPO_ERR_SHAPE;
+    if (!(temperature > 0.f) || !finite_f(temperature)) return PPO_ERR_PARAM;
+    if (M == 0) return PPO_OK;
+    if (!H || !W || !tokens || !logprob || !workspace) return PPO_ERR_NULL;
+    if (K % kBlockK != 0 || V % 8 != 0) return PPO_ERR_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(H) % 16 || reinterpret_cast<uintptr_t>(W) % 16 ||
+        reinterpret_cast<uintptr_t>(workspace) % 256)
+        return PPO_ERR_ALIGN;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+
+    LmArgs a;
+    a.M = (int)M;
+    a.K = (int)K;
+    a.V = (int)V;
+    lm_shape(M, V, &a.m_tiles, &a.n_tiles, &a.n_chunks);
+    const int64_t units = (int64_t)a.m_tiles * a.n_chunks;
+    if (units >= ((int64_t)1 << 31)) return PPO_ERR_SHAPE;
+    a.n_units = (int)units;
+    a.tokens = tokens;
+    a.c = kLog2e / temperature;
+    a.partials = reinterpret_cast<float4 *>(reinterpret_cast<unsigned char *>(workspace) + kHeaderBytes);
+    a.status = &ws_header(workspace)->status;
+
+    CUtensorMap map_h, map_w;
+    int rc = make_map(&map_h, H, (uint64_t)K, (uint64_t)M, kBlockM);
+    if (rc) return rc;
+    rc = make_map(&map_w, W, (uint64_t)V, (uint64_t)K, kBlockK);
+    if (rc) return rc;
+
+    int dev = 0, sms = 148;
+    PPO_RETURN_IF_CUDA(cudaGetDevice(&dev));
+    PPO_RETURN_IF_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const size_t smem = (size_t)kStages * kStageBytes + 1024;   // + slack to align the ring to 1024 bytes
+    PPO_RETURN_IF_CUDA(cudaFuncSetAttribute(lmhead_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const int grid = a.n_units < sms ? a.n_units : sms;
+    lmhead_kernel<<<grid, kLmThreads, smem, s>>>(map_h, map_w, a);
+    rc = launch_status();
+    if (rc) return rc;
+    lmhead_finalize_kernel<<<(unsigned)((M + 255) / 256), 256, 0, s>>>(a.partials, a.M, a.V, a.n_chunks, tokens, mask, a.c,
+                                                                       logprob, entropy, lse, a.status);
+    return launch_status();
 }
