@@ -232,6 +232,31 @@ int ppo_loss_from_logprob(const float *new_logprob, const float *entropy, int32_
                           float *dvalues, void *workspace, void *stream);
 
 /*
+ * Allocation-free variant of ppo_loss_from_logprob (an addition of this library; the paper has no
+ * counterpart).  It is meant for callers that cannot obtain device memory at the point of the call:
+ * code running under a framework whose allocator must not be re-entered, inside a region where
+ * cudaMalloc is forbidden or would synchronise the device, or in a process whose memory budget
+ * has been handed out in full.  Its scratch (what the other entry point takes as `workspace`) is
+ * a fixed array built into the library: 256 + 36 * PPO_STATIC_MAX_TOKENS bytes (about 1.2 MB) of
+ * device memory on every GPU that loads the library, held until the process exits.
+ *   - Same arguments, results and error codes as ppo_loss_from_logprob, minus `workspace`;
+ *     B*T > PPO_STATIC_MAX_TOKENS returns PPO_ERR_UNSUPPORTED before anything is launched.
+ *   - Neither this call nor anything it uses calls cudaMalloc, cudaFree or an allocating library
+ *     routine.  The first call on each device looks up the array's device address (with that
+ *     device current); make that first call outside any stream capture.
+ *   - All calls share the one array and it keeps the last call's contents; each call rewrites what
+ *     it reads and clears the status word itself.  Two calls that overlap on the same GPU (different
+ *     streams, or different host threads) race on it: serialise them.
+ *   - There is no status word to read back; an all-zero mask shows as losses[PPO_LOSS_N] == 0.
+ */
+#define PPO_STATIC_MAX_TOKENS 32768
+int ppo_loss_from_logprob_static(const float *new_logprob, const float *entropy, int32_t B, int32_t T,
+                                 const uint8_t *mask, const float *old_logprob, const float *advantages,
+                                 const float *values_new, const float *values_old, const float *returns,
+                                 const ppo_params *p /* host */, float *losses, float *dlogprob,
+                                 float *dvalues, void *stream);
+
+/*
  * Step 7 (fused LM head): logits[r, :] = H[r, :] . W are formed tile by tile on the tensor
  * cores (bf16 inputs, fp32 accumulation in tensor memory) and consumed by step 1's reduction
  * in the epilogue; they are never written to memory.

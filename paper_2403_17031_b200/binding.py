@@ -62,6 +62,8 @@ _SIGS = {
                          [C.POINTER(PPOParams)] + [C.c_void_p] * 8),
     "ppo_loss_from_logprob": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32] + [C.c_void_p] * 6 +
                               [C.POINTER(PPOParams)] + [C.c_void_p] * 5),
+    "ppo_loss_from_logprob_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32] + [C.c_void_p] * 6 +
+                                     [C.POINTER(PPOParams)] + [C.c_void_p] * 4),
     "ppo_lmhead_logprob_entropy": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p,
                                              C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                              C.c_void_p]),
@@ -287,6 +289,24 @@ def loss_from_logprob(new_logprob, entropy, mask, old_logprob, advantages, value
                                      _ptr(out["losses"], f32), _ptr(out["dlogprob"], f32), _ptr(out["dvalues"], f32),
                                      _ptr(workspace), _stream())
     _check("ppo_loss_from_logprob", rc)
+    return out
+
+
+STATIC_MAX_TOKENS = 32768
+
+
+def loss_from_logprob_static(new_logprob, entropy, mask, old_logprob, advantages, values_new, values_old, returns,
+                             params: PPOParams, out):
+    """Allocation-free variant of loss_from_logprob: scratch is built into the library, and `out`
+    (dict with preallocated losses[8], dlogprob, dvalues) is mandatory so that nothing here allocates."""
+    B, T = new_logprob.shape
+    f32 = torch.float32
+    rc = lib().ppo_loss_from_logprob_static(_ptr(new_logprob, f32), _ptr(entropy, f32), B, T, _ptr(mask, torch.uint8),
+                                            _ptr(old_logprob, f32), _ptr(advantages, f32), _ptr(values_new, f32),
+                                            _ptr(values_old, f32), _ptr(returns, f32), C.byref(params),
+                                            _ptr(out["losses"], f32), _ptr(out["dlogprob"], f32),
+                                            _ptr(out["dvalues"], f32), _stream())
+    _check("ppo_loss_from_logprob_static", rc)
     return out
 
 

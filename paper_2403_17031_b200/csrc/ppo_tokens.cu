@@ -385,3 +385,64 @@ extern "C" int ppo_loss_from_logprob(const float *new_logprob, const float *entr
     if (rc) return rc;
     return launch_loss_finalize(rows, p->vf_coef, losses, workspace, s);
 }
+
+// ---------------------------------------------------------------- allocation-free variant
+// Scratch for ppo_loss_from_logprob_static lives in this file-scope device array instead of a
+// caller-provided workspace: same layout as a workspace (header, per-token partials, row order).
+// Every GPU that loads the library carries these bytes until the process exits.
+namespace {
+constexpr size_t kStaticPartialBytes = ((size_t)PPO_STATIC_MAX_TOKENS * kPartialsPerToken * sizeof(float) + 255) & ~size_t(255);
+constexpr size_t kStaticOrderBytes = ((size_t)PPO_STATIC_MAX_TOKENS * sizeof(int32_t) + 255) & ~size_t(255);
+constexpr size_t kStaticScratchBytes = kHeaderBytes + kStaticPartialBytes + kStaticOrderBytes;
+}   // namespace
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// Device address of g_static_scratch on the current device. In host code the array's name is only a
+// handle for the runtime, not an address a kernel could use; cudaGetSymbolAddress translates it,
+// once per device, with that device current.
+static int static_scratch_address(void **out)
+{
+    static void *cached[64] = {nullptr};
+    int dev = 0;
+    PPO_RETURN_IF_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return PPO_ERR_UNSUPPORTED;
+    if (!cached[dev]) {
+        void *p = nullptr;
+        PPO_RETURN_IF_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
+        cached[dev] = p;
+    }
+    *out = cached[dev];
+    return PPO_OK;
+}
+
+extern "C" int ppo_loss_from_logprob_static(const float *new_logprob, const float *entropy, int32_t B, int32_t T,
+                                            const uint8_t *mask, const float *old_logprob, const float *advantages,
+                                            const float *values_new, const float *values_old, const float *returns,
+                                            const ppo_params *p, float *losses, float *dlogprob, float *dvalues,
+                                            void *stream)
+{
+    if (B <= 0 || T <= 0) return PPO_ERR_SHAPE;
+    if ((int64_t)B * T > PPO_STATIC_MAX_TOKENS) return PPO_ERR_UNSUPPORTED;   // beyond the built-in scratch
+    if (!new_logprob || !mask || !old_logprob || !advantages || !values_new || !values_old || !returns || !p ||
+        !losses || !dvalues)
+        return PPO_ERR_NULL;
+    if (!(p->cliprange >= 0.f) || !(p->cliprange_value >= 0.f) || !finite_f(p->vf_coef)) return PPO_ERR_PARAM;
+    void *scratch = nullptr;
+    int rc = static_scratch_address(&scratch);
+    if (rc) return rc;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const int64_t rows = (int64_t)B * T;
+    // the array keeps whatever the previous call left: the prologue rewrites the token count, the work
+    // counters and the row order, the token kernel rewrites every partial it later sums; the sticky
+    // status word is the one thing that has to be cleared by hand
+    PPO_RETURN_IF_CUDA(cudaMemsetAsync(&ws_header(scratch)->status, 0, sizeof(int), s));
+    rc = launch_loss_prepare(mask, rows, scratch, s);
+    if (rc) return rc;
+    loss_from_logprob_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, s>>>(
+        new_logprob, entropy, rows, mask, old_logprob, advantages, values_new, values_old, returns, p->cliprange,
+        p->cliprange_value, p->vf_coef, ws_header(scratch), ws_partials(scratch), dlogprob, dvalues);
+    rc = launch_status();
+    if (rc) return rc;
+    return launch_loss_finalize(rows, p->vf_coef, losses, scratch, s);
+}
