@@ -30,18 +30,21 @@ if ROOT not in sys.path:
 
 import torch  # noqa: E402
 
+# DRAM bytes (read + write) of one launch of the dominant kernel, from the committed ncu capture of the same
+# configuration (profiles/loss_fwd_bwd_row_engine_config1.md); None where no capture of the current kernel exists.
+NCU_TRAFFIC_BYTES = {1: 160.078e6 + 282.428e6}
 LAUNCHES_PER_STEP = 8   # truncate, 2x logprob, kl_rewards, gae, whiten, loss_prepare, row_engine (loss)
 
 
-def _peaks():
+def _peaks(key="hbm_gbs", fallback=6650.0):
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         try:
             d = json.load(open(path))
-            return float(d["hbm_gbs"]), "measured"
+            return float(d[key]), "measured"
         except Exception:
             pass
-    return 6650.0, "fallback"
+    return fallback, "fallback"
 
 
 class ClockSampler:
@@ -355,7 +358,8 @@ def run_ours(args, cfg):
                        "device_status": status},
             "roofline": {"bound": "hbm", "kernel": "loss_rows_kernel (ppo_loss_fwd_bwd)", "achieved": loss_gbs,
                          "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": loss_gbs / peak,
-                         "frac_of_8tbs": loss_gbs / 8000.0, "traffic": None,
+                         "frac_of_8tbs": loss_gbs / 8000.0, "traffic": NCU_TRAFFIC_BYTES.get(cfg.index),
+                         "algorithmic_bytes": loss_bytes,
                          "timing": "CUDA events around the C-ABI call (3 launches: count, rows, finalize)"},
             "clocks": clk.summary(),
             "e2e": e2e,
@@ -367,12 +371,121 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
+def run_lmhead(args, cfg):
+    """Config 4: fused LM head (policy and reference) + token-level steps + loss at log-prob level."""
+    rank, world, local = _dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    distributed = world > 1
+    if distributed:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2403_17031_b200 import binding, build
+    from paper_2403_17031_b200.synthetic import make_lmhead_batch
+    if rank == 0:
+        build.build()
+    if distributed:
+        dist.barrier()
+    binding.lib()
+    h = cfg.hyper
+    p = binding.params_from(h)
+    b = make_lmhead_batch(cfg, dev, M=args.lm_rows, seed=cfg.seed + 1000 * rank)
+    M, K = b["H"].shape
+    V = b["W"].shape[1]
+    B, T = b["responses"].shape
+    f32 = torch.float32
+    ws = binding.new_workspace(max(binding.lmhead_workspace_bytes(M, K, V), binding.workspace_bytes(B, T, V)), dev)
+    bt = lambda dt=f32: torch.empty((B, T), dtype=dt, device=dev)
+    o = {"ro": bt(torch.int32), "ei": torch.empty(B, dtype=torch.int32, device=dev),
+         "sl": torch.empty(B, dtype=torch.int32, device=dev), "mask": bt(torch.uint8),
+         "so": torch.empty(B, dtype=f32, device=dev), "lp": bt(), "ent": bt(), "lse": bt(), "rlp": bt(), "rent": bt(),
+         "kl": bt(), "rew": bt(), "adv": bt(), "ret": bt(), "aw": bt(), "st": torch.empty(3, dtype=f32, device=dev)}
+    loss_out = {"losses": torch.empty(8, dtype=f32, device=dev), "dlogprob": bt(), "dvalues": bt()}
+    tok = b["responses"].reshape(-1)
+
+    def step(old):
+        binding.truncate_and_score(b["responses"], b["scores"], p.eos_id, p.pad_id, p.no_eos_score,
+                                   out=(o["ro"], o["ei"], o["sl"], o["mask"], o["so"]))
+        binding.lmhead_logprob_entropy(b["H"], b["W"], tok, p.temperature, ws,
+                                       out=(o["lp"].view(-1), o["ent"].view(-1), o["lse"].view(-1)))
+        binding.lmhead_logprob_entropy(b["H"], b["W_ref"], tok, p.temperature, ws,
+                                       out=(o["rlp"].view(-1), o["rent"].view(-1), None))
+        binding.kl_rewards(o["lp"], o["rlp"], o["mask"], o["sl"], o["so"], p.kl_coef, out=(o["kl"], o["rew"]))
+        binding.gae(o["rew"], b["values"], o["sl"], p.gamma, p.lam, out=(o["adv"], o["ret"]))
+        binding.whiten(o["adv"], o["mask"], True, p.whiten_eps, workspace=ws, out=o["aw"], stats=o["st"])
+        binding.loss_from_logprob(o["lp"], o["ent"], o["mask"], o["lp"] if old is None else old, o["aw"],
+                                  b["values_new"], b["values"], o["ret"], p, ws, out=loss_out)
+    step(None)
+    old = (o["lp"] + b["old_logprob_noise"]).contiguous()
+    for _ in range(max(args.warmup, 3)):
+        step(old)
+    torch.cuda.synchronize()
+    K_steps = args.steps
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    lm_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K_steps)]
+    if distributed:
+        dist.barrier()
+    torch.cuda.synchronize()
+    with ClockSampler(local) as clk:
+        ev0.record()
+        for i in range(K_steps):
+            binding.truncate_and_score(b["responses"], b["scores"], p.eos_id, p.pad_id, p.no_eos_score,
+                                       out=(o["ro"], o["ei"], o["sl"], o["mask"], o["so"]))
+            lm_ev[i][0].record()
+            binding.lmhead_logprob_entropy(b["H"], b["W"], tok, p.temperature, ws,
+                                           out=(o["lp"].view(-1), o["ent"].view(-1), o["lse"].view(-1)))
+            lm_ev[i][1].record()
+            binding.lmhead_logprob_entropy(b["H"], b["W_ref"], tok, p.temperature, ws,
+                                           out=(o["rlp"].view(-1), o["rent"].view(-1), None))
+            binding.kl_rewards(o["lp"], o["rlp"], o["mask"], o["sl"], o["so"], p.kl_coef, out=(o["kl"], o["rew"]))
+            binding.gae(o["rew"], b["values"], o["sl"], p.gamma, p.lam, out=(o["adv"], o["ret"]))
+            binding.whiten(o["adv"], o["mask"], True, p.whiten_eps, workspace=ws, out=o["aw"], stats=o["st"])
+            binding.loss_from_logprob(o["lp"], o["ent"], o["mask"], old, o["aw"], b["values_new"], b["values"],
+                                      o["ret"], p, ws, out=loss_out)
+        ev1.record()
+        torch.cuda.synchronize()
+    total_ms = ev0.elapsed_time(ev1)
+    if distributed:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / K_steps
+    lm_ms = statistics.mean(a.elapsed_time(c) for a, c in lm_ev)
+    status = binding.last_device_status(ws)
+    flops = 2.0 * M * K * V
+    tf = flops / (lm_ms * 1e-3) / 1e12
+    # the kernel runs back to back for the whole timed region: compare with the sustained figure
+    peak, kind = _peaks("bf16_tflops_sustained", 1400.0)
+    burst, _ = _peaks("bf16_tflops", 1590.0)
+    if rank == 0:
+        line = {
+            "metric": "response tokens/s", "value": M * world / (ms_per_step * 1e-3), "unit": "tokens/s",
+            "n_gpus": world, "steps": K_steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "config4 %s" % cfg.name, "M_per_gpu": M, "K": K, "V": V,
+                       "l2": "inputs larger than L2 (H %.0f MB + 2 x W %.0f MB per step)" %
+                             (M * K * 2 / 1e6, K * V * 2 / 1e6),
+                       "lmhead_ms": lm_ms, "device_status": status},
+            "roofline": {"bound": "tensor", "kernel": "lmhead_kernel (ppo_lmhead_logprob_entropy)", "achieved": tf,
+                         "peak": peak, "peak_kind": kind + " (sustained)", "unit": "TFLOP/s", "frac": tf / peak,
+                         "frac_of_burst": tf / burst, "traffic": None,
+                         "timing": "CUDA events around the C-ABI call (GEMM kernel + finalize kernel)"},
+            "clocks": clk.summary(), "e2e": None, "cpu_baseline": None, "gpu_launches": 9 * K_steps,
+        }
+        print(json.dumps(line), flush=True)
+    if distributed:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--config", type=int, default=1, choices=[1, 2, 3])
+    ap.add_argument("--config", type=int, default=1, choices=[1, 2, 3, 4])
+    ap.add_argument("--lm-rows", type=int, default=None, help="config 4: rows of H (default 512*53)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -384,7 +497,9 @@ def main():
     from paper_2403_17031_b200.synthetic import CONFIGS
     cfg = CONFIGS[args.config]
     if args.impl == "reference":
-        run_reference(args, cfg)
+        run_reference(args, CONFIGS[1] if args.config == 4 else cfg)
+    elif args.config == 4:
+        run_lmhead(args, cfg)
     else:
         run_ours(args, cfg)
 
