@@ -301,14 +301,12 @@ def run_ours(args, cfg):
         host_res = {k: torch.empty_like(hp.out[k], device="cpu").pin_memory() for k in res_names}
         h2d = sum(v.numel() * v.element_size() for v in host.values())
         d2h = sum(v.numel() * v.element_size() for v in host_res.values())
+        host_io = binding.PPOStepIO.from_tensors({**host, **host_res}, cuda=False)
+        dev_io = hp.step_io(devbuf)
 
         def e2e_step():
-            for k, v in host.items():
-                devbuf[k].copy_(v, non_blocking=True)
-            hp.step(devbuf["policy_logits"], devbuf["ref_logits"], devbuf["responses"], devbuf["scores"],
-                    devbuf["values"], devbuf["values_new"], old_logprob=devbuf["old_logprob"])
-            for k, v in host_res.items():
-                v.copy_(hp.out[k], non_blocking=True)
+            # one C-ABI call: host->device copies, the whole path, device->host copies, stream sync
+            binding.step_host(host_io, dev_io, cfg.torch_dtype, B, T, V, hp.params)
         Ke = max(3, min(K, args.e2e_steps))
         for _ in range(2):
             e2e_step()
@@ -327,7 +325,7 @@ def run_ours(args, cfg):
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
             e_ms = float(t.item())
         e2e = {"value": tokens_per_step / (e_ms / Ke * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "steps": Ke}
+               "d2h_bytes_per_step": d2h, "steps": Ke, "call": "ppo_step_host (pinned host buffers)"}
         del host, devbuf
 
     # ---- CPU baseline: the oracle on a bounded sample, rank 0, N = 1 only

@@ -270,6 +270,44 @@ int ppo_lmhead_logprob_entropy(const void *H, const void *W, int64_t M, int64_t 
                                float *logprob, float *entropy, float *lse, void *workspace,
                                void *stream);
 
+/*
+ * The whole path in one call.  ppo_step_io names every buffer of one PPO iteration over a batch of
+ * B responses x T tokens; all pointers of one struct live in the same memory space.
+ *   inputs   policy_logits, ref_logits [B,T,V] (dtype); loss_logits [B,T,V] or NULL (= policy_logits);
+ *            responses [B,T] i32; scores [B]; values, values_new [B,T];
+ *            old_logprob [B,T] or NULL (= the log-probs this call computes: first PPO epoch, ratio 1)
+ *   outputs  responses_out, eos_index, seq_len, mask, scores_out (step 2); logprob, entropy,
+ *            ref_logprob (step 1); kl, rewards (step 3); advantages, returns (step 4);
+ *            advantages_whitened, whiten_stats[3] (step 5); losses[8], dlogits, dvalues and the
+ *            nullable new_logprob, new_entropy, dlogprob (step 6); workspace (device only)
+ *
+ * ppo_step: `io` is a host struct of DEVICE pointers; runs steps 2, 1 (policy), 1 (reference), 3, 4,
+ * 5, 6 in that order on `stream` without synchronising.  Errors are those of the individual calls.
+ *
+ * ppo_step_host: `host` is a host struct of HOST pointers (pinned memory makes the copies
+ * asynchronous), `dev` a host struct of DEVICE pointers used as staging and output buffers.  Copies
+ * every input host -> device, runs ppo_step on `dev`, copies back each output whose pointer in
+ * `host` is not NULL, and waits for the stream.  Inputs that are NULL in `host` (loss_logits,
+ * old_logprob) are treated as in ppo_step.
+ */
+typedef struct ppo_step_io {
+    const void *policy_logits, *ref_logits, *loss_logits;
+    const int32_t *responses;
+    const float *scores, *values, *values_new, *old_logprob;
+    int32_t *responses_out, *eos_index, *seq_len;
+    uint8_t *mask;
+    float *scores_out, *logprob, *entropy, *ref_logprob, *kl, *rewards, *advantages, *returns,
+        *advantages_whitened, *whiten_stats, *losses;
+    void *dlogits;
+    float *dvalues, *new_logprob, *new_entropy, *dlogprob;
+    void *workspace;
+} ppo_step_io;
+
+int ppo_step(const ppo_step_io *io /* host */, int dtype, int32_t B, int32_t T, int64_t V,
+             const ppo_params *p /* host */, void *stream);
+int ppo_step_host(const ppo_step_io *host /* host */, const ppo_step_io *dev /* host */, int dtype,
+                  int32_t B, int32_t T, int64_t V, const ppo_params *p /* host */, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -1,11 +1,11 @@
 """B200-native per-token PPO-for-RLHF hot path (arXiv 2403.17031): thin Python binding over the
 C-ABI CUDA library. Importing the package does not load the library; the first call does and
 fails loudly if it is missing (there is no CPU or PyTorch fallback)."""
-from .binding import (PPOParams, default_params, gae, kl_rewards, last_device_status, lib, lmhead_logprob_entropy,
+from .binding import (PPOParams, PPOStepIO, step, step_host, default_params, gae, kl_rewards, last_device_status, lib, lmhead_logprob_entropy,
                       lmhead_workspace_bytes, logprob_entropy, loss_from_logprob, loss_from_logprob_static, loss_fwd_bwd, new_workspace,
                       set_option, truncate_and_score, version, whiten, workspace_bytes, PPOError, LOSS_NAMES)
 
-__all__ = ["PPOParams", "default_params", "gae", "kl_rewards", "last_device_status", "lib",
+__all__ = ["PPOParams", "PPOStepIO", "step", "step_host", "default_params", "gae", "kl_rewards", "last_device_status", "lib",
            "lmhead_logprob_entropy", "lmhead_workspace_bytes", "logprob_entropy", "loss_from_logprob", "loss_from_logprob_static",
            "loss_fwd_bwd", "new_workspace", "set_option", "truncate_and_score", "version", "whiten",
            "workspace_bytes", "PPOError", "LOSS_NAMES"]

@@ -37,6 +37,29 @@ class PPOParams(C.Structure):
                 ("pad_id", C.c_int32)]
 
 
+class PPOStepIO(C.Structure):
+    """Mirror of ppo_step_io: every buffer of one iteration (all pointers in one memory space)."""
+    _in = ("policy_logits", "ref_logits", "loss_logits", "responses", "scores", "values", "values_new", "old_logprob")
+    _out = ("responses_out", "eos_index", "seq_len", "mask", "scores_out", "logprob", "entropy", "ref_logprob", "kl",
+            "rewards", "advantages", "returns", "advantages_whitened", "whiten_stats", "losses", "dlogits", "dvalues",
+            "new_logprob", "new_entropy", "dlogprob", "workspace")
+    _fields_ = [(n, C.c_void_p) for n in _in + _out]
+
+    @classmethod
+    def from_tensors(cls, tensors: dict, cuda: bool):
+        """Fill from {field: tensor or None}; checks that every tensor is contiguous and on the right side."""
+        io = cls()
+        for name in cls._in + cls._out:
+            t = tensors.get(name)
+            if t is None:
+                setattr(io, name, None)
+                continue
+            if t.is_cuda != cuda or not t.is_contiguous():
+                raise TypeError("%s must be a contiguous %s tensor" % (name, "CUDA" if cuda else "CPU"))
+            setattr(io, name, t.data_ptr())
+        return io
+
+
 _lib = None
 
 _SIGS = {
@@ -64,6 +87,10 @@ _SIGS = {
                               [C.POINTER(PPOParams)] + [C.c_void_p] * 5),
     "ppo_loss_from_logprob_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32] + [C.c_void_p] * 6 +
                                      [C.POINTER(PPOParams)] + [C.c_void_p] * 4),
+    "ppo_step": (C.c_int, [C.POINTER(PPOStepIO), C.c_int, C.c_int32, C.c_int32, C.c_int64, C.POINTER(PPOParams),
+                           C.c_void_p]),
+    "ppo_step_host": (C.c_int, [C.POINTER(PPOStepIO), C.POINTER(PPOStepIO), C.c_int, C.c_int32, C.c_int32, C.c_int64,
+                                C.POINTER(PPOParams), C.c_void_p]),
     "ppo_lmhead_logprob_entropy": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p,
                                              C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                              C.c_void_p]),
@@ -290,6 +317,18 @@ def loss_from_logprob(new_logprob, entropy, mask, old_logprob, advantages, value
                                      _ptr(workspace), _stream())
     _check("ppo_loss_from_logprob", rc)
     return out
+
+
+def step(io: PPOStepIO, dtype: torch.dtype, B: int, T: int, V: int, params: PPOParams) -> None:
+    """The whole path in one C call on device buffers (asynchronous on the current stream)."""
+    code = PPO_F32 if dtype == torch.float32 else PPO_BF16
+    _check("ppo_step", lib().ppo_step(C.byref(io), code, B, T, V, C.byref(params), _stream()))
+
+
+def step_host(host: PPOStepIO, dev: PPOStepIO, dtype: torch.dtype, B: int, T: int, V: int, params: PPOParams) -> None:
+    """Host buffers in, host buffers out: copies, the whole path, copies back, stream synchronised."""
+    code = PPO_F32 if dtype == torch.float32 else PPO_BF16
+    _check("ppo_step_host", lib().ppo_step_host(C.byref(host), C.byref(dev), code, B, T, V, C.byref(params), _stream()))
 
 
 STATIC_MAX_TOKENS = 32768

@@ -1,0 +1,113 @@
+// The whole path as one call (ppo_step) and its host-buffer variant (ppo_step_host): pure sequencing
+// of the per-step entry points plus the host<->device copies.
+#include "ppo_common.cuh"
+
+using namespace ppo;
+
+extern "C" int ppo_step(const ppo_step_io *io, int dtype, int32_t B, int32_t T, int64_t V, const ppo_params *p,
+                        void *stream)
+{
+    if (!io || !p) return PPO_ERR_NULL;
+    if (B <= 0 || T <= 0 || V <= 0) return PPO_ERR_SHAPE;
+    if (!io->responses_out || !io->eos_index || !io->seq_len || !io->mask || !io->scores_out || !io->logprob ||
+        !io->entropy || !io->ref_logprob || !io->kl || !io->rewards || !io->advantages || !io->returns ||
+        !io->advantages_whitened || !io->workspace)
+        return PPO_ERR_NULL;
+    const int64_t rows = (int64_t)B * T;
+    int rc = ppo_truncate_and_score(io->responses, B, T, p->eos_id, p->pad_id, io->scores, p->no_eos_score,
+                                    io->responses_out, io->eos_index, io->seq_len, io->mask, io->scores_out, stream);
+    if (rc) return rc;
+    rc = ppo_logprob_entropy(io->policy_logits, dtype, rows, V, V, io->responses, nullptr, p->temperature, io->logprob,
+                             io->entropy, nullptr, io->workspace, stream);
+    if (rc) return rc;
+    rc = ppo_logprob_entropy(io->ref_logits, dtype, rows, V, V, io->responses, nullptr, p->temperature,
+                             io->ref_logprob, nullptr, nullptr, io->workspace, stream);
+    if (rc) return rc;
+    rc = ppo_kl_rewards(io->logprob, io->ref_logprob, io->mask, io->seq_len, io->scores_out, B, T, p->kl_coef, io->kl,
+                        io->rewards, stream);
+    if (rc) return rc;
+    rc = ppo_gae(io->rewards, io->values, io->seq_len, B, T, p->gamma, p->lam, io->advantages, io->returns, stream);
+    if (rc) return rc;
+    rc = ppo_whiten(io->advantages, io->mask, rows, 1, p->whiten_eps, io->advantages_whitened, io->whiten_stats,
+                    io->workspace, stream);
+    if (rc) return rc;
+    return ppo_loss_fwd_bwd(io->loss_logits ? io->loss_logits : io->policy_logits, dtype, B, T, V, io->responses,
+                            io->mask, io->old_logprob ? io->old_logprob : io->logprob, io->advantages_whitened,
+                            io->values_new, io->values, io->returns, p, io->losses, io->dlogits, io->dvalues,
+                            io->new_logprob, io->new_entropy, io->dlogprob, io->workspace, stream);
+}
+
+namespace {
+
+int copy_in(void *dst, const void *src, size_t bytes, cudaStream_t s)
+{
+    if (!src) return PPO_OK;          // optional input not supplied
+    if (!dst) return PPO_ERR_NULL;    // supplied on the host but no staging buffer on the device
+    PPO_RETURN_IF_CUDA(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, s));
+    return PPO_OK;
+}
+
+int copy_out(void *dst, const void *src, size_t bytes, cudaStream_t s)
+{
+    if (!dst) return PPO_OK;          // the caller does not want this output on the host
+    if (!src) return PPO_ERR_NULL;
+    PPO_RETURN_IF_CUDA(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, s));
+    return PPO_OK;
+}
+
+}   // namespace
+
+#define PPO_TRY(expr)          \
+    do {                       \
+        int rc__ = (expr);     \
+        if (rc__) return rc__; \
+    } while (0)
+
+extern "C" int ppo_step_host(const ppo_step_io *host, const ppo_step_io *dev, int dtype, int32_t B, int32_t T,
+                             int64_t V, const ppo_params *p, void *stream)
+{
+    if (!host || !dev || !p) return PPO_ERR_NULL;
+    if (dtype != PPO_F32 && dtype != PPO_BF16) return PPO_ERR_DTYPE;
+    if (B <= 0 || T <= 0 || V <= 0) return PPO_ERR_SHAPE;
+    if (!host->policy_logits || !host->ref_logits || !host->responses || !host->scores || !host->values ||
+        !host->values_new)
+        return PPO_ERR_NULL;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const size_t bt = (size_t)B * (size_t)T, es = dtype == PPO_F32 ? 4 : 2;
+    const size_t logits_bytes = bt * (size_t)V * es;
+    // device staging buffers are written here, so drop the const the struct carries for inputs
+    PPO_TRY(copy_in(const_cast<void *>(dev->policy_logits), host->policy_logits, logits_bytes, s));
+    PPO_TRY(copy_in(const_cast<void *>(dev->ref_logits), host->ref_logits, logits_bytes, s));
+    PPO_TRY(copy_in(const_cast<void *>(dev->loss_logits), host->loss_logits, logits_bytes, s));
+    PPO_TRY(copy_in(const_cast<int32_t *>(dev->responses), host->responses, bt * 4, s));
+    PPO_TRY(copy_in(const_cast<float *>(dev->scores), host->scores, (size_t)B * 4, s));
+    PPO_TRY(copy_in(const_cast<float *>(dev->values), host->values, bt * 4, s));
+    PPO_TRY(copy_in(const_cast<float *>(dev->values_new), host->values_new, bt * 4, s));
+    PPO_TRY(copy_in(const_cast<float *>(dev->old_logprob), host->old_logprob, bt * 4, s));
+    ppo_step_io run = *dev;
+    if (!host->loss_logits) run.loss_logits = nullptr;
+    if (!host->old_logprob) run.old_logprob = nullptr;
+    PPO_TRY(ppo_step(&run, dtype, B, T, V, p, stream));
+    PPO_TRY(copy_out(host->responses_out, dev->responses_out, bt * 4, s));
+    PPO_TRY(copy_out(host->eos_index, dev->eos_index, (size_t)B * 4, s));
+    PPO_TRY(copy_out(host->seq_len, dev->seq_len, (size_t)B * 4, s));
+    PPO_TRY(copy_out(host->mask, dev->mask, bt, s));
+    PPO_TRY(copy_out(host->scores_out, dev->scores_out, (size_t)B * 4, s));
+    PPO_TRY(copy_out(host->logprob, dev->logprob, bt * 4, s));
+    PPO_TRY(copy_out(host->entropy, dev->entropy, bt * 4, s));
+    PPO_TRY(copy_out(host->ref_logprob, dev->ref_logprob, bt * 4, s));
+    PPO_TRY(copy_out(host->kl, dev->kl, bt * 4, s));
+    PPO_TRY(copy_out(host->rewards, dev->rewards, bt * 4, s));
+    PPO_TRY(copy_out(host->advantages, dev->advantages, bt * 4, s));
+    PPO_TRY(copy_out(host->returns, dev->returns, bt * 4, s));
+    PPO_TRY(copy_out(host->advantages_whitened, dev->advantages_whitened, bt * 4, s));
+    PPO_TRY(copy_out(host->whiten_stats, dev->whiten_stats, 3 * 4, s));
+    PPO_TRY(copy_out(host->losses, dev->losses, 8 * 4, s));
+    PPO_TRY(copy_out(host->dlogits, dev->dlogits, logits_bytes, s));
+    PPO_TRY(copy_out(host->dvalues, dev->dvalues, bt * 4, s));
+    PPO_TRY(copy_out(host->new_logprob, dev->new_logprob, bt * 4, s));
+    PPO_TRY(copy_out(host->new_entropy, dev->new_entropy, bt * 4, s));
+    PPO_TRY(copy_out(host->dlogprob, dev->dlogprob, bt * 4, s));
+    PPO_RETURN_IF_CUDA(cudaStreamSynchronize(s));
+    return PPO_OK;
+}

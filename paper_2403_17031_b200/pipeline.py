@@ -68,10 +68,28 @@ class PPOHotPath:
     def step(self, policy_logits, ref_logits, responses, scores, values, values_new, old_logprob=None,
              loss_logits=None, skip_masked_rows=False):
         """One pass of the whole path. old_logprob defaults to the rollout log-probs just computed
-        (first PPO epoch: ratio = 1); loss_logits defaults to policy_logits."""
-        o = self.rollout_stats(policy_logits, ref_logits, responses, scores, values, skip_masked_rows)
-        return self.loss(policy_logits if loss_logits is None else loss_logits, responses,
-                         o["logprob"] if old_logprob is None else old_logprob, values_new, values)
+        (first PPO epoch: ratio = 1); loss_logits defaults to policy_logits. One C call (ppo_step)
+        unless masked rows are to be skipped in step 1."""
+        if skip_masked_rows:
+            o = self.rollout_stats(policy_logits, ref_logits, responses, scores, values, True)
+            return self.loss(policy_logits if loss_logits is None else loss_logits, responses,
+                             o["logprob"] if old_logprob is None else old_logprob, values_new, values)
+        io = self.step_io({"policy_logits": policy_logits, "ref_logits": ref_logits, "loss_logits": loss_logits,
+                           "responses": responses, "scores": scores, "values": values, "values_new": values_new,
+                           "old_logprob": old_logprob})
+        _b.step(io, policy_logits.dtype, self.B, self.T, self.V, self.params)
+        return self.out
+
+    def step_io(self, inputs: dict, cuda: bool = True) -> "_b.PPOStepIO":
+        """ppo_step_io for this object's output buffers plus the given input tensors."""
+        o = self.out
+        t = dict(inputs)
+        t.update({k: o[k] for k in ("responses_out", "eos_index", "seq_len", "mask", "scores_out", "logprob", "entropy",
+                                    "ref_logprob", "kl", "rewards", "advantages", "returns", "advantages_whitened",
+                                    "whiten_stats", "losses", "dlogits", "dvalues", "new_logprob", "new_entropy",
+                                    "dlogprob")})
+        t["workspace"] = self.workspace
+        return _b.PPOStepIO.from_tensors(t, cuda)
 
     def device_status(self) -> int:
         return _b.last_device_status(self.workspace)

@@ -258,3 +258,41 @@ def _check_sampled(P, O, cfg, batch, n_rows, seed):
     # and the scalars against the oracle's log-prob-level arithmetic on the GPU's own new_logprob is
     # covered stage-wise at the smaller configs; here check the normaliser and finiteness
     assert torch.isfinite(o["losses"]).all()
+
+
+def test_single_call_step_and_host_step_match_the_separate_calls(P):
+    """ppo_step / ppo_step_host only sequence the per-step entry points: same bits as calling them one by one."""
+    from paper_2403_17031_b200 import binding
+    from paper_2403_17031_b200.pipeline import PPOHotPath
+    from paper_2403_17031_b200.synthetic import CONFIGS, make_batch
+    cfg = CONFIGS[0]
+    batch = make_batch(cfg, "cuda")
+    pp = _params(P, cfg.hyper)
+    names = ("mask", "seq_len", "logprob", "entropy", "ref_logprob", "kl", "rewards", "advantages", "returns",
+             "advantages_whitened", "losses", "dlogits", "dvalues", "new_logprob", "dlogprob")
+    a = PPOHotPath(cfg.B, cfg.T, cfg.V, torch.float32, pp)
+    o = a.rollout_stats(batch["policy_logits"], batch["ref_logits"], batch["responses"], batch["scores"], batch["values"])
+    old = (o["logprob"] + batch["old_logprob_noise"]).contiguous()
+    a.loss(batch["policy_logits"], batch["responses"], old, batch["values_new"], batch["values"])
+    b = PPOHotPath(cfg.B, cfg.T, cfg.V, torch.float32, pp)
+    b.step(batch["policy_logits"], batch["ref_logits"], batch["responses"], batch["scores"], batch["values"],
+           batch["values_new"], old_logprob=old)
+    torch.cuda.synchronize()
+    for k in names:
+        assert torch.equal(a.out[k], b.out[k]), k
+    # host buffers in, host buffers out
+    c = PPOHotPath(cfg.B, cfg.T, cfg.V, torch.float32, pp)
+    inp = {"policy_logits": batch["policy_logits"], "ref_logits": batch["ref_logits"], "responses": batch["responses"],
+           "scores": batch["scores"], "values": batch["values"], "values_new": batch["values_new"], "old_logprob": old}
+    host_in = {k: v.cpu().pin_memory() for k, v in inp.items()}
+    host_out = {k: torch.empty_like(c.out[k], device="cpu").pin_memory() for k in names}
+    stage = {k: torch.empty_like(v, device="cuda") for k, v in host_in.items()}
+    binding.step_host(binding.PPOStepIO.from_tensors({**host_in, **host_out}, cuda=False), c.step_io(stage),
+                      torch.float32, cfg.B, cfg.T, cfg.V, pp)
+    for k in names:
+        assert torch.equal(host_out[k], a.out[k].cpu()), k
+    # first-epoch default: no stored old log-probs -> ratio 1 -> nothing clipped
+    b.step(batch["policy_logits"], batch["ref_logits"], batch["responses"], batch["scores"], batch["values"],
+           batch["values_new"])
+    torch.cuda.synchronize()
+    assert float(b.out["losses"][3]) == 0.0 and float(b.out["losses"][4]) == 0.0
