@@ -141,6 +141,48 @@ __device__ __forceinline__ SoftmaxState block_merge(SoftmaxState st, float *red)
     return st;
 }
 
+__device__ __forceinline__ float warp_sum_f(float v)
+{
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    return v;
+}
+
+// Block-wide merge for the common case in which every thread kept the same reference m_common:
+// then merging is adding s and u. One barrier, which also ORs a "my reference differs" flag over
+// the block; if any thread moved its reference (overflow rescue) the general merge runs instead.
+// The result is valid in thread 0 only. `red` holds 96 floats and is free again after the
+// caller's next block-wide barrier.
+template <int THREADS>
+__device__ __forceinline__ SoftmaxState block_merge_common(SoftmaxState st, float m_common, float *red)
+{
+    constexpr int WARPS = THREADS / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (st.s == 0.f) st.m = m_common;                    // a thread without elements
+    const int differs = st.m != m_common;
+    const float s = warp_sum_f(st.s), u = warp_sum_f(st.u);
+    if (lane == 0) {
+        red[warp] = s;
+        red[32 + warp] = u;
+    }
+    if (__syncthreads_or(differs)) {
+        __syncthreads();                                 // everyone has left the fast path's use of red
+        return block_merge<THREADS>(st, red);
+    }
+    SoftmaxState r;
+    r.m = m_common;
+    r.s = 0.f;
+    r.u = 0.f;
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 0; w < WARPS; ++w) {
+            r.s += red[w];
+            r.u += red[32 + w];
+        }
+    }
+    return r;
+}
+
 __device__ __forceinline__ double warp_sum(double v)
 {
 #pragma unroll

@@ -13,43 +13,49 @@
 namespace ppo {
 
 // ---------------------------------------------------------------- step 1 kernel
+// One block per row (grid = rows). Kept free of loop-carried state so that it fits 32 registers:
+// eight blocks of 256 threads per SM.
 template <typename T, bool VECTOR, bool ENTROPY, int THREADS>
 __global__ void __launch_bounds__(THREADS)
-logprob_entropy_kernel(const T *__restrict__ logits, int64_t rows, int V, int64_t row_stride,
-                       const int32_t *__restrict__ tokens, const uint8_t *__restrict__ mask, float c,
-                       float *__restrict__ logprob, float *__restrict__ entropy, float *__restrict__ lse,
-                       int *status)
+logprob_entropy_kernel(const T *__restrict__ logits, int V, int64_t row_stride, const int32_t *__restrict__ tokens,
+                       const uint8_t *__restrict__ mask, float c, float *__restrict__ logprob,
+                       float *__restrict__ entropy, float *__restrict__ lse, int *status)
 {
     __shared__ float red[96];
-    for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
-        if (mask && !mask[row]) {
-            if (threadIdx.x == 0) {
-                logprob[row] = 0.f;
-                if (entropy) entropy[row] = 0.f;
-                if (lse) lse[row] = 0.f;
-            }
-            continue;
+    const int64_t row = blockIdx.x;
+    if (mask && !mask[row]) {
+        if (threadIdx.x == 0) {
+            logprob[row] = 0.f;
+            if (entropy) entropy[row] = 0.f;
+            if (lse) lse[row] = 0.f;
         }
-        const T *src = logits + row * row_stride;
+        return;
+    }
+    const T *src = logits + row * row_stride;
+    SoftmaxState st;
+    if (VECTOR) {
+        const float m_common = row_reference<T>(src, c);
+        st = row_statistics<T, true, false, ENTROPY, THREADS, 4>(src, V, c, nullptr, m_common);
+        st = block_merge_common<THREADS>(st, m_common, red);
+    } else {
+        st = row_statistics<T, false, false, ENTROPY, THREADS, 4>(src, V, c, nullptr, 0.f);
+        st = block_merge<THREADS>(st, red);
+    }
+    if (threadIdx.x == 0) {
         const int tok = tokens[row];
         const bool bad = tok < 0 || tok >= V;
-        float xtok = 0.f;
-        if (threadIdx.x == 0 && !bad) xtok = Pack<T>::load1(src + tok);
-        SoftmaxState st = row_statistics<T, VECTOR, false, ENTROPY, THREADS, 4>(src, V, c, nullptr);
-        st = block_merge<THREADS>(st, red);
-        if (threadIdx.x == 0) {
-            const float l2s = log2f(st.s);
-            float lp = (fmaf(xtok, c, -st.m) - l2s) * kLn2;
-            float H = (l2s - st.u / st.s) * kLn2;
-            float L = (st.m + l2s) * kLn2;
-            if (bad) {
-                lp = H = L = __int_as_float(0x7fc00000);
-                if (status) atomicOr(status, PPO_DEV_BAD_TOKEN);
-            }
-            logprob[row] = lp;
-            if (entropy) entropy[row] = H;
-            if (lse) lse[row] = L;
+        const float xtok = bad ? 0.f : Pack<T>::load1(src + tok);
+        const float l2s = log2f(st.s);
+        float lp = (fmaf(xtok, c, -st.m) - l2s) * kLn2;
+        float H = (l2s - st.u / st.s) * kLn2;
+        float L = (st.m + l2s) * kLn2;
+        if (bad) {
+            lp = H = L = __int_as_float(0x7fc00000);
+            if (status) atomicOr(status, PPO_DEV_BAD_TOKEN);
         }
+        logprob[row] = lp;
+        if (entropy) entropy[row] = H;
+        if (lse) lse[row] = L;
     }
 }
 
@@ -111,8 +117,15 @@ loss_rows_kernel(const LossArgs a)
             t_vo = a.values_old[row];
             t_ret = a.returns[row];
         }
-        SoftmaxState st = row_statistics<T, VECTOR, ROW_IN_SMEM, true, THREADS, 4>(src, V, a.c, row_stage);
-        st = block_merge<THREADS>(st, red);
+        SoftmaxState st;
+        if (VECTOR) {
+            const float m_common = row_reference<T>(src, a.c);
+            st = row_statistics<T, true, ROW_IN_SMEM, true, THREADS, 4>(src, V, a.c, row_stage, m_common);
+            st = block_merge_common<THREADS>(st, m_common, red);
+        } else {
+            st = row_statistics<T, false, ROW_IN_SMEM, true, THREADS, 4>(src, V, a.c, row_stage, 0.f);
+            st = block_merge<THREADS>(st, red);
+        }
         if (threadIdx.x == 0) {
             const float l2s = log2f(st.s);
             float lp = (fmaf(xtok, a.c, -st.m) - l2s) * kLn2;
@@ -194,10 +207,10 @@ static int launch_logprob(const void *logits, int64_t rows, int V, int64_t row_s
 {
     constexpr int THREADS = 256;
     const bool vec = aligned16(logits) && (row_stride * sizeof(T)) % 16 == 0 && V % Pack<T>::N == 0;
-    const unsigned grid = (unsigned)(rows < (int64_t)1 << 30 ? rows : (int64_t)1 << 30);
+    const unsigned grid = (unsigned)rows;   // rows < 2^31 is checked by the caller
     const T *lg = reinterpret_cast<const T *>(logits);
-#define PPO_LAUNCH_LP(VEC, ENT)                                                                             \
-    logprob_entropy_kernel<T, VEC, ENT, THREADS><<<grid, THREADS, 0, s>>>(lg, rows, V, row_stride, tokens, mask, c, \
+#define PPO_LAUNCH_LP(VEC, ENT)                                                                       \
+    logprob_entropy_kernel<T, VEC, ENT, THREADS><<<grid, THREADS, 0, s>>>(lg, V, row_stride, tokens, mask, c, \
                                                                           logprob, entropy, lse, status)
     if (vec) {
         if (entropy) PPO_LAUNCH_LP(true, true); else PPO_LAUNCH_LP(true, false);
@@ -255,7 +268,8 @@ extern "C" int ppo_logprob_entropy(const void *logits, int dtype, int64_t rows, 
                                    float *logprob, float *entropy, float *lse, void *workspace, void *stream)
 {
     if (dtype != PPO_F32 && dtype != PPO_BF16) return PPO_ERR_DTYPE;
-    if (rows < 0 || V <= 0 || V >= ((int64_t)1 << 31) || row_stride < V) return PPO_ERR_SHAPE;
+    if (rows < 0 || rows >= ((int64_t)1 << 31) || V <= 0 || V >= ((int64_t)1 << 31) || row_stride < V)
+        return PPO_ERR_SHAPE;
     if (!(temperature > 0.f) || !finite_f(temperature)) return PPO_ERR_PARAM;
     if (rows == 0) return PPO_OK;
     if (!logits || !tokens || !logprob) return PPO_ERR_NULL;

@@ -111,11 +111,14 @@ struct FixedAcc {
     __device__ __forceinline__ void init() { s0 = u0 = s1 = u1 = 0.f; }
 };
 
-template <typename T, bool ENTROPY>
+// CLAMP = false is the fast path: a -inf logit then gives 0 * -inf = NaN in the entropy sum, which
+// the caller detects after the fact and repairs by redoing the packs with CLAMP = true.
+template <typename T, bool ENTROPY, bool CLAMP = false>
 __device__ __forceinline__ void accumulate_fixed(const uint4 &v, float c, float nm, FixedAcc &a)
 {
     float x[Pack<T>::N];
-    Pack<T>::unpack_clamped(v, x);
+    if (CLAMP) Pack<T>::unpack_clamped(v, x);
+    else Pack<T>::unpack_raw(v, x);
 #pragma unroll
     for (int k = 0; k < Pack<T>::N; k += 2) {
         const float t0 = fmaf(x[k], c, nm), t1 = fmaf(x[k + 1], c, nm);
@@ -133,12 +136,24 @@ __device__ __forceinline__ void accumulate_fixed(const uint4 &v, float c, float 
 // otherwise element by element. STAGE: also park the raw packs / elements in shared memory.
 //
 // Fast path: the softmax sums do not need the exact maximum as reference, only one that keeps
-// 2^(y - ref) inside fp32 range. Each thread takes the maximum of its first pack as a fixed
-// reference and never moves it, which removes the per-pack maximum, compare and rescale from the
-// inner loop. If a later element exceeds the reference by more than ~2^127 the sum overflows to
-// inf; that is detected after the loop and the thread redoes its packs with the online update.
+// 2^(y - ref) inside fp32 range. Every thread of the row uses the same fixed reference m_common
+// (see row_reference) and never moves it, which removes the per-pack maximum, compare and rescale
+// from the inner loop and lets the block merge its threads by plain addition. If a later element exceeds the reference by more than ~2^127 the sum overflows to
+// inf, and a -inf logit turns the entropy sum into NaN (0 * -inf); both are detected after the loop
+// and the thread redoes its packs with the clamped online update.
+// Common reference of a row for the vector path: the maximum of the row's first pack (every thread
+// reads the same 16 bytes), in base-2 units.
+template <typename T>
+__device__ __forceinline__ float row_reference(const T *__restrict__ src, float c)
+{
+    float x[Pack<T>::N], xmax;
+    Pack<T>::unpack(*reinterpret_cast<const uint4 *>(src), x, xmax);
+    return safe_reference(xmax, c);
+}
+
 template <typename T, bool VECTOR, bool STAGE, bool ENTROPY, int THREADS, int UNROLL>
-__device__ __forceinline__ SoftmaxState row_statistics(const T *__restrict__ src, int V, float c, void *stage)
+__device__ __forceinline__ SoftmaxState row_statistics(const T *__restrict__ src, int V, float c, void *stage,
+                                                       float m_common)
 {
     SoftmaxState st;
     st.init();
@@ -156,11 +171,7 @@ __device__ __forceinline__ SoftmaxState row_statistics(const T *__restrict__ src
 #pragma unroll
             for (int k = 0; k < UNROLL; ++k)
                 if (i + k * THREADS < nvec) v[k] = ld_stream(src4 + i + k * THREADS);
-            {
-                float x[N], xmax;
-                Pack<T>::unpack(v[0], x, xmax);
-                st.m = safe_reference(xmax, c);
-            }
+            st.m = m_common;
             const float nm = -st.m;
 #pragma unroll
             for (int k = 0; k < UNROLL; ++k)

@@ -34,7 +34,7 @@ constexpr uint32_t kWaitTries = 1u << 20;           // x ~1 us per try
 struct EngineSmem {
     unsigned long long full[kMaxChunks];
     unsigned long long empty[kMaxChunks];
-    float red[96];
+    float red[2][96];      // by row parity: a row's sums are read while the next row's are written
     float bc[4];
     int next_item;
     int is_last;
@@ -126,17 +126,58 @@ __device__ __forceinline__ SoftmaxState consumer_merge(SoftmaxState st, float *r
     return st;
 }
 
-// per-thread statistics with a fixed reference that is only moved when a chunk overflows
+// Merge for the common case in which no consumer thread moved its reference: plain addition and one
+// named barrier, which also ORs the "my reference differs" flags. Result valid in consumer thread 0.
+// `red` (96 floats) must not be rewritten before the caller's next consumer-wide barrier.
+__device__ __forceinline__ SoftmaxState consumer_merge_common(SoftmaxState st, float m_common, float *red, int ct)
+{
+    const int lane = ct & 31, warp = ct >> 5;
+    if (st.s == 0.f) st.m = m_common;
+    const uint32_t differs = st.m != m_common;
+    const float s = warp_sum_f(st.s), u = warp_sum_f(st.u);
+    if (lane == 0) {
+        red[warp] = s;
+        red[32 + warp] = u;
+    }
+    uint32_t any;
+    asm volatile(
+        "{\n"
+        ".reg .pred p, q;\n"
+        "setp.ne.u32 q, %1, 0;\n"
+        "bar.red.or.pred p, 1, %2, q;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(any)
+        : "r"(differs), "n"(kConsumers)
+        : "memory");
+    if (any) {
+        consumer_sync();
+        return consumer_merge(st, red, ct);
+    }
+    SoftmaxState r;
+    r.m = m_common;
+    r.s = 0.f;
+    r.u = 0.f;
+    if (ct == 0) {
+#pragma unroll
+        for (int w = 0; w < kConsumerWarps; ++w) {
+            r.s += red[w];
+            r.u += red[32 + w];
+        }
+    }
+    return r;
+}
+
+// per-thread statistics with a fixed reference (the same for all threads of the row: the maximum of
+// the row's first pack) that is only moved when a chunk overflows
 template <typename T, bool ENTROPY>
 struct ThreadStats {
     float m;          // reference, base-2 units
     FixedAcc acc;
-    bool have_ref;
-    __device__ __forceinline__ void init()
+    __device__ __forceinline__ void init(float m_common)
     {
-        m = kNegBig;
+        m = m_common;
         acc.init();
-        have_ref = false;
     }
     __device__ __forceinline__ void rebase(float nm)
     {
@@ -151,25 +192,19 @@ struct ThreadStats {
     __device__ __forceinline__ void chunk(const uint4 &v0, bool h0, const uint4 &v1, bool h1, float c)
     {
         if (!h0) return;                      // h1 implies h0
-        if (!have_ref) {
-            float x[Pack<T>::N], xm0, xm1 = kNegBig;
-            Pack<T>::unpack(v0, x, xm0);
-            if (h1) Pack<T>::unpack(v1, x, xm1);
-            m = safe_reference(fmaxf(xm0, xm1), c);
-            have_ref = true;
-        }
         const FixedAcc save = acc;
         accumulate_fixed<T, ENTROPY>(v0, c, -m, acc);
         if (h1) accumulate_fixed<T, ENTROPY>(v1, c, -m, acc);
-        if (!(acc.s0 + acc.s1 < 1.0e35f)) {   // overflow (or NaN): move the reference up and redo the chunk
+        if (!(acc.s0 + acc.s1 < 1.0e35f) || !(fabsf(acc.u0 + acc.u1) < 1.0e35f)) {
+            // overflow, or -inf/NaN logits: move the reference up and redo the chunk with clamped values
             acc = save;
             float x[Pack<T>::N], xm0, xm1 = kNegBig;
             Pack<T>::unpack(v0, x, xm0);
             if (h1) Pack<T>::unpack(v1, x, xm1);
             const float nm = safe_reference(fmaxf(xm0, xm1), c);
             if (nm > m) rebase(nm);
-            accumulate_fixed<T, ENTROPY>(v0, c, -m, acc);
-            if (h1) accumulate_fixed<T, ENTROPY>(v1, c, -m, acc);
+            accumulate_fixed<T, ENTROPY, true>(v0, c, -m, acc);
+            if (h1) accumulate_fixed<T, ENTROPY, true>(v1, c, -m, acc);
         }
     }
     __device__ __forceinline__ SoftmaxState state() const
@@ -292,26 +327,29 @@ row_engine_kernel(const EngineArgs a)
     if (threadIdx.x >= kConsumers) {
         // ------------------------------------------------------------ producer
         if (threadIdx.x == kConsumers) {
-        const uint64_t policy = policy_evict_first();
-        uint32_t k = 0;
-        for (int64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
-            int64_t row;
-            if (MODE == 0) {
-                row = item;
-                if (a.mask && !a.mask[row]) continue;
-            } else {
-                row = a.order[item];
+            const uint64_t policy = policy_evict_first();
+            uint32_t k = 0;
+            // the row index of the next item is fetched one row ahead (it is a dependent load)
+            int64_t row_next = (MODE == 1 && (int64_t)blockIdx.x < n_items) ? a.order[blockIdx.x] : -1;
+            for (int64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+                int64_t row;
+                if (MODE == 0) {
+                    row = item;
+                    if (a.mask && !a.mask[row]) continue;
+                } else {
+                    row = row_next;
+                    if (item + gridDim.x < n_items) row_next = a.order[item + gridDim.x];
+                }
+                const unsigned char *src = reinterpret_cast<const unsigned char *>(logits + row * stride);
+                for (int c = 0; c < nch; ++c) {
+                    if (k > 0) mbar_wait(&sm.empty[c], (k - 1) & 1, status);
+                    const int packs = min(kChunkPacks, nvec - c * kChunkPacks);
+                    mbar_expect_tx(&sm.full[c], (uint32_t)packs * 16u);
+                    bulk_load(smem_raw + (size_t)c * kChunkBytes, src + (size_t)c * kChunkBytes, (uint32_t)packs * 16u,
+                              &sm.full[c], policy);
+                }
+                ++k;
             }
-            const unsigned char *src = reinterpret_cast<const unsigned char *>(logits + row * stride);
-            for (int c = 0; c < nch; ++c) {
-                if (k > 0) mbar_wait(&sm.empty[c], (k - 1) & 1, status);
-                const int packs = min(kChunkPacks, nvec - c * kChunkPacks);
-                mbar_expect_tx(&sm.full[c], (uint32_t)packs * 16u);
-                bulk_load(smem_raw + (size_t)c * kChunkBytes, src + (size_t)c * kChunkBytes, (uint32_t)packs * 16u,
-                          &sm.full[c], policy);
-            }
-            ++k;
-        }
         }
         if (MODE == 1) {
             __syncwarp();
@@ -323,55 +361,95 @@ row_engine_kernel(const EngineArgs a)
     // ---------------------------------------------------------------- consumers
     const int ct = threadIdx.x;
     const uint4 *buf = reinterpret_cast<const uint4 *>(smem_raw);
+    const T *buf_elems = reinterpret_cast<const T *>(smem_raw);
     const double n_tok = MODE == 1 ? (double)a.hdr->n_tokens : 0.0;
+    const int64_t G = gridDim.x;
     uint32_t k = 0;
-    for (int64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
-        int64_t row;
-        if (MODE == 0) {
-            row = item;
-            if (a.mask && !a.mask[row]) {
-                if (ct == 0) {
-                    a.logprob[row] = 0.f;
-                    if (a.entropy) a.entropy[row] = 0.f;
-                    if (a.lse) a.lse[row] = 0.f;
-                }
-                continue;
-            }
+    // Per-row scalars come through dependent loads (row index -> token id -> ...). They are fetched
+    // ahead of time so that no warp starts a row late: row index two rows ahead, token id and the
+    // per-token inputs one row ahead. The token's logit itself is read from the resident row.
+    int64_t row_c = -1, row_n = -1;
+    int tok_c = -1, tok_n = -1;
+    float in_c[5] = {0.f, 0.f, 0.f, 0.f, 0.f}, in_n[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
+    {
+        const int64_t item0 = blockIdx.x;
+        if (MODE == 1) {
+            if (item0 < n_items) row_c = a.order[item0];
+            if (item0 + G < n_items) row_n = a.order[item0 + G];
         } else {
-            row = a.order[item];
+            if (item0 < n_items) row_c = item0;
+            if (item0 + G < n_items) row_n = item0 + G;
         }
-        const T *src = logits + row * stride;
-        const int tok = a.tokens[row];
-        const bool bad = tok < 0 || tok >= V;
-        float xtok = 0.f, t_old = 0.f, t_adv = 0.f, t_vn = 0.f, t_vo = 0.f, t_ret = 0.f;
-        if (ct == 0) {   // per-token scalars: fetched now, used after the row reduction
-            if (!bad) xtok = Pack<T>::load1(src + tok);
-            if (MODE == 1) {
-                t_old = a.loss.old_logprob[row];
-                t_adv = a.loss.advantages[row];
-                t_vn = a.loss.values_new[row];
-                t_vo = a.loss.values_old[row];
-                t_ret = a.loss.returns[row];
+        if (row_c >= 0) {
+            tok_c = a.tokens[row_c];
+            if (MODE == 1 && ct == 0) {
+                in_c[0] = a.loss.old_logprob[row_c];
+                in_c[1] = a.loss.advantages[row_c];
+                in_c[2] = a.loss.values_new[row_c];
+                in_c[3] = a.loss.values_old[row_c];
+                in_c[4] = a.loss.returns[row_c];
             }
         }
+    }
+    for (int64_t item = blockIdx.x; item < n_items; item += G) {
+        // prefetch for the rows that follow
+        int64_t row_nn = -1;
+        if (item + 2 * G < n_items) row_nn = MODE == 1 ? (int64_t)a.order[item + 2 * G] : item + 2 * G;
+        if (row_n >= 0) {
+            tok_n = a.tokens[row_n];
+            if (MODE == 1 && ct == 0) {
+                in_n[0] = a.loss.old_logprob[row_n];
+                in_n[1] = a.loss.advantages[row_n];
+                in_n[2] = a.loss.values_new[row_n];
+                in_n[3] = a.loss.values_old[row_n];
+                in_n[4] = a.loss.returns[row_n];
+            }
+        }
+        const int64_t row = row_c;
+        const int tok = tok_c;
+        const float t_old = in_c[0], t_adv = in_c[1], t_vn = in_c[2], t_vo = in_c[3], t_ret = in_c[4];
+        row_c = row_n;
+        row_n = row_nn;
+        tok_c = tok_n;
+#pragma unroll
+        for (int q = 0; q < 5; ++q) in_c[q] = in_n[q];
+
+        if (MODE == 0 && a.mask && !a.mask[row]) {
+            if (ct == 0) {
+                a.logprob[row] = 0.f;
+                if (a.entropy) a.entropy[row] = 0.f;
+                if (a.lse) a.lse[row] = 0.f;
+            }
+            continue;
+        }
+        const bool bad = tok < 0 || tok >= V;
+        const int tok_chunk = bad ? -1 : (tok / N) / kChunkPacks;
+        float xtok = 0.f;
         // ---- pass 1: statistics, chunk by chunk as the bytes land
         ThreadStats<T, ENTROPY> ts;
-        ts.init();
         const uint32_t parity = k & 1;
+        float m_common = 0.f;
         for (int c = 0; c < nch; ++c) {
             mbar_wait(&sm.full[c], parity, status);
+            if (c == 0) {   // every thread reads the row's first pack: one reference for the whole row
+                float x[N], xmax;
+                Pack<T>::unpack(buf[0], x, xmax);
+                m_common = safe_reference(xmax, a.c);
+                ts.init(m_common);
+            }
             const int i0 = c * kChunkPacks + ct, i1 = i0 + kConsumers;
             const bool h0 = i0 < nvec, h1 = i1 < nvec;
             uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
             if (h0) v0 = buf[i0];
             if (h1) v1 = buf[i1];
+            if (ct == 0 && c == tok_chunk) xtok = Pack<T>::load1(buf_elems + tok);
             ts.chunk(v0, h0, v1, h1, a.c);
             if (MODE == 0) {
                 __syncwarp();
                 if ((ct & 31) == 0) mbar_arrive(&sm.empty[c]);
             }
         }
-        SoftmaxState st = consumer_merge(ts.state(), sm.red, ct);
+        const SoftmaxState st = consumer_merge_common(ts.state(), m_common, sm.red[parity], ct);   // thread 0 only
         const float l2s = log2f(st.s);
         if (MODE == 0) {
             if (ct == 0) {
@@ -409,10 +487,12 @@ row_engine_kernel(const EngineArgs a)
             consumer_sync();
             const float Y = sm.bc[0], gs = sm.bc[1];
             // ---- pass 2: gradient row, chunk by chunk; each chunk is handed back to the producer
-            uint4 *dst4 = reinterpret_cast<uint4 *>(reinterpret_cast<T *>(la.dlogits) + row * (int64_t)V);
+            T *dst = reinterpret_cast<T *>(la.dlogits) + row * (int64_t)V;
+            uint4 *dst4 = reinterpret_cast<uint4 *>(dst);
             // -gs * 2^(y - Y) = -+ 2^(y - Y + log2|gs|): the scale rides in the exponent
             const float off = log2f(fabsf(gs)) - Y;
             const bool zero = gs == 0.f, neg = gs > 0.f;
+            const bool fix_owner = !zero && !bad && ct == (tok / N) % kConsumers;
             for (int c = 0; c < nch; ++c) {
                 const int i0 = c * kChunkPacks + ct;
 #pragma unroll
@@ -429,13 +509,13 @@ row_engine_kernel(const EngineArgs a)
                         st_stream(dst4 + i, Pack<T>::pack(d));
                     }
                 }
+                // the thread that wrote the pack holding the sampled token adds the one-hot term
+                if (fix_owner && c == tok_chunk) {
+                    const float e = ex2(fmaf(Pack<T>::load1(buf_elems + tok), a.c, off));
+                    Pack<T>::store1(dst + tok, gs + (neg ? -e : e));
+                }
                 __syncwarp();
                 if ((ct & 31) == 0) mbar_arrive(&sm.empty[c]);
-            }
-            // the thread that wrote the pack holding the sampled token adds the one-hot term
-            if (!zero && !bad && ct == (tok / N) % kConsumers) {
-                const float e = ex2(fmaf(Pack<T>::load1(src + tok), a.c, off));
-                Pack<T>::store1(reinterpret_cast<T *>(dst4) + tok, gs + (neg ? -e : e));
             }
         }
         ++k;
