@@ -282,6 +282,19 @@ __device__ __forceinline__ void reduce_loss_partials(const float *partials, int6
 }
 
 // launchers shared between translation units
+int launch_step_prologue(const int32_t *responses, int B, int T, const ppo_params *p, const float *scores,
+                         int32_t *responses_out, int32_t *eos_index, int32_t *seq_len, uint8_t *mask, float *scores_out,
+                         void *workspace, cudaStream_t s);
+int launch_advantages(const float *logprob, const float *ref_logprob, const int32_t *seq_len, const float *scores,
+                      const float *values, const uint8_t *mask, int B, int T, const ppo_params *p, float *kl,
+                      float *rewards, float *advantages, float *returns, float *whitened, float *stats3, void *workspace,
+                      cudaStream_t s);
+// ppo_loss_fwd_bwd without its prologue launch (the caller has already run the prologue on this mask)
+int loss_fwd_bwd_prepared(const void *logits, int dtype, int32_t B, int32_t T, int64_t V, const int32_t *tokens,
+                          const uint8_t *mask, const float *old_logprob, const float *advantages,
+                          const float *values_new, const float *values_old, const float *returns, const ppo_params *p,
+                          float *losses, void *dlogits, float *dvalues, float *new_logprob, float *entropy,
+                          float *dlogprob, void *workspace, void *stream, bool prepared);
 int launch_loss_prepare(const uint8_t *mask, int64_t rows, void *workspace, cudaStream_t s);
 int launch_loss_finalize(int64_t rows, float vf_coef, float *losses, void *workspace, cudaStream_t s);
 

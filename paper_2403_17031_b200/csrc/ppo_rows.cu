@@ -297,6 +297,17 @@ extern "C" int ppo_loss_fwd_bwd(const void *logits, int dtype, int32_t B, int32_
                                 float *dvalues, float *new_logprob, float *entropy, float *dlogprob,
                                 void *workspace, void *stream)
 {
+    return loss_fwd_bwd_prepared(logits, dtype, B, T, V, tokens, mask, old_logprob, advantages, values_new, values_old,
+                                 returns, p, losses, dlogits, dvalues, new_logprob, entropy, dlogprob, workspace, stream,
+                                 false);
+}
+
+int ppo::loss_fwd_bwd_prepared(const void *logits, int dtype, int32_t B, int32_t T, int64_t V, const int32_t *tokens,
+                               const uint8_t *mask, const float *old_logprob, const float *advantages,
+                               const float *values_new, const float *values_old, const float *returns,
+                               const ppo_params *p, float *losses, void *dlogits, float *dvalues, float *new_logprob,
+                               float *entropy, float *dlogprob, void *workspace, void *stream, bool prepared)
+{
     if (dtype != PPO_F32 && dtype != PPO_BF16) return PPO_ERR_DTYPE;
     if (B <= 0 || T <= 0 || V <= 0 || V >= ((int64_t)1 << 31) || (int64_t)B * T >= ((int64_t)1 << 31))
         return PPO_ERR_SHAPE;
@@ -313,7 +324,7 @@ extern "C" int ppo_loss_fwd_bwd(const void *logits, int dtype, int32_t B, int32_
     if (dlogits == logits) return PPO_ERR_PARAM;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     const int64_t rows = (int64_t)B * T;
-    int rc = launch_loss_prepare(mask, rows, workspace, s);
+    int rc = prepared ? PPO_OK : launch_loss_prepare(mask, rows, workspace, s);
     if (rc) return rc;
     LossArgs a;
     a.logits = logits;

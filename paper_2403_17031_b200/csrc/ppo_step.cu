@@ -1,5 +1,5 @@
-// The whole path as one call (ppo_step) and its host-buffer variant (ppo_step_host): pure sequencing
-// of the per-step entry points plus the host<->device copies.
+// The whole path as one call (ppo_step) and its host-buffer variant (ppo_step_host): sequencing of the
+// steps (the token-level ones fused into two launches) plus the host<->device copies.
 #include "ppo_common.cuh"
 
 using namespace ppo;
@@ -13,9 +13,20 @@ extern "C" int ppo_step(const ppo_step_io *io, int dtype, int32_t B, int32_t T, 
         !io->entropy || !io->ref_logprob || !io->kl || !io->rewards || !io->advantages || !io->returns ||
         !io->advantages_whitened || !io->workspace)
         return PPO_ERR_NULL;
+    if (!io->responses || !io->scores || !io->values || !io->policy_logits || !io->ref_logits || !io->losses ||
+        !io->dvalues)
+        return PPO_ERR_NULL;
+    if (p->eos_id == p->pad_id || !finite_f(p->kl_coef) || !finite_f(p->gamma) || !finite_f(p->lam) ||
+        !(p->whiten_eps >= 0.f))
+        return PPO_ERR_PARAM;
+    if (reinterpret_cast<uintptr_t>(io->workspace) % 256) return PPO_ERR_ALIGN;
     const int64_t rows = (int64_t)B * T;
-    int rc = ppo_truncate_and_score(io->responses, B, T, p->eos_id, p->pad_id, io->scores, p->no_eos_score,
-                                    io->responses_out, io->eos_index, io->seq_len, io->mask, io->scores_out, stream);
+    if (rows >= ((int64_t)1 << 31)) return PPO_ERR_SHAPE;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    // five launches: [EOS trick + loss prologue] -> log-probs (policy) -> log-probs (reference) ->
+    // [KL rewards + GAE + whitening] -> loss forward/backward
+    int rc = launch_step_prologue(io->responses, B, T, p, io->scores, io->responses_out, io->eos_index, io->seq_len,
+                                  io->mask, io->scores_out, io->workspace, s);
     if (rc) return rc;
     rc = ppo_logprob_entropy(io->policy_logits, dtype, rows, V, V, io->responses, nullptr, p->temperature, io->logprob,
                              io->entropy, nullptr, io->workspace, stream);
@@ -23,18 +34,14 @@ extern "C" int ppo_step(const ppo_step_io *io, int dtype, int32_t B, int32_t T, 
     rc = ppo_logprob_entropy(io->ref_logits, dtype, rows, V, V, io->responses, nullptr, p->temperature,
                              io->ref_logprob, nullptr, nullptr, io->workspace, stream);
     if (rc) return rc;
-    rc = ppo_kl_rewards(io->logprob, io->ref_logprob, io->mask, io->seq_len, io->scores_out, B, T, p->kl_coef, io->kl,
-                        io->rewards, stream);
+    rc = launch_advantages(io->logprob, io->ref_logprob, io->seq_len, io->scores_out, io->values, io->mask, B, T, p, io->kl,
+                           io->rewards, io->advantages, io->returns, io->advantages_whitened, io->whiten_stats,
+                           io->workspace, s);
     if (rc) return rc;
-    rc = ppo_gae(io->rewards, io->values, io->seq_len, B, T, p->gamma, p->lam, io->advantages, io->returns, stream);
-    if (rc) return rc;
-    rc = ppo_whiten(io->advantages, io->mask, rows, 1, p->whiten_eps, io->advantages_whitened, io->whiten_stats,
-                    io->workspace, stream);
-    if (rc) return rc;
-    return ppo_loss_fwd_bwd(io->loss_logits ? io->loss_logits : io->policy_logits, dtype, B, T, V, io->responses,
-                            io->mask, io->old_logprob ? io->old_logprob : io->logprob, io->advantages_whitened,
-                            io->values_new, io->values, io->returns, p, io->losses, io->dlogits, io->dvalues,
-                            io->new_logprob, io->new_entropy, io->dlogprob, io->workspace, stream);
+    return loss_fwd_bwd_prepared(io->loss_logits ? io->loss_logits : io->policy_logits, dtype, B, T, V, io->responses,
+                                 io->mask, io->old_logprob ? io->old_logprob : io->logprob, io->advantages_whitened,
+                                 io->values_new, io->values, io->returns, p, io->losses, io->dlogits, io->dvalues,
+                                 io->new_logprob, io->new_entropy, io->dlogprob, io->workspace, stream, true);
 }
 
 namespace {

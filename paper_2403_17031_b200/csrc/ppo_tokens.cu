@@ -10,15 +10,12 @@ int option_value(int key) { return (key >= 0 && key < 8) ? g_options[key] : 0; }
 
 // ---------------------------------------------------------------- step 2: EOS trick
 // One warp per response: lanes stride over t, a warp-wide min finds the first EOS.
-__global__ void __launch_bounds__(128)
-truncate_kernel(const int32_t *responses, int B, int T, int eos_id, int pad_id,
-                const float *__restrict__ scores, float no_eos_score, int32_t *responses_out,
-                int32_t *__restrict__ eos_index, int32_t *__restrict__ seq_len, uint8_t *__restrict__ mask,
-                float *__restrict__ scores_out)
+__device__ __forceinline__ void truncate_sequence(const int32_t *responses, int b, int T, int eos_id, int pad_id,
+                                                  const float *__restrict__ scores, float no_eos_score,
+                                                  int32_t *responses_out, int32_t *__restrict__ eos_index,
+                                                  int32_t *__restrict__ seq_len, uint8_t *__restrict__ mask,
+                                                  float *__restrict__ scores_out, int lane)
 {
-    const int b = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
-    const int lane = threadIdx.x & 31;
-    if (b >= B) return;
     const int32_t *r = responses + (int64_t)b * T;
     int first = T;
     for (int t = lane; t < T; t += 32)
@@ -40,7 +37,27 @@ truncate_kernel(const int32_t *responses, int B, int T, int eos_id, int pad_id,
     }
 }
 
+__global__ void __launch_bounds__(128)
+truncate_kernel(const int32_t *responses, int B, int T, int eos_id, int pad_id,
+                const float *__restrict__ scores, float no_eos_score, int32_t *responses_out,
+                int32_t *__restrict__ eos_index, int32_t *__restrict__ seq_len, uint8_t *__restrict__ mask,
+                float *__restrict__ scores_out)
+{
+    const int b = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
+    if (b >= B) return;
+    truncate_sequence(responses, b, T, eos_id, pad_id, scores, no_eos_score, responses_out, eos_index, seq_len, mask,
+                      scores_out, threadIdx.x & 31);
+}
+
 // ---------------------------------------------------------------- step 3: KL rewards
+// Explicitly rounded fp32 operations: the fused kernel below must reproduce these bits.
+__device__ __forceinline__ float kl_reward(float k, bool real, float kl_coef, bool last, float score)
+{
+    float r = real ? __fmul_rn(-kl_coef, k) : 0.f;
+    if (last) r = __fadd_rn(r, score);
+    return r;
+}
+
 __global__ void __launch_bounds__(256)
 kl_rewards_kernel(const float *__restrict__ logprob, const float *__restrict__ ref_logprob,
                   const uint8_t *__restrict__ mask, const int32_t *__restrict__ seq_len,
@@ -50,13 +67,10 @@ kl_rewards_kernel(const float *__restrict__ logprob, const float *__restrict__ r
     const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     if (i >= (int64_t)B * T) return;
     const int b = (int)(i / T), t = (int)(i - (int64_t)b * T);
-    const float k = mask[i] ? logprob[i] - ref_logprob[i] : 0.f;
+    const bool real = mask[i] != 0;
+    const float k = real ? __fsub_rn(logprob[i], ref_logprob[i]) : 0.f;
     if (kl) kl[i] = k;
-    if (rewards) {
-        float r = mask[i] ? -kl_coef * k : 0.f;
-        if (t == seq_len[b] - 1) r += scores[b];
-        rewards[i] = r;
-    }
+    if (rewards) rewards[i] = kl_reward(k, real, kl_coef, t == seq_len[b] - 1, scores[b]);
 }
 
 // ---------------------------------------------------------------- step 4: GAE
@@ -64,27 +78,21 @@ kl_rewards_kernel(const float *__restrict__ logprob, const float *__restrict__ r
 // recurrence A_t = delta_t + c*A_{t+1} over a segment is an affine map of the incoming A, so
 // (1) each lane folds its segment into (a, b), (2) a reverse inclusive warp scan composes the
 // maps, (3) each lane replays its segment from the correct incoming value. fp64 throughout.
-__global__ void __launch_bounds__(128)
-gae_kernel(const float *__restrict__ rewards, const float *__restrict__ values,
-           const int32_t *__restrict__ seq_len, int B, int T, double gamma, double c /* gamma*lam */,
-           float *__restrict__ advantages, float *__restrict__ returns)
+// `reward(t)` yields the fp32 reward of token t.
+template <typename RewardFn>
+__device__ __forceinline__ void gae_sequence(RewardFn reward, const float *__restrict__ v, int L, int T, double gamma,
+                                             double c, float *__restrict__ advantages, float *__restrict__ returns,
+                                             int lane)
 {
-    const int b = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
-    const int lane = threadIdx.x & 31;
-    if (b >= B) return;
-    int L = seq_len[b];
     L = L < 0 ? 0 : (L > T ? T : L);
-    const float *r = rewards + (int64_t)b * T;
-    const float *v = values + (int64_t)b * T;
     const int S = (T + 31) / 32;
     const int s0 = min(lane * S, T), s1 = min(s0 + S, T);
-
     double a = 1.0, bb = 0.0;
     for (int t = s1 - 1; t >= s0; --t) {
         double d = 0.0;
         if (t < L) {
             const double vn = (t + 1 < L) ? (double)v[t + 1] : 0.0;
-            d = ((double)r[t] + gamma * vn) - (double)v[t];
+            d = ((double)reward(t) + gamma * vn) - (double)v[t];
         }
         bb = d + c * bb;
         a = c * a;
@@ -101,29 +109,39 @@ gae_kernel(const float *__restrict__ rewards, const float *__restrict__ values,
     double A = __shfl_down_sync(0xffffffffu, bb, 1);
     if (lane == 31) A = 0.0;
     for (int t = s1 - 1; t >= s0; --t) {
-        const int64_t i = (int64_t)b * T + t;
         if (t < L) {
             const double vn = (t + 1 < L) ? (double)v[t + 1] : 0.0;
-            const double d = ((double)r[t] + gamma * vn) - (double)v[t];
+            const double d = ((double)reward(t) + gamma * vn) - (double)v[t];
             A = d + c * A;
-            advantages[i] = (float)A;
-            returns[i] = (float)(A + (double)v[t]);
+            advantages[t] = (float)A;
+            returns[t] = (float)(A + (double)v[t]);
         } else {
             A = c * A;
-            advantages[i] = 0.f;
-            returns[i] = 0.f;
+            advantages[t] = 0.f;
+            returns[t] = 0.f;
         }
     }
+}
+
+__global__ void __launch_bounds__(128)
+gae_kernel(const float *__restrict__ rewards, const float *__restrict__ values,
+           const int32_t *__restrict__ seq_len, int B, int T, double gamma, double c /* gamma*lam */,
+           float *__restrict__ advantages, float *__restrict__ returns)
+{
+    const int b = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
+    if (b >= B) return;
+    const float *r = rewards + (int64_t)b * T;
+    gae_sequence([r](int t) { return r[t]; }, values + (int64_t)b * T, seq_len[b], T, gamma, c,
+                 advantages + (int64_t)b * T, returns + (int64_t)b * T, threadIdx.x & 31);
 }
 
 // ---------------------------------------------------------------- step 5: masked whitening
 // One block: three passes over the (L1/L2-resident) array, fp64 sums in a fixed order.
 constexpr int kWhitenThreads = 1024;
-__global__ void __launch_bounds__(kWhitenThreads)
-whiten_kernel(const float *x, const uint8_t *__restrict__ mask, int64_t n_elems, int shift_mean, float eps,
-              float *out, float *__restrict__ stats3, int *status)
+__device__ __forceinline__ void whiten_block(const float *x, const uint8_t *__restrict__ mask, int64_t n_elems,
+                                             int shift_mean, float eps, float *out, float *__restrict__ stats3,
+                                             int *status, double *red /* 32 doubles */)
 {
-    __shared__ double red[32];
     double sum = 0.0, cnt = 0.0;
     for (int64_t i = threadIdx.x; i < n_elems; i += kWhitenThreads)
         if (!mask || mask[i]) { sum += (double)x[i]; cnt += 1.0; }
@@ -148,16 +166,23 @@ whiten_kernel(const float *x, const uint8_t *__restrict__ mask, int64_t n_elems,
     }
 }
 
+__global__ void __launch_bounds__(kWhitenThreads)
+whiten_kernel(const float *x, const uint8_t *__restrict__ mask, int64_t n_elems, int shift_mean, float eps,
+              float *out, float *__restrict__ stats3, int *status)
+{
+    __shared__ double red[32];
+    whiten_block(x, mask, n_elems, shift_mean, eps, out, stats3, status, red);
+}
+
 // ---------------------------------------------------------------- loss plumbing
 constexpr int kReduceThreads = 1024;
 
-// Prologue of a loss call (one block): counts the real tokens, resets the zero-fill work counter
-// and writes the row order: indices of real rows ascending from the front, masked rows from the
-// back. Each thread owns one contiguous segment of rows, so the order is deterministic.
-__global__ void __launch_bounds__(kReduceThreads)
-loss_prepare_kernel(const uint8_t *__restrict__ mask, int64_t rows, WorkspaceHeader *hdr, int32_t *__restrict__ order)
+// Prologue of a loss call (one block): counts the real tokens, resets the work counters and writes
+// the row order: indices of real rows ascending from the front, masked rows from the back. Each
+// thread owns one contiguous segment of rows, so the order is deterministic.
+__device__ __forceinline__ void loss_prepare_block(const uint8_t *mask, int64_t rows, WorkspaceHeader *hdr,
+                                                   int32_t *__restrict__ order, int *warp_tot /* 32 ints */)
 {
-    __shared__ int warp_tot[32];
     const int64_t seg = (rows + kReduceThreads - 1) / kReduceThreads;
     const int64_t r0 = min(rows, (int64_t)threadIdx.x * seg), r1 = min(rows, r0 + seg);
     int c = 0;
@@ -194,6 +219,71 @@ loss_prepare_kernel(const uint8_t *__restrict__ mask, int64_t rows, WorkspaceHea
         if (mask[r]) order[real_pos++] = (int32_t)r;
         else order[rows - 1 - masked_pos++] = (int32_t)r;
     }
+}
+
+__global__ void __launch_bounds__(kReduceThreads)
+loss_prepare_kernel(const uint8_t *__restrict__ mask, int64_t rows, WorkspaceHeader *hdr, int32_t *__restrict__ order)
+{
+    __shared__ int warp_tot[32];
+    loss_prepare_block(mask, rows, hdr, order, warp_tot);
+}
+
+// ---------------------------------------------------------------- fused launches of ppo_step
+// (1) EOS trick for every response, then the loss prologue on the mask just written: one block.
+__global__ void __launch_bounds__(kReduceThreads)
+step_prologue_kernel(const int32_t *responses, int B, int T, int eos_id, int pad_id, const float *__restrict__ scores,
+                     float no_eos_score, int32_t *responses_out, int32_t *__restrict__ eos_index,
+                     int32_t *__restrict__ seq_len, uint8_t *mask, float *__restrict__ scores_out,
+                     WorkspaceHeader *hdr, int32_t *__restrict__ order)
+{
+    __shared__ int warp_tot[32];
+    const int lane = threadIdx.x & 31;
+    for (int b = threadIdx.x >> 5; b < B; b += kReduceThreads / 32)
+        truncate_sequence(responses, b, T, eos_id, pad_id, scores, no_eos_score, responses_out, eos_index, seq_len, mask,
+                          scores_out, lane);
+    __syncthreads();   // the mask written above is read below by other threads of this block
+    loss_prepare_block(mask, (int64_t)B * T, hdr, order, warp_tot);
+}
+
+// (2) KL rewards + GAE, one warp per sequence; the last block to finish whitens the advantages of the
+// whole batch exactly as whiten_kernel does (same thread assignment, same sums).
+__global__ void __launch_bounds__(kWhitenThreads)
+advantages_kernel(const float *__restrict__ logprob, const float *__restrict__ ref_logprob,
+                  const int32_t *__restrict__ seq_len, const float *__restrict__ scores,
+                  const float *__restrict__ values, const uint8_t *__restrict__ mask, int B, int T, float kl_coef,
+                  double gamma, double c, float eps, float *__restrict__ kl, float *__restrict__ rewards,
+                  float *advantages, float *__restrict__ returns, float *whitened, float *__restrict__ stats3,
+                  WorkspaceHeader *hdr)
+{
+    __shared__ double red[32];
+    __shared__ int is_last;
+    const int lane = threadIdx.x & 31;
+    const int b = blockIdx.x * (kWhitenThreads / 32) + (threadIdx.x >> 5);
+    if (b < B) {
+        const int L = seq_len[b];
+        const float score = scores[b];
+        const float *lp = logprob + (int64_t)b * T, *lr = ref_logprob + (int64_t)b * T;
+        for (int t = lane; t < T; t += 32) {
+            const bool real = t < L;
+            const float k = real ? __fsub_rn(lp[t], lr[t]) : 0.f;
+            kl[(int64_t)b * T + t] = k;
+            rewards[(int64_t)b * T + t] = kl_reward(k, real, kl_coef, t == L - 1, score);
+        }
+        gae_sequence(
+            [=](int t) { return kl_reward(t < L ? __fsub_rn(lp[t], lr[t]) : 0.f, t < L, kl_coef, t == L - 1, score); },
+            values + (int64_t)b * T, L, T, gamma, c, advantages + (int64_t)b * T, returns + (int64_t)b * T, lane);
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int ticket = atomicAdd(&hdr->done_blocks, 1);
+        is_last = ticket == (int)gridDim.x - 1;
+        if (is_last) hdr->done_blocks = 0;   // the loss kernel counts its own blocks with the same word
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    whiten_block(advantages, mask, (int64_t)B * T, 1, eps, whitened, stats3, &hdr->status, red);
 }
 
 // Sum the per-token partials (fixed thread assignment, fp64) and write the eight loss scalars.
@@ -236,6 +326,29 @@ loss_from_logprob_kernel(const float *__restrict__ new_logprob, const float *__r
 int launch_loss_prepare(const uint8_t *mask, int64_t rows, void *workspace, cudaStream_t s)
 {
     loss_prepare_kernel<<<1, kReduceThreads, 0, s>>>(mask, rows, ws_header(workspace), ws_order(workspace, rows));
+    return launch_status();
+}
+
+int launch_step_prologue(const int32_t *responses, int B, int T, const ppo_params *p, const float *scores,
+                         int32_t *responses_out, int32_t *eos_index, int32_t *seq_len, uint8_t *mask, float *scores_out,
+                         void *workspace, cudaStream_t s)
+{
+    step_prologue_kernel<<<1, kReduceThreads, 0, s>>>(responses, B, T, p->eos_id, p->pad_id, scores, p->no_eos_score,
+                                                      responses_out, eos_index, seq_len, mask, scores_out,
+                                                      ws_header(workspace), ws_order(workspace, (int64_t)B * T));
+    return launch_status();
+}
+
+int launch_advantages(const float *logprob, const float *ref_logprob, const int32_t *seq_len, const float *scores,
+                      const float *values, const uint8_t *mask, int B, int T, const ppo_params *p, float *kl,
+                      float *rewards, float *advantages, float *returns, float *whitened, float *stats3, void *workspace,
+                      cudaStream_t s)
+{
+    const unsigned grid = (unsigned)((B + kWhitenThreads / 32 - 1) / (kWhitenThreads / 32));
+    advantages_kernel<<<grid, kWhitenThreads, 0, s>>>(logprob, ref_logprob, seq_len, scores, values, mask, B, T, p->kl_coef,
+                                                      (double)p->gamma, (double)p->gamma * (double)p->lam, p->whiten_eps,
+                                                      kl, rewards, advantages, returns, whitened, stats3,
+                                                      ws_header(workspace));
     return launch_status();
 }
 

@@ -80,6 +80,17 @@ class PPOHotPath:
         _b.step(io, policy_logits.dtype, self.B, self.T, self.V, self.params)
         return self.out
 
+    def capture_step(self, policy_logits, ref_logits, responses, scores, values, values_new, old_logprob=None,
+                     loss_logits=None):
+        """Record one step() on these (fixed) buffers into a CUDA graph; graph.replay() then runs the
+        whole path with a single launch call. The caller must have run step() once before (the first
+        call sets kernel attributes) and keeps the input tensors alive and in place."""
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.step(policy_logits, ref_logits, responses, scores, values, values_new, old_logprob=old_logprob,
+                      loss_logits=loss_logits)
+        return graph
+
     def step_io(self, inputs: dict, cuda: bool = True) -> "_b.PPOStepIO":
         """ppo_step_io for this object's output buffers plus the given input tensors."""
         o = self.out
