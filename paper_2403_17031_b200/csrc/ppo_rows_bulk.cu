@@ -257,6 +257,27 @@ __device__ __forceinline__ void engine_epilogue(const EngineArgs &a, EngineSmem 
                                          (int)threadIdx.x, [] { block_sync_all(); });
 }
 
+// pass 2 of the loss for one thread's two packs of a chunk: d = -+ 2^(x*c + off), packed and stored
+template <typename T, bool NEG>
+__device__ __forceinline__ void gradient_packs(const uint4 *buf, uint4 *dst4, int i0, int nvec, float c, float off)
+{
+    constexpr int N = Pack<T>::N;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int i = i0 + h * kConsumers;
+        if (i < nvec) {
+            float x[N], d[N];
+            Pack<T>::unpack_raw(buf[i], x);
+#pragma unroll
+            for (int q = 0; q < N; ++q) {
+                const float e = ex2(fmaf(x[q], c, off));
+                d[q] = NEG ? -e : e;
+            }
+            st_stream(dst4 + i, Pack<T>::pack(d));
+        }
+    }
+}
+
 // MODE 0: log-prob/entropy. MODE 1: loss forward + backward.
 template <typename T, int MODE, bool ENTROPY, int MIN_BLOCKS>
 __global__ void __launch_bounds__(kEngineThreads, MIN_BLOCKS)
@@ -495,19 +516,16 @@ row_engine_kernel(const EngineArgs a)
             const bool fix_owner = !zero && !bad && ct == (tok / N) % kConsumers;
             for (int c = 0; c < nch; ++c) {
                 const int i0 = c * kChunkPacks + ct;
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int i = i0 + h * kConsumers;
-                    if (i < nvec) {
-                        float x[N], d[N];
-                        Pack<T>::unpack_raw(buf[i], x);
-#pragma unroll
-                        for (int q = 0; q < N; ++q) {
-                            const float e = ex2(fmaf(x[q], a.c, off));
-                            d[q] = zero ? 0.f : (neg ? -e : e);
-                        }
-                        st_stream(dst4 + i, Pack<T>::pack(d));
-                    }
+                // three uniform variants of the same loop: the sign of the scale and the all-zero row
+                // (clipped token, g = 0) are decided once per row, not per element
+                if (zero) {
+                    const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+                    if (i0 < nvec) st_stream(dst4 + i0, z);
+                    if (i0 + kConsumers < nvec) st_stream(dst4 + i0 + kConsumers, z);
+                } else if (neg) {
+                    gradient_packs<T, true>(buf, dst4, i0, nvec, a.c, off);
+                } else {
+                    gradient_packs<T, false>(buf, dst4, i0, nvec, a.c, off);
                 }
                 // the thread that wrote the pack holding the sampled token adds the one-hot term
                 if (fix_owner && c == tok_chunk) {
