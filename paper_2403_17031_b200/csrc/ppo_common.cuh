@@ -212,24 +212,39 @@ struct TokenLoss {
     float pg, vf, kl, pg_clipped, vf_clipped;
 };
 
-// Clipped surrogate and clipped value loss of one real token (Table "PPO hyperparameters":
-// epsilon, epsilon-hat, c1, value-loss clipping on). Evaluated in fp64 from the fp32 inputs so
-// that the branch decisions do not depend on fp32 rounding of intermediate products.
-__device__ __forceinline__ TokenLoss token_loss(float lp_new, float lp_old, float adv, float v, float v_old,
-                                               float ret, float eps, float eps_v, float c1, double n)
+// Clipped surrogate of one real token (Table "PPO hyperparameters": epsilon). fp32: the ratio is one
+// ex2, so that this sits cheaply on the critical path between the two passes over a row; inv_n = 1/n.
+struct PolicyTerm {
+    float g;        // d loss / d new_logprob
+    float pg, kl, pg_clipped;
+};
+
+__device__ __forceinline__ PolicyTerm policy_term(float lp_new, float lp_old, float adv, float eps, float inv_n)
 {
-    TokenLoss o;
-    const double A = adv;
-    const double lr = (double)lp_new - (double)lp_old;
-    const double rho = exp(lr);
-    const double lo = 1.0 - (double)eps, hi = 1.0 + (double)eps;
-    const double rc = rho < lo ? lo : (rho > hi ? hi : rho);
-    const double l1 = -A * rho, l2 = -A * rc;
+    PolicyTerm o;
+    const float lr = lp_new - lp_old;
+    const float rho = ex2(lr * kLog2e);
+    const float lo = 1.f - eps, hi = 1.f + eps;
+    const float rc = rho < lo ? lo : (rho > hi ? hi : rho);
+    const float l1 = -adv * rho, l2 = -adv * rc;
     const bool pclip = l2 > l1;
-    o.pg = (float)(pclip ? l2 : l1);
-    o.g = pclip ? 0.f : (float)(l1 / n);
+    o.pg = pclip ? l2 : l1;
+    o.g = pclip ? 0.f : l1 * inv_n;
     o.pg_clipped = pclip ? 1.f : 0.f;
-    o.kl = (float)(0.5 * lr * lr);
+    o.kl = 0.5f * lr * lr;
+    return o;
+}
+
+// Clipped value loss of one real token (epsilon-hat, c1, value-loss clipping on). Evaluated in fp64
+// from the fp32 inputs so that the branch decision does not depend on fp32 rounding.
+struct ValueTerm {
+    float dvalue;   // d loss / d value
+    float vf, vf_clipped;
+};
+
+__device__ __forceinline__ ValueTerm value_term(float v, float v_old, float ret, float eps_v, float c1, double inv_n)
+{
+    ValueTerm o;
     const double dv = v, dvo = v_old, dr = ret;
     const double vlo = dvo - (double)eps_v, vhi = dvo + (double)eps_v;
     const double vc = dv < vlo ? vlo : (dv > vhi ? vhi : dv);
@@ -237,7 +252,24 @@ __device__ __forceinline__ TokenLoss token_loss(float lp_new, float lp_old, floa
     const bool vclip = e2 > e1;
     o.vf = (float)(vclip ? e2 : e1);
     o.vf_clipped = vclip ? 1.f : 0.f;
-    o.dvalue = vclip ? 0.f : (float)((double)c1 * (dv - dr) / n);
+    o.dvalue = vclip ? 0.f : (float)((double)c1 * (dv - dr) * inv_n);
+    return o;
+}
+
+__device__ __forceinline__ TokenLoss token_loss(float lp_new, float lp_old, float adv, float v, float v_old,
+                                               float ret, float eps, float eps_v, float c1, double n)
+{
+    const double inv_n = 1.0 / n;
+    const PolicyTerm pt = policy_term(lp_new, lp_old, adv, eps, (float)inv_n);
+    const ValueTerm vt = value_term(v, v_old, ret, eps_v, c1, inv_n);
+    TokenLoss o;
+    o.g = pt.g;
+    o.pg = pt.pg;
+    o.kl = pt.kl;
+    o.pg_clipped = pt.pg_clipped;
+    o.dvalue = vt.dvalue;
+    o.vf = vt.vf;
+    o.vf_clipped = vt.vf_clipped;
     return o;
 }
 

@@ -127,8 +127,10 @@ __device__ __forceinline__ SoftmaxState consumer_merge(SoftmaxState st, float *r
 }
 
 // Merge for the common case in which no consumer thread moved its reference: plain addition and one
-// named barrier, which also ORs the "my reference differs" flags. Result valid in consumer thread 0.
-// `red` (96 floats) must not be rewritten before the caller's next consumer-wide barrier.
+// named barrier, which also ORs the "my reference differs" flags. Result valid in consumer thread 0,
+// or in every consumer thread when ALL is set (each then adds the 16 warp sums itself, in the same
+// order). `red` (96 floats) must not be rewritten before the caller's next consumer-wide barrier.
+template <bool ALL>
 __device__ __forceinline__ SoftmaxState consumer_merge_common(SoftmaxState st, float m_common, float *red, int ct)
 {
     const int lane = ct & 31, warp = ct >> 5;
@@ -158,7 +160,7 @@ __device__ __forceinline__ SoftmaxState consumer_merge_common(SoftmaxState st, f
     r.m = m_common;
     r.s = 0.f;
     r.u = 0.f;
-    if (ct == 0) {
+    if (ALL || ct == 0) {
 #pragma unroll
         for (int w = 0; w < kConsumerWarps; ++w) {
             r.s += red[w];
@@ -383,7 +385,8 @@ row_engine_kernel(const EngineArgs a)
     const int ct = threadIdx.x;
     const uint4 *buf = reinterpret_cast<const uint4 *>(smem_raw);
     const T *buf_elems = reinterpret_cast<const T *>(smem_raw);
-    const double n_tok = MODE == 1 ? (double)a.hdr->n_tokens : 0.0;
+    const double inv_n = MODE == 1 ? 1.0 / (double)a.hdr->n_tokens : 0.0;
+    const float inv_n_f = (float)inv_n;
     const int64_t G = gridDim.x;
     uint32_t k = 0;
     // Per-row scalars come through dependent loads (row index -> token id -> ...). They are fetched
@@ -403,9 +406,11 @@ row_engine_kernel(const EngineArgs a)
         }
         if (row_c >= 0) {
             tok_c = a.tokens[row_c];
-            if (MODE == 1 && ct == 0) {
+            if (MODE == 1) {
                 in_c[0] = a.loss.old_logprob[row_c];
                 in_c[1] = a.loss.advantages[row_c];
+            }
+            if (MODE == 1 && ct == 0) {
                 in_c[2] = a.loss.values_new[row_c];
                 in_c[3] = a.loss.values_old[row_c];
                 in_c[4] = a.loss.returns[row_c];
@@ -418,9 +423,11 @@ row_engine_kernel(const EngineArgs a)
         if (item + 2 * G < n_items) row_nn = MODE == 1 ? (int64_t)a.order[item + 2 * G] : item + 2 * G;
         if (row_n >= 0) {
             tok_n = a.tokens[row_n];
-            if (MODE == 1 && ct == 0) {
+            if (MODE == 1) {   // every thread derives the gradient scale itself, so every thread needs these two
                 in_n[0] = a.loss.old_logprob[row_n];
                 in_n[1] = a.loss.advantages[row_n];
+            }
+            if (MODE == 1 && ct == 0) {
                 in_n[2] = a.loss.values_new[row_n];
                 in_n[3] = a.loss.values_old[row_n];
                 in_n[4] = a.loss.returns[row_n];
@@ -463,14 +470,14 @@ row_engine_kernel(const EngineArgs a)
             uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
             if (h0) v0 = buf[i0];
             if (h1) v1 = buf[i1];
-            if (ct == 0 && c == tok_chunk) xtok = Pack<T>::load1(buf_elems + tok);
+            if ((MODE == 1 || ct == 0) && c == tok_chunk) xtok = Pack<T>::load1(buf_elems + tok);
             ts.chunk(v0, h0, v1, h1, a.c);
             if (MODE == 0) {
                 __syncwarp();
                 if ((ct & 31) == 0) mbar_arrive(&sm.empty[c]);
             }
         }
-        const SoftmaxState st = consumer_merge_common(ts.state(), m_common, sm.red[parity], ct);   // thread 0 only
+        const SoftmaxState st = consumer_merge_common<MODE == 1>(ts.state(), m_common, sm.red[parity], ct);
         const float l2s = log2f(st.s);
         if (MODE == 0) {
             if (ct == 0) {
@@ -487,26 +494,29 @@ row_engine_kernel(const EngineArgs a)
             }
         } else {
             const LossArgs &la = a.loss;
-            if (ct == 0) {
-                float lp = (fmaf(xtok, a.c, -st.m) - l2s) * kLn2;
+            // Every consumer thread derives the gradient scale from the row sums by itself (a few dozen
+            // fp32 instructions, identical in all threads): no second barrier and no single-thread
+            // section between the two passes over the row.
+            float lp = (fmaf(xtok, a.c, -st.m) - l2s) * kLn2;
+            if (bad) lp = __int_as_float(0x7fc00000);
+            const PolicyTerm pt = policy_term(lp, t_old, t_adv, la.eps, inv_n_f);
+            const float Y = st.m + l2s;           // log2-sum-exp
+            const float gs = pt.g * la.inv_tau;   // gradient scale
+            if (ct == 0) {   // per-token outputs; the other warps are already in pass 2
                 float H = (l2s - st.u / st.s) * kLn2;
                 if (bad) {
-                    lp = H = __int_as_float(0x7fc00000);
+                    H = lp;
                     if (status) atomicOr(status, PPO_DEV_BAD_TOKEN);
                 }
-                const TokenLoss tl = token_loss(lp, t_old, t_adv, t_vn, t_vo, t_ret, la.eps, la.eps_v, la.c1, n_tok);
-                la.dvalues[row] = tl.dvalue;
+                const ValueTerm vt = value_term(t_vn, t_vo, t_ret, la.eps_v, la.c1, inv_n);
+                la.dvalues[row] = vt.dvalue;
                 if (la.new_logprob) la.new_logprob[row] = lp;
                 if (la.entropy) la.entropy[row] = H;
-                if (la.dlogprob) la.dlogprob[row] = tl.g;
+                if (la.dlogprob) la.dlogprob[row] = pt.g;
                 float4 *p4 = reinterpret_cast<float4 *>(la.partials + row * kPartialsPerToken);
-                p4[0] = make_float4(tl.pg, tl.vf, tl.kl, tl.pg_clipped);
-                p4[1] = make_float4(tl.vf_clipped, H, 0.f, 0.f);
-                sm.bc[0] = st.m + l2s;          // log2-sum-exp
-                sm.bc[1] = tl.g * la.inv_tau;   // gradient scale
+                p4[0] = make_float4(pt.pg, vt.vf, pt.kl, pt.pg_clipped);
+                p4[1] = make_float4(vt.vf_clipped, H, 0.f, 0.f);
             }
-            consumer_sync();
-            const float Y = sm.bc[0], gs = sm.bc[1];
             // ---- pass 2: gradient row, chunk by chunk; each chunk is handed back to the producer
             T *dst = reinterpret_cast<T *>(la.dlogits) + row * (int64_t)V;
             uint4 *dst4 = reinterpret_cast<uint4 *>(dst);
