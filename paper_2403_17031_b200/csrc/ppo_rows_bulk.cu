@@ -263,6 +263,7 @@ __device__ __forceinline__ void engine_epilogue(const EngineArgs &a, EngineSmem 
 template <typename T, bool NEG>
 __device__ __forceinline__ void gradient_packs(const uint4 *buf, uint4 *dst4, int i0, int nvec, float c, float off)
 {
+    // (dst4 is the shared-memory row itself in the loss kernel: the gradient replaces the logits in place)
     constexpr int N = Pack<T>::N;
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
@@ -275,7 +276,7 @@ __device__ __forceinline__ void gradient_packs(const uint4 *buf, uint4 *dst4, in
                 const float e = ex2(fmaf(x[q], c, off));
                 d[q] = NEG ? -e : e;
             }
-            st_stream(dst4 + i, Pack<T>::pack(d));
+            dst4[i] = Pack<T>::pack(d);
         }
     }
 }
@@ -354,6 +355,23 @@ row_engine_kernel(const EngineArgs a)
             uint32_t k = 0;
             // the row index of the next item is fetched one row ahead (it is a dependent load)
             int64_t row_next = (MODE == 1 && (int64_t)blockIdx.x < n_items) ? a.order[blockIdx.x] : -1;
+            int64_t prev_row = -1;
+            const auto load_chunk = [&](const unsigned char *src, int c) {
+                const int packs = min(kChunkPacks, nvec - c * kChunkPacks);
+                mbar_expect_tx(&sm.full[c], (uint32_t)packs * 16u);
+                bulk_load(smem_raw + (size_t)c * kChunkBytes, src + (size_t)c * kChunkBytes, (uint32_t)packs * 16u,
+                          &sm.full[c], policy);
+            };
+            // step 6: chunk c of the previous row now holds that row's gradient (written in place by
+            // the consumers): ship it with one bulk shared->global copy
+            const auto store_chunk = [&](int64_t row, int c) {
+                const int packs = min(kChunkPacks, nvec - c * kChunkPacks);
+                unsigned char *dst = reinterpret_cast<unsigned char *>(reinterpret_cast<T *>(a.loss.dlogits) + row * stride);
+                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst + (size_t)c * kChunkBytes),
+                             "r"(smem_addr(smem_raw + (size_t)c * kChunkBytes)), "r"((uint32_t)packs * 16u)
+                             : "memory");
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            };
             for (int64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
                 int64_t row;
                 if (MODE == 0) {
@@ -364,14 +382,34 @@ row_engine_kernel(const EngineArgs a)
                     if (item + gridDim.x < n_items) row_next = a.order[item + gridDim.x];
                 }
                 const unsigned char *src = reinterpret_cast<const unsigned char *>(logits + row * stride);
-                for (int c = 0; c < nch; ++c) {
-                    if (k > 0) mbar_wait(&sm.empty[c], (k - 1) & 1, status);
-                    const int packs = min(kChunkPacks, nvec - c * kChunkPacks);
-                    mbar_expect_tx(&sm.full[c], (uint32_t)packs * 16u);
-                    bulk_load(smem_raw + (size_t)c * kChunkBytes, src + (size_t)c * kChunkBytes, (uint32_t)packs * 16u,
-                              &sm.full[c], policy);
+                if (MODE == 0 || k == 0) {
+                    for (int c = 0; c < nch; ++c) {
+                        if (k > 0) mbar_wait(&sm.empty[c], (k - 1) & 1, status);
+                        load_chunk(src, c);
+                    }
+                } else {
+                    // the store of chunk c must have read shared memory before new bytes may land
+                    // there: the load of a chunk trails its store by one chunk
+                    for (int c = 0; c < nch; ++c) {
+                        mbar_wait(&sm.empty[c], (k - 1) & 1, status);
+                        store_chunk(prev_row, c);
+                        if (c > 0) {
+                            asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                            load_chunk(src, c - 1);
+                        }
+                    }
+                    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    load_chunk(src, nch - 1);
                 }
+                prev_row = row;
                 ++k;
+            }
+            if (MODE == 1 && k > 0) {   // gradient of the block's last row
+                for (int c = 0; c < nch; ++c) {
+                    mbar_wait(&sm.empty[c], (k - 1) & 1, status);
+                    store_chunk(prev_row, c);
+                }
+                asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
             }
         }
         if (MODE == 1) {
@@ -518,20 +556,23 @@ row_engine_kernel(const EngineArgs a)
                 p4[1] = make_float4(vt.vf_clipped, H, 0.f, 0.f);
             }
             // ---- pass 2: gradient row, chunk by chunk; each chunk is handed back to the producer
-            T *dst = reinterpret_cast<T *>(la.dlogits) + row * (int64_t)V;
-            uint4 *dst4 = reinterpret_cast<uint4 *>(dst);
+            // the gradient is written over the logits in shared memory; the producer ships each chunk
+            T *dst = reinterpret_cast<T *>(smem_raw);
+            uint4 *dst4 = reinterpret_cast<uint4 *>(smem_raw);
             // -gs * 2^(y - Y) = -+ 2^(y - Y + log2|gs|): the scale rides in the exponent
             const float off = log2f(fabsf(gs)) - Y;
             const bool zero = gs == 0.f, neg = gs > 0.f;
             const bool fix_owner = !zero && !bad && ct == (tok / N) % kConsumers;
             for (int c = 0; c < nch; ++c) {
                 const int i0 = c * kChunkPacks + ct;
+                float xt_fix = 0.f;   // the token's logit, read before its pack is overwritten in place
+                if (fix_owner && c == tok_chunk) xt_fix = Pack<T>::load1(buf_elems + tok);
                 // three uniform variants of the same loop: the sign of the scale and the all-zero row
                 // (clipped token, g = 0) are decided once per row, not per element
                 if (zero) {
                     const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-                    if (i0 < nvec) st_stream(dst4 + i0, z);
-                    if (i0 + kConsumers < nvec) st_stream(dst4 + i0 + kConsumers, z);
+                    if (i0 < nvec) dst4[i0] = z;
+                    if (i0 + kConsumers < nvec) dst4[i0 + kConsumers] = z;
                 } else if (neg) {
                     gradient_packs<T, true>(buf, dst4, i0, nvec, a.c, off);
                 } else {
@@ -539,9 +580,10 @@ row_engine_kernel(const EngineArgs a)
                 }
                 // the thread that wrote the pack holding the sampled token adds the one-hot term
                 if (fix_owner && c == tok_chunk) {
-                    const float e = ex2(fmaf(Pack<T>::load1(buf_elems + tok), a.c, off));
+                    const float e = ex2(fmaf(xt_fix, a.c, off));
                     Pack<T>::store1(dst + tok, gs + (neg ? -e : e));
                 }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the bulk store
                 __syncwarp();
                 if ((ct & 31) == 0) mbar_arrive(&sm.empty[c]);
             }
