@@ -44,7 +44,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     procs, objs = [], []
     for src in sources():
         obj = os.path.join(obj_dir, os.path.basename(src)[:-3] + ".o")
-        cmd = [_nvcc(), *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-I", INCLUDE, "-I", CSRC,
+        extra = os.environ.get("PPO_NVCC_EXTRA", "").split()      # e.g. -DNAME for a tuning experiment
+        cmd = [_nvcc(), *NVCC_FLAGS, *extra, *(["-Xptxas", "-v"] if verbose else []), "-I", INCLUDE, "-I", CSRC,
                "-c", src, "-o", obj]
         procs.append(subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True))
         objs.append(obj)
