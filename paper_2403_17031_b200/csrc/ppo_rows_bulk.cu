@@ -22,13 +22,13 @@
 
 namespace ppo {
 
-constexpr int kConsumers = 512;                     // 16 consumer warps
-constexpr int kConsumerWarps = kConsumers / 32;
-constexpr int kEngineThreads = kConsumers + 64;     // + one producer warp + one filler warp
+// CONS consumer threads per block (template parameter of everything below): 512 (16 warps) when two
+// blocks share an SM, 960 (30 warps) when a row is so large that only one block fits. Derived sizes:
+// CONS + 64 threads per block (+ one producer warp + one filler warp); two packs per consumer thread
+// and chunk, i.e. chunks of CONS * 32 bytes (16 KB / 30 KB).
 constexpr int kZeroBytes = 4096;                    // shared zeros, source of the bulk zero-fill stores
-constexpr int kChunkPacks = 2 * kConsumers;         // two packs per consumer thread and chunk
-constexpr int kChunkBytes = kChunkPacks * 16;       // 16 KB
-constexpr int kMaxChunks = 14;                      // 224 KB: the largest row one block can hold
+constexpr int kMaxChunks = 14;                      // barriers provided per block
+constexpr size_t kMaxRowBytes = 224 * 1024;         // the largest row one block can hold
 constexpr uint32_t kWaitTries = 1u << 20;           // x ~1 us per try
 
 struct EngineSmem {
@@ -100,11 +100,14 @@ __device__ __forceinline__ uint64_t policy_evict_first()
     return p;
 }
 
-__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory"); }
+template <int CONS>
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"r"(CONS) : "memory"); }
 
-// merge over the 16 consumer warps (named barrier 1); result to every consumer thread
+// merge over the consumer warps (named barrier 1); result to every consumer thread
+template <int CONS>
 __device__ __forceinline__ SoftmaxState consumer_merge(SoftmaxState st, float *red, int ct)
 {
+    constexpr int kConsumerWarps = CONS / 32;
     st = warp_merge(st);
     const int lane = ct & 31, warp = ct >> 5;
     if (lane == 0) {
@@ -112,7 +115,7 @@ __device__ __forceinline__ SoftmaxState consumer_merge(SoftmaxState st, float *r
         red[32 + warp] = st.s;
         red[64 + warp] = st.u;
     }
-    consumer_sync();
+    consumer_sync<CONS>();
     SoftmaxState t;
     if (lane < kConsumerWarps) {
         t.m = red[lane];
@@ -122,7 +125,7 @@ __device__ __forceinline__ SoftmaxState consumer_merge(SoftmaxState st, float *r
         t.init();
     }
     st = warp_merge(t);
-    consumer_sync();
+    consumer_sync<CONS>();
     return st;
 }
 
@@ -130,9 +133,10 @@ __device__ __forceinline__ SoftmaxState consumer_merge(SoftmaxState st, float *r
 // named barrier, which also ORs the "my reference differs" flags. Result valid in consumer thread 0,
 // or in every consumer thread when ALL is set (each then adds the 16 warp sums itself, in the same
 // order). `red` (96 floats) must not be rewritten before the caller's next consumer-wide barrier.
-template <bool ALL>
+template <bool ALL, int CONS>
 __device__ __forceinline__ SoftmaxState consumer_merge_common(SoftmaxState st, float m_common, float *red, int ct)
 {
+    constexpr int kConsumerWarps = CONS / 32;
     const int lane = ct & 31, warp = ct >> 5;
     if (st.s == 0.f) st.m = m_common;
     const uint32_t differs = st.m != m_common;
@@ -150,11 +154,11 @@ __device__ __forceinline__ SoftmaxState consumer_merge_common(SoftmaxState st, f
         "selp.u32 %0, 1, 0, p;\n"
         "}\n"
         : "=r"(any)
-        : "r"(differs), "n"(kConsumers)
+        : "r"(differs), "r"(CONS)
         : "memory");
     if (any) {
-        consumer_sync();
-        return consumer_merge(st, red, ct);
+        consumer_sync<CONS>();
+        return consumer_merge<CONS>(st, red, ct);
     }
     SoftmaxState r;
     r.m = m_common;
@@ -238,31 +242,34 @@ struct EngineArgs {
     float vf_coef;
 };
 
-__device__ __forceinline__ void block_sync_all() { asm volatile("bar.sync 2, %0;" ::"n"(kEngineThreads) : "memory"); }
+template <int CONS>
+__device__ __forceinline__ void block_sync_all() { asm volatile("bar.sync 2, %0;" ::"r"(CONS + 64) : "memory"); }
 
 // End of the loss kernel, reached by every thread of the block once its role is finished: the
 // block takes a ticket; the block that draws the last one sums the per-token partials of the whole
 // batch in a fixed order and writes the loss scalars (so no separate reduction launch is needed
 // and the result does not depend on which block happens to be last).
+template <int CONS>
 __device__ __forceinline__ void engine_epilogue(const EngineArgs &a, EngineSmem &sm)
 {
-    block_sync_all();                       // every partial of this block has been written
+    block_sync_all<CONS>();                       // every partial of this block has been written
     if (threadIdx.x == 0) {
         __threadfence();
         const int ticket = atomicAdd(&a.hdr->done_blocks, 1);
         sm.is_last = ticket == (int)gridDim.x - 1;
     }
-    block_sync_all();
+    block_sync_all<CONS>();
     if (!sm.is_last) return;
     __threadfence();
-    reduce_loss_partials<kEngineThreads>(a.loss.partials, a.loss.rows, a.hdr->n_tokens, a.vf_coef, a.losses, sm.lred,
-                                         (int)threadIdx.x, [] { block_sync_all(); });
+    reduce_loss_partials<CONS + 64>(a.loss.partials, a.loss.rows, a.hdr->n_tokens, a.vf_coef, a.losses, sm.lred,
+                                    (int)threadIdx.x, [] { block_sync_all<CONS>(); });
 }
 
 // pass 2 of the loss for one thread's two packs of a chunk: d = -+ 2^(x*c + off), packed and stored
-template <typename T, bool NEG>
+template <typename T, bool NEG, int CONS>
 __device__ __forceinline__ void gradient_packs(const uint4 *buf, uint4 *dst4, int i0, int nvec, float c, float off)
 {
+    constexpr int kConsumers = CONS;
     // (dst4 is the shared-memory row itself in the loss kernel: the gradient replaces the logits in place)
     constexpr int N = Pack<T>::N;
 #pragma unroll
@@ -282,10 +289,12 @@ __device__ __forceinline__ void gradient_packs(const uint4 *buf, uint4 *dst4, in
 }
 
 // MODE 0: log-prob/entropy. MODE 1: loss forward + backward.
-template <typename T, int MODE, bool ENTROPY, int MIN_BLOCKS>
-__global__ void __launch_bounds__(kEngineThreads, MIN_BLOCKS)
+template <typename T, int MODE, bool ENTROPY, int MIN_BLOCKS, int CONS>
+__global__ void __launch_bounds__(CONS + 64, MIN_BLOCKS)
 row_engine_kernel(const EngineArgs a)
 {
+    constexpr int kConsumers = CONS, kConsumerWarps = CONS / 32, kEngineThreads = CONS + 64;
+    constexpr int kChunkPacks = 2 * CONS, kChunkBytes = kChunkPacks * 16;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ EngineSmem sm;
     constexpr int N = Pack<T>::N;
@@ -344,7 +353,7 @@ row_engine_kernel(const EngineArgs a)
         asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all stores done before the block retires
         }
         __syncwarp();
-        engine_epilogue(a, sm);
+        engine_epilogue<CONS>(a, sm);
         return;
     }
 
@@ -414,7 +423,7 @@ row_engine_kernel(const EngineArgs a)
         }
         if (MODE == 1) {
             __syncwarp();
-            engine_epilogue(a, sm);
+            engine_epilogue<CONS>(a, sm);
         }
         return;
     }
@@ -515,7 +524,7 @@ row_engine_kernel(const EngineArgs a)
                 if ((ct & 31) == 0) mbar_arrive(&sm.empty[c]);
             }
         }
-        const SoftmaxState st = consumer_merge_common<MODE == 1>(ts.state(), m_common, sm.red[parity], ct);
+        const SoftmaxState st = consumer_merge_common<MODE == 1, CONS>(ts.state(), m_common, sm.red[parity], ct);
         const float l2s = log2f(st.s);
         if (MODE == 0) {
             if (ct == 0) {
@@ -574,9 +583,9 @@ row_engine_kernel(const EngineArgs a)
                     if (i0 < nvec) dst4[i0] = z;
                     if (i0 + kConsumers < nvec) dst4[i0 + kConsumers] = z;
                 } else if (neg) {
-                    gradient_packs<T, true>(buf, dst4, i0, nvec, a.c, off);
+                    gradient_packs<T, true, CONS>(buf, dst4, i0, nvec, a.c, off);
                 } else {
-                    gradient_packs<T, false>(buf, dst4, i0, nvec, a.c, off);
+                    gradient_packs<T, false, CONS>(buf, dst4, i0, nvec, a.c, off);
                 }
                 // the thread that wrote the pack holding the sampled token adds the one-hot term
                 if (fix_owner && c == tok_chunk) {
@@ -597,9 +606,9 @@ row_engine_kernel(const EngineArgs a)
         const int64_t n_masked = a.loss.rows - n_items;
         const uint4 z = make_uint4(0u, 0u, 0u, 0u);
         for (;;) {
-            consumer_sync();
+            consumer_sync<CONS>();
             if (ct == 0) sm.next_item = atomicAdd(&a.hdr->masked_next, 1);
-            consumer_sync();
+            consumer_sync<CONS>();
             const int64_t j = sm.next_item;
             if (j >= n_masked) break;
             const int64_t row = a.order[a.loss.rows - 1 - j];
@@ -615,7 +624,7 @@ row_engine_kernel(const EngineArgs a)
                 p4[1] = make_float4(0.f, 0.f, 0.f, 0.f);
             }
         }
-        engine_epilogue(a, sm);
+        engine_epilogue<CONS>(a, sm);
     }
 }
 
@@ -637,21 +646,22 @@ template <typename T, int MODE, bool ENTROPY>
 static int launch_engine(const EngineArgs &a, int64_t max_items, cudaStream_t s)
 {
     const size_t row_bytes = (size_t)a.V * sizeof(T);
-    const int nch = (int)((row_bytes + kChunkBytes - 1) / kChunkBytes);
-    if (nch > kMaxChunks) return PPO_ERR_UNSUPPORTED;
+    if (row_bytes > kMaxRowBytes) return PPO_ERR_UNSUPPORTED;
     const size_t smem = (row_bytes + 127) & ~size_t(127);   // the last chunk may be partial
     const bool two = smem <= 110 * 1024;
     int64_t grid = (int64_t)sm_count() * (two ? 2 : 1);
     if (MODE == 0 && max_items < grid) grid = max_items;
     if (grid < 1) grid = 1;
     if (two) {
-        auto kern = row_engine_kernel<T, MODE, ENTROPY, 2>;
+        // two blocks per SM: 16 consumer warps each, 16 KB chunks
+        auto kern = row_engine_kernel<T, MODE, ENTROPY, 2, 512>;
         PPO_RETURN_IF_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        kern<<<(unsigned)grid, kEngineThreads, smem, s>>>(a);
+        kern<<<(unsigned)grid, 512 + 64, smem, s>>>(a);
     } else {
-        auto kern = row_engine_kernel<T, MODE, ENTROPY, 1>;
+        // one block per SM: 30 consumer warps (a block holds at most 1024 threads), 30 KB chunks
+        auto kern = row_engine_kernel<T, MODE, ENTROPY, 1, 960>;
         PPO_RETURN_IF_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        kern<<<(unsigned)grid, kEngineThreads, smem, s>>>(a);
+        kern<<<(unsigned)grid, 960 + 64, smem, s>>>(a);
     }
     return launch_status();
 }
@@ -660,7 +670,7 @@ template <typename T>
 static bool bulk_ok(const void *base, int64_t stride_elems, int V)
 {
     return aligned16(base) && (stride_elems * (int64_t)sizeof(T)) % 16 == 0 && V % Pack<T>::N == 0 &&
-           (size_t)V * sizeof(T) <= (size_t)kMaxChunks * kChunkBytes;
+           (size_t)V * sizeof(T) <= kMaxRowBytes;
 }
 
 int launch_logprob_bulk(const void *logits, int dtype, int64_t rows, int V, int64_t row_stride,
