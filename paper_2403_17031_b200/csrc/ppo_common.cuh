@@ -20,7 +20,8 @@ struct WorkspaceHeader {
     int n_tokens;      // number of mask==1 tokens of the loss call in flight
     int masked_next;   // work counter of the zero-fill phase (reset by every loss call)
     int done_blocks;   // blocks of the loss kernel that have retired (reset by every loss call)
-    int reserved[60];
+    int step_blocks;   // blocks of ppo_step's token-level kernel that have finished (resets itself)
+    int reserved[59];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header is one 256-byte block");
 
@@ -314,13 +315,8 @@ __device__ __forceinline__ void reduce_loss_partials(const float *partials, int6
 }
 
 // launchers shared between translation units
-int launch_step_prologue(const int32_t *responses, int B, int T, const ppo_params *p, const float *scores,
-                         int32_t *responses_out, int32_t *eos_index, int32_t *seq_len, uint8_t *mask, float *scores_out,
-                         void *workspace, cudaStream_t s);
-int launch_advantages(const float *logprob, const float *ref_logprob, const int32_t *seq_len, const float *scores,
-                      const float *values, const uint8_t *mask, int B, int T, const ppo_params *p, float *kl,
-                      float *rewards, float *advantages, float *returns, float *whitened, float *stats3, void *workspace,
-                      cudaStream_t s);
+// all token-level steps of ppo_step in one launch (EOS trick, KL rewards, GAE, loss prologue, whitening)
+int launch_rollout(const ppo_step_io *io, int B, int T, const ppo_params *p, cudaStream_t s);
 // ppo_loss_fwd_bwd without its prologue launch (the caller has already run the prologue on this mask)
 int loss_fwd_bwd_prepared(const void *logits, int dtype, int32_t B, int32_t T, int64_t V, const int32_t *tokens,
                           const uint8_t *mask, const float *old_logprob, const float *advantages,

@@ -23,20 +23,15 @@ extern "C" int ppo_step(const ppo_step_io *io, int dtype, int32_t B, int32_t T, 
     const int64_t rows = (int64_t)B * T;
     if (rows >= ((int64_t)1 << 31)) return PPO_ERR_SHAPE;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    // five launches: [EOS trick + loss prologue] -> log-probs (policy) -> log-probs (reference) ->
-    // [KL rewards + GAE + whitening] -> loss forward/backward
-    int rc = launch_step_prologue(io->responses, B, T, p, io->scores, io->responses_out, io->eos_index, io->seq_len,
-                                  io->mask, io->scores_out, io->workspace, s);
-    if (rc) return rc;
-    rc = ppo_logprob_entropy(io->policy_logits, dtype, rows, V, V, io->responses, nullptr, p->temperature, io->logprob,
-                             io->entropy, nullptr, io->workspace, stream);
+    // four launches: log-probs (policy) -> log-probs (reference) -> [EOS trick + KL rewards + GAE, then
+    // loss prologue + whitening in the last block] -> loss forward/backward
+    int rc = ppo_logprob_entropy(io->policy_logits, dtype, rows, V, V, io->responses, nullptr, p->temperature,
+                                 io->logprob, io->entropy, nullptr, io->workspace, stream);
     if (rc) return rc;
     rc = ppo_logprob_entropy(io->ref_logits, dtype, rows, V, V, io->responses, nullptr, p->temperature,
                              io->ref_logprob, nullptr, nullptr, io->workspace, stream);
     if (rc) return rc;
-    rc = launch_advantages(io->logprob, io->ref_logprob, io->seq_len, io->scores_out, io->values, io->mask, B, T, p, io->kl,
-                           io->rewards, io->advantages, io->returns, io->advantages_whitened, io->whiten_stats,
-                           io->workspace, s);
+    rc = launch_rollout(io, B, T, p, s);
     if (rc) return rc;
     return loss_fwd_bwd_prepared(io->loss_logits ? io->loss_logits : io->policy_logits, dtype, B, T, V, io->responses,
                                  io->mask, io->old_logprob ? io->old_logprob : io->logprob, io->advantages_whitened,

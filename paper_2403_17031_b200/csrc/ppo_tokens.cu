@@ -10,7 +10,7 @@ int option_value(int key) { return (key >= 0 && key < 8) ? g_options[key] : 0; }
 
 // ---------------------------------------------------------------- step 2: EOS trick
 // One warp per response: lanes stride over t, a warp-wide min finds the first EOS.
-__device__ __forceinline__ void truncate_sequence(const int32_t *responses, int b, int T, int eos_id, int pad_id,
+__device__ __forceinline__ int truncate_sequence(const int32_t *responses, int b, int T, int eos_id, int pad_id,
                                                   const float *__restrict__ scores, float no_eos_score,
                                                   int32_t *responses_out, int32_t *__restrict__ eos_index,
                                                   int32_t *__restrict__ seq_len, uint8_t *__restrict__ mask,
@@ -35,6 +35,7 @@ __device__ __forceinline__ void truncate_sequence(const int32_t *responses, int 
         if (seq_len) seq_len[b] = L;
         if (scores_out) scores_out[b] = e >= 0 ? scores[b] : no_eos_score;
     }
+    return L;   // known to every lane
 }
 
 __global__ void __launch_bounds__(128)
@@ -228,40 +229,36 @@ loss_prepare_kernel(const uint8_t *__restrict__ mask, int64_t rows, WorkspaceHea
     loss_prepare_block(mask, rows, hdr, order, warp_tot);
 }
 
-// ---------------------------------------------------------------- fused launches of ppo_step
-// (1) EOS trick for every response, then the loss prologue on the mask just written: one block.
-__global__ void __launch_bounds__(kReduceThreads)
-step_prologue_kernel(const int32_t *responses, int B, int T, int eos_id, int pad_id, const float *__restrict__ scores,
-                     float no_eos_score, int32_t *responses_out, int32_t *__restrict__ eos_index,
-                     int32_t *__restrict__ seq_len, uint8_t *mask, float *__restrict__ scores_out,
-                     WorkspaceHeader *hdr, int32_t *__restrict__ order)
-{
-    __shared__ int warp_tot[32];
-    const int lane = threadIdx.x & 31;
-    for (int b = threadIdx.x >> 5; b < B; b += kReduceThreads / 32)
-        truncate_sequence(responses, b, T, eos_id, pad_id, scores, no_eos_score, responses_out, eos_index, seq_len, mask,
-                          scores_out, lane);
-    __syncthreads();   // the mask written above is read below by other threads of this block
-    loss_prepare_block(mask, (int64_t)B * T, hdr, order, warp_tot);
-}
-
-// (2) KL rewards + GAE, one warp per sequence; the last block to finish whitens the advantages of the
-// whole batch exactly as whiten_kernel does (same thread assignment, same sums).
+// ---------------------------------------------------------------- fused launch of ppo_step
+// Everything token-level in one launch, after the two log-prob calls (which do not need the mask):
+// one warp per sequence runs the EOS trick, the KL rewards and GAE; the last block to finish then
+// runs the loss prologue (token count, row order) and whitens the advantages of the whole batch,
+// each with exactly the code and thread assignment of the stand-alone kernels, so the results are
+// bit-identical to calling the steps one by one.
 __global__ void __launch_bounds__(kWhitenThreads)
-advantages_kernel(const float *__restrict__ logprob, const float *__restrict__ ref_logprob,
-                  const int32_t *__restrict__ seq_len, const float *__restrict__ scores,
-                  const float *__restrict__ values, const uint8_t *__restrict__ mask, int B, int T, float kl_coef,
-                  double gamma, double c, float eps, float *__restrict__ kl, float *__restrict__ rewards,
-                  float *advantages, float *__restrict__ returns, float *whitened, float *__restrict__ stats3,
-                  WorkspaceHeader *hdr)
+rollout_kernel(const int32_t *responses, int B, int T, int eos_id, int pad_id, const float *__restrict__ scores,
+               float no_eos_score, int32_t *responses_out, int32_t *__restrict__ eos_index,
+               int32_t *__restrict__ seq_len, uint8_t *mask, float *__restrict__ scores_out,
+               const float *__restrict__ logprob, const float *__restrict__ ref_logprob,
+               const float *__restrict__ values, float kl_coef, double gamma, double c, float eps,
+               float *__restrict__ kl, float *__restrict__ rewards, float *advantages, float *__restrict__ returns,
+               float *whitened, float *__restrict__ stats3, WorkspaceHeader *hdr, int32_t *__restrict__ order)
 {
+    static_assert(kWhitenThreads == kReduceThreads, "one block shape for both block-wide helpers");
     __shared__ double red[32];
+    __shared__ int warp_tot[32];
     __shared__ int is_last;
     const int lane = threadIdx.x & 31;
     const int b = blockIdx.x * (kWhitenThreads / 32) + (threadIdx.x >> 5);
     if (b < B) {
-        const int L = seq_len[b];
-        const float score = scores[b];
+        const int L = truncate_sequence(responses, b, T, eos_id, pad_id, scores, no_eos_score, responses_out, eos_index,
+                                        seq_len, mask, scores_out, lane);
+        int first_eos = 0;   // whether the sequence has an EOS decides the score that is used
+        {
+            const int32_t *r = responses + (int64_t)b * T;
+            first_eos = (L < T) || (r[T - 1] == eos_id);
+        }
+        const float score = first_eos ? scores[b] : no_eos_score;
         const float *lp = logprob + (int64_t)b * T, *lr = ref_logprob + (int64_t)b * T;
         for (int t = lane; t < T; t += 32) {
             const bool real = t < L;
@@ -276,14 +273,17 @@ advantages_kernel(const float *__restrict__ logprob, const float *__restrict__ r
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
-        const int ticket = atomicAdd(&hdr->done_blocks, 1);
+        const int ticket = atomicAdd(&hdr->step_blocks, 1);
         is_last = ticket == (int)gridDim.x - 1;
-        if (is_last) hdr->done_blocks = 0;   // the loss kernel counts its own blocks with the same word
+        if (is_last) hdr->step_blocks = 0;   // ready for the next call
     }
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    whiten_block(advantages, mask, (int64_t)B * T, 1, eps, whitened, stats3, &hdr->status, red);
+    const int64_t rows = (int64_t)B * T;
+    loss_prepare_block(mask, rows, hdr, order, warp_tot);
+    __syncthreads();
+    whiten_block(advantages, mask, rows, 1, eps, whitened, stats3, &hdr->status, red);
 }
 
 // Sum the per-token partials (fixed thread assignment, fp64) and write the eight loss scalars.
@@ -329,26 +329,14 @@ int launch_loss_prepare(const uint8_t *mask, int64_t rows, void *workspace, cuda
     return launch_status();
 }
 
-int launch_step_prologue(const int32_t *responses, int B, int T, const ppo_params *p, const float *scores,
-                         int32_t *responses_out, int32_t *eos_index, int32_t *seq_len, uint8_t *mask, float *scores_out,
-                         void *workspace, cudaStream_t s)
-{
-    step_prologue_kernel<<<1, kReduceThreads, 0, s>>>(responses, B, T, p->eos_id, p->pad_id, scores, p->no_eos_score,
-                                                      responses_out, eos_index, seq_len, mask, scores_out,
-                                                      ws_header(workspace), ws_order(workspace, (int64_t)B * T));
-    return launch_status();
-}
-
-int launch_advantages(const float *logprob, const float *ref_logprob, const int32_t *seq_len, const float *scores,
-                      const float *values, const uint8_t *mask, int B, int T, const ppo_params *p, float *kl,
-                      float *rewards, float *advantages, float *returns, float *whitened, float *stats3, void *workspace,
-                      cudaStream_t s)
+int launch_rollout(const ppo_step_io *io, int B, int T, const ppo_params *p, cudaStream_t s)
 {
     const unsigned grid = (unsigned)((B + kWhitenThreads / 32 - 1) / (kWhitenThreads / 32));
-    advantages_kernel<<<grid, kWhitenThreads, 0, s>>>(logprob, ref_logprob, seq_len, scores, values, mask, B, T, p->kl_coef,
-                                                      (double)p->gamma, (double)p->gamma * (double)p->lam, p->whiten_eps,
-                                                      kl, rewards, advantages, returns, whitened, stats3,
-                                                      ws_header(workspace));
+    rollout_kernel<<<grid, kWhitenThreads, 0, s>>>(
+        io->responses, B, T, p->eos_id, p->pad_id, io->scores, p->no_eos_score, io->responses_out, io->eos_index,
+        io->seq_len, io->mask, io->scores_out, io->logprob, io->ref_logprob, io->values, p->kl_coef, (double)p->gamma,
+        (double)p->gamma * (double)p->lam, p->whiten_eps, io->kl, io->rewards, io->advantages, io->returns,
+        io->advantages_whitened, io->whiten_stats, ws_header(io->workspace), ws_order(io->workspace, (int64_t)B * T));
     return launch_status();
 }
 
