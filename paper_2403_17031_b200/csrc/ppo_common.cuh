@@ -21,7 +21,8 @@ struct WorkspaceHeader {
     int masked_next;   // work counter of the zero-fill phase (reset by every loss call)
     int done_blocks;   // blocks of the loss kernel that have retired (reset by every loss call)
     int step_blocks;   // blocks of ppo_step's token-level kernel that have finished (resets itself)
-    int reserved[59];
+    int real_next;     // work counter of the loss kernel's mask==1 rows (reset by every loss call)
+    int reserved[58];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header is one 256-byte block");
 

@@ -38,6 +38,7 @@ struct EngineSmem {
     float bc[4];
     int next_item;
     int is_last;
+    int ring[4];           // row of the block's k-th item at [k % 4], -1 = no further item
     double lred[6 * 32];
     alignas(128) unsigned char zeros[kZeroBytes];
 };
@@ -312,6 +313,7 @@ row_engine_kernel(const EngineArgs a)
             mbar_init(&sm.full[c], 1);
             mbar_init(&sm.empty[c], kConsumerWarps);
         }
+        for (int q = 0; q < 4; ++q) sm.ring[q] = -1;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (MODE == 1) {
@@ -362,8 +364,32 @@ row_engine_kernel(const EngineArgs a)
         if (threadIdx.x == kConsumers) {
             const uint64_t policy = policy_evict_first();
             uint32_t k = 0;
-            // the row index of the next item is fetched one row ahead (it is a dependent load)
-            int64_t row_next = (MODE == 1 && (int64_t)blockIdx.x < n_items) ? a.order[blockIdx.x] : -1;
+            // Rows are handed out dynamically (SMs do not all stream at the same speed): step 6 draws
+            // items from a counter in the workspace header, step 1 walks the rows with a grid stride
+            // and settles rows with mask 0 on the way. -1 = nothing left.
+            int64_t it_static = blockIdx.x;
+            const auto fetch = [&]() -> int {
+                if constexpr (MODE == 1) {
+                    const int64_t item = atomicAdd(&a.hdr->real_next, 1);
+                    return item < n_items ? a.order[item] : -1;
+                } else {
+                    while (it_static < n_items) {
+                        const int64_t row = it_static;
+                        it_static += gridDim.x;
+                        if (!a.mask || a.mask[row]) return (int)row;
+                        a.logprob[row] = 0.f;
+                        if (a.entropy) a.entropy[row] = 0.f;
+                        if (a.lse) a.lse[row] = 0.f;
+                    }
+                    return -1;
+                }
+            };
+            // the block's rows reach the consumers through sm.ring; the entry for item k + 1 is written
+            // before the first copy of item k is armed, and read after that copy has landed
+            int row_c = fetch();
+            int row_n = row_c >= 0 ? fetch() : -1;
+            sm.ring[0] = row_c;
+            if (row_c < 0) mbar_arrive(&sm.full[0]);   // no row at all: complete the phase the consumers wait for
             int64_t prev_row = -1;
             const auto load_chunk = [&](const unsigned char *src, int c) {
                 const int packs = min(kChunkPacks, nvec - c * kChunkPacks);
@@ -381,15 +407,10 @@ row_engine_kernel(const EngineArgs a)
                              : "memory");
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             };
-            for (int64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
-                int64_t row;
-                if (MODE == 0) {
-                    row = item;
-                    if (a.mask && !a.mask[row]) continue;
-                } else {
-                    row = row_next;
-                    if (item + gridDim.x < n_items) row_next = a.order[item + gridDim.x];
-                }
+            while (row_c >= 0) {
+                const int64_t row = row_c;
+                sm.ring[(k + 1) & 3] = row_n;
+                const int row_nn = row_n >= 0 ? fetch() : -1;   // needed one row from now
                 const unsigned char *src = reinterpret_cast<const unsigned char *>(logits + row * stride);
                 if (MODE == 0 || k == 0) {
                     for (int c = 0; c < nch; ++c) {
@@ -411,6 +432,8 @@ row_engine_kernel(const EngineArgs a)
                     load_chunk(src, nch - 1);
                 }
                 prev_row = row;
+                row_c = row_n;
+                row_n = row_nn;
                 ++k;
             }
             if (MODE == 1 && k > 0) {   // gradient of the block's last row
@@ -434,69 +457,31 @@ row_engine_kernel(const EngineArgs a)
     const T *buf_elems = reinterpret_cast<const T *>(smem_raw);
     const double inv_n = MODE == 1 ? 1.0 / (double)a.hdr->n_tokens : 0.0;
     const float inv_n_f = (float)inv_n;
-    const int64_t G = gridDim.x;
     uint32_t k = 0;
-    // Per-row scalars come through dependent loads (row index -> token id -> ...). They are fetched
-    // ahead of time so that no warp starts a row late: row index two rows ahead, token id and the
-    // per-token inputs one row ahead. The token's logit itself is read from the resident row.
-    int64_t row_c = -1, row_n = -1;
+    // The block's rows come from sm.ring (see the producer). Per-row scalars are dependent loads
+    // (row -> token id, old log-prob, ...): they are requested for the NEXT row as soon as its index is
+    // known (first chunk of the current row) and become current at the end of the iteration.
+    int row_c, row_n = -1;
     int tok_c = -1, tok_n = -1;
     float in_c[5] = {0.f, 0.f, 0.f, 0.f, 0.f}, in_n[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
-    {
-        const int64_t item0 = blockIdx.x;
+    mbar_wait(&sm.full[0], 0, status);
+    row_c = sm.ring[0];
+    if (row_c >= 0) {
+        tok_c = a.tokens[row_c];
         if (MODE == 1) {
-            if (item0 < n_items) row_c = a.order[item0];
-            if (item0 + G < n_items) row_n = a.order[item0 + G];
-        } else {
-            if (item0 < n_items) row_c = item0;
-            if (item0 + G < n_items) row_n = item0 + G;
+            in_c[0] = a.loss.old_logprob[row_c];
+            in_c[1] = a.loss.advantages[row_c];
         }
-        if (row_c >= 0) {
-            tok_c = a.tokens[row_c];
-            if (MODE == 1) {
-                in_c[0] = a.loss.old_logprob[row_c];
-                in_c[1] = a.loss.advantages[row_c];
-            }
-            if (MODE == 1 && ct == 0) {
-                in_c[2] = a.loss.values_new[row_c];
-                in_c[3] = a.loss.values_old[row_c];
-                in_c[4] = a.loss.returns[row_c];
-            }
+        if (MODE == 1 && ct == 0) {
+            in_c[2] = a.loss.values_new[row_c];
+            in_c[3] = a.loss.values_old[row_c];
+            in_c[4] = a.loss.returns[row_c];
         }
     }
-    for (int64_t item = blockIdx.x; item < n_items; item += G) {
-        // prefetch for the rows that follow
-        int64_t row_nn = -1;
-        if (item + 2 * G < n_items) row_nn = MODE == 1 ? (int64_t)a.order[item + 2 * G] : item + 2 * G;
-        if (row_n >= 0) {
-            tok_n = a.tokens[row_n];
-            if (MODE == 1) {   // every thread derives the gradient scale itself, so every thread needs these two
-                in_n[0] = a.loss.old_logprob[row_n];
-                in_n[1] = a.loss.advantages[row_n];
-            }
-            if (MODE == 1 && ct == 0) {
-                in_n[2] = a.loss.values_new[row_n];
-                in_n[3] = a.loss.values_old[row_n];
-                in_n[4] = a.loss.returns[row_n];
-            }
-        }
+    while (row_c >= 0) {
         const int64_t row = row_c;
         const int tok = tok_c;
         const float t_old = in_c[0], t_adv = in_c[1], t_vn = in_c[2], t_vo = in_c[3], t_ret = in_c[4];
-        row_c = row_n;
-        row_n = row_nn;
-        tok_c = tok_n;
-#pragma unroll
-        for (int q = 0; q < 5; ++q) in_c[q] = in_n[q];
-
-        if (MODE == 0 && a.mask && !a.mask[row]) {
-            if (ct == 0) {
-                a.logprob[row] = 0.f;
-                if (a.entropy) a.entropy[row] = 0.f;
-                if (a.lse) a.lse[row] = 0.f;
-            }
-            continue;
-        }
         const bool bad = tok < 0 || tok >= V;
         const int tok_chunk = bad ? -1 : (tok / N) / kChunkPacks;
         float xtok = 0.f;
@@ -511,6 +496,20 @@ row_engine_kernel(const EngineArgs a)
                 Pack<T>::unpack(buf[0], x, xmax);
                 m_common = safe_reference(xmax, a.c);
                 ts.init(m_common);
+                // the next row is known now: request its scalars
+                row_n = sm.ring[(k + 1) & 3];
+                if (row_n >= 0) {
+                    tok_n = a.tokens[row_n];
+                    if (MODE == 1) {   // every thread derives the gradient scale itself, so every thread needs these two
+                        in_n[0] = a.loss.old_logprob[row_n];
+                        in_n[1] = a.loss.advantages[row_n];
+                    }
+                    if (MODE == 1 && ct == 0) {
+                        in_n[2] = a.loss.values_new[row_n];
+                        in_n[3] = a.loss.values_old[row_n];
+                        in_n[4] = a.loss.returns[row_n];
+                    }
+                }
             }
             const int i0 = c * kChunkPacks + ct, i1 = i0 + kConsumers;
             const bool h0 = i0 < nvec, h1 = i1 < nvec;
@@ -597,6 +596,10 @@ row_engine_kernel(const EngineArgs a)
                 if ((ct & 31) == 0) mbar_arrive(&sm.empty[c]);
             }
         }
+        row_c = row_n;
+        tok_c = tok_n;
+#pragma unroll
+        for (int q = 0; q < 5; ++q) in_c[q] = in_n[q];
         ++k;
     }
 

@@ -209,6 +209,7 @@ __device__ __forceinline__ void loss_prepare_block(const uint8_t *mask, int64_t 
         if (lane == 31) {
             hdr->n_tokens = wi;
             hdr->masked_next = 0;
+            hdr->real_next = 0;
             hdr->done_blocks = 0;
             if (wi == 0) atomicOr(&hdr->status, PPO_DEV_EMPTY_MASK);
         }
