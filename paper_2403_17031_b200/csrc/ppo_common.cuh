@@ -283,10 +283,26 @@ __device__ __forceinline__ void reduce_loss_partials(const float *partials, int6
                                                      float *losses, double *red, int t, SyncFn sync)
 {
     double acc[6] = {0, 0, 0, 0, 0, 0};
-    for (int64_t r = t; r < rows; r += NT) {
-        const float4 p0 = __ldcg(reinterpret_cast<const float4 *>(partials + r * kPartialsPerToken));
-        const float4 p1 = __ldcg(reinterpret_cast<const float4 *>(partials + r * kPartialsPerToken) + 1);
-        acc[0] += p0.x; acc[1] += p0.y; acc[2] += p0.z; acc[3] += p0.w; acc[4] += p1.x; acc[5] += p1.y;
+    // the loads of four rows are issued before the first sum needs one (the block that runs this is
+    // the only one left: nothing else hides the latency); the order of the additions stays r = t, t + NT, ...
+    constexpr int kBatch = 4;
+    for (int64_t r = t; r < rows; r += kBatch * (int64_t)NT) {
+        float4 p0[kBatch], p1[kBatch];
+#pragma unroll
+        for (int q = 0; q < kBatch; ++q) {
+            const int64_t rq = r + q * (int64_t)NT;
+            p0[q] = p1[q] = make_float4(0.f, 0.f, 0.f, 0.f);   // past the end: adds +0, which changes no sum
+            if (rq < rows) {
+                const float4 *src = reinterpret_cast<const float4 *>(partials + rq * kPartialsPerToken);
+                p0[q] = __ldcg(src);
+                p1[q] = __ldcg(src + 1);
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < kBatch; ++q) {
+            acc[0] += p0[q].x; acc[1] += p0[q].y; acc[2] += p0[q].z; acc[3] += p0[q].w;
+            acc[4] += p1[q].x; acc[5] += p1[q].y;
+        }
     }
     const int lane = t & 31, warp = t >> 5;
 #pragma unroll
