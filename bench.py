@@ -33,7 +33,7 @@ import torch  # noqa: E402
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the committed ncu capture of the same
 # configuration (profiles/loss_fwd_bwd_row_engine_config1.md); None where no capture of the current kernel exists.
 NCU_TRAFFIC_BYTES = {1: 161.627e6 + 288.077e6}
-LAUNCHES_PER_STEP = 4   # ppo_step: 2x logprob, rollout (token-level steps + loss prologue), row_engine (loss)
+LAUNCHES_PER_STEP = 3   # ppo_step: logprob pair (policy + reference), rollout (token-level steps + loss prologue), row_engine (loss)
 
 
 def _peaks(key="hbm_gbs", fallback=6650.0):

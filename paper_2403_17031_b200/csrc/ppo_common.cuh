@@ -341,6 +341,10 @@ int loss_fwd_bwd_prepared(const void *logits, int dtype, int32_t B, int32_t T, i
                           float *losses, void *dlogits, float *dvalues, float *new_logprob, float *entropy,
                           float *dlogprob, void *workspace, void *stream, bool prepared);
 int launch_loss_prepare(const uint8_t *mask, int64_t rows, void *workspace, cudaStream_t s);
+// step 1 for policy and reference logits in one launch; PPO_ERR_UNSUPPORTED if the layout rules it out
+int launch_logprob_pair(const void *policy_logits, const void *ref_logits, int dtype, int64_t rows, int V,
+                        const int32_t *tokens, float c, float *logprob, float *entropy, float *ref_logprob,
+                        int *status, cudaStream_t s);
 int launch_loss_finalize(int64_t rows, float vf_coef, float *losses, void *workspace, cudaStream_t s);
 
 // tuning options (ppo_set_option)

@@ -16,12 +16,12 @@ namespace ppo {
 // One block per row (grid = rows). Kept free of loop-carried state so that it fits 32 registers:
 // eight blocks of 256 threads per SM.
 template <typename T, bool VECTOR, bool ENTROPY, int THREADS>
-__global__ void __launch_bounds__(THREADS)
-logprob_entropy_kernel(const T *__restrict__ logits, int V, int64_t row_stride, const int32_t *__restrict__ tokens,
-                       const uint8_t *__restrict__ mask, float c, float *__restrict__ logprob,
-                       float *__restrict__ entropy, float *__restrict__ lse, int *status)
+__device__ __forceinline__ void logprob_entropy_row(const T *__restrict__ logits, int V, int64_t row_stride,
+                                                    const int32_t *__restrict__ tokens,
+                                                    const uint8_t *__restrict__ mask, float c,
+                                                    float *__restrict__ logprob, float *__restrict__ entropy,
+                                                    float *__restrict__ lse, int *status, float *red)
 {
-    __shared__ float red[96];
     const int64_t row = blockIdx.x;
     if (mask && !mask[row]) {
         if (threadIdx.x == 0) {
@@ -57,6 +57,35 @@ logprob_entropy_kernel(const T *__restrict__ logits, int V, int64_t row_stride, 
         if (entropy) entropy[row] = H;
         if (lse) lse[row] = L;
     }
+}
+
+template <typename T, bool VECTOR, bool ENTROPY, int THREADS>
+__global__ void __launch_bounds__(THREADS)
+logprob_entropy_kernel(const T *__restrict__ logits, int V, int64_t row_stride, const int32_t *__restrict__ tokens,
+                       const uint8_t *__restrict__ mask, float c, float *__restrict__ logprob,
+                       float *__restrict__ entropy, float *__restrict__ lse, int *status)
+{
+    __shared__ float red[96];
+    logprob_entropy_row<T, VECTOR, ENTROPY, THREADS>(logits, V, row_stride, tokens, mask, c, logprob, entropy, lse,
+                                                     status, red);
+}
+
+// Step 1 for the policy and the frozen reference in one launch (grid.y = 2): same tokens, same shape.
+// y = 0: policy logits -> log-prob and entropy; y = 1: reference logits -> log-prob only. One launch
+// instead of two saves a launch boundary, at which the SMs drain and refill.
+template <typename T, int THREADS>
+__global__ void __launch_bounds__(THREADS)
+logprob_pair_kernel(const T *__restrict__ policy_logits, const T *__restrict__ ref_logits, int V,
+                    const int32_t *__restrict__ tokens, float c, float *__restrict__ logprob,
+                    float *__restrict__ entropy, float *__restrict__ ref_logprob, int *status)
+{
+    __shared__ float red[96];
+    if (blockIdx.y == 0)
+        logprob_entropy_row<T, true, true, THREADS>(policy_logits, V, V, tokens, nullptr, c, logprob, entropy, nullptr,
+                                                    status, red);
+    else
+        logprob_entropy_row<T, true, false, THREADS>(ref_logits, V, V, tokens, nullptr, c, ref_logprob, nullptr,
+                                                     nullptr, status, red);
 }
 
 // ---------------------------------------------------------------- step 6 kernel
@@ -218,6 +247,28 @@ static int launch_logprob(const void *logits, int64_t rows, int V, int64_t row_s
         if (entropy) PPO_LAUNCH_LP(false, true); else PPO_LAUNCH_LP(false, false);
     }
 #undef PPO_LAUNCH_LP
+    return launch_status();
+}
+
+// PPO_ERR_UNSUPPORTED when the pointers or the shape do not allow 16-byte packs (the caller then makes two calls)
+int launch_logprob_pair(const void *policy_logits, const void *ref_logits, int dtype, int64_t rows, int V,
+                        const int32_t *tokens, float c, float *logprob, float *entropy, float *ref_logprob,
+                        int *status, cudaStream_t s)
+{
+    constexpr int THREADS = 256;
+    const size_t es = dtype == PPO_F32 ? 4 : 2;
+    const int N = dtype == PPO_F32 ? 4 : 8;
+    if (!aligned16(policy_logits) || !aligned16(ref_logits) || ((size_t)V * es) % 16 != 0 || V % N != 0)
+        return PPO_ERR_UNSUPPORTED;
+    const dim3 grid((unsigned)rows, 2);
+    if (dtype == PPO_F32)
+        logprob_pair_kernel<float, THREADS><<<grid, THREADS, 0, s>>>(
+            reinterpret_cast<const float *>(policy_logits), reinterpret_cast<const float *>(ref_logits), V, tokens, c,
+            logprob, entropy, ref_logprob, status);
+    else
+        logprob_pair_kernel<__nv_bfloat16, THREADS><<<grid, THREADS, 0, s>>>(
+            reinterpret_cast<const __nv_bfloat16 *>(policy_logits), reinterpret_cast<const __nv_bfloat16 *>(ref_logits),
+            V, tokens, c, logprob, entropy, ref_logprob, status);
     return launch_status();
 }
 

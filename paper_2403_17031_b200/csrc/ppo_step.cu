@@ -23,13 +23,21 @@ extern "C" int ppo_step(const ppo_step_io *io, int dtype, int32_t B, int32_t T, 
     const int64_t rows = (int64_t)B * T;
     if (rows >= ((int64_t)1 << 31)) return PPO_ERR_SHAPE;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    // four launches: log-probs (policy) -> log-probs (reference) -> [EOS trick + KL rewards + GAE, then
-    // loss prologue + whitening in the last block] -> loss forward/backward
-    int rc = ppo_logprob_entropy(io->policy_logits, dtype, rows, V, V, io->responses, nullptr, p->temperature,
+    // three launches: log-probs (policy and reference) -> [EOS trick + KL rewards + GAE, then loss
+    // prologue + whitening in the last block] -> loss forward/backward
+    int rc = PPO_ERR_UNSUPPORTED;
+    if ((dtype == PPO_F32 || dtype == PPO_BF16) && V < ((int64_t)1 << 31) && p->temperature > 0.f &&
+        finite_f(p->temperature) && option_value(PPO_OPT_ROW_ENGINE) != 2)
+        rc = launch_logprob_pair(io->policy_logits, io->ref_logits, dtype, rows, (int)V, io->responses,
+                                 kLog2e / p->temperature, io->logprob, io->entropy, io->ref_logprob,
+                                 &ws_header(io->workspace)->status, s);
+    if (rc == PPO_ERR_UNSUPPORTED) {   // layout without 16-byte packs (or the row engine was asked for): two calls
+        rc = ppo_logprob_entropy(io->policy_logits, dtype, rows, V, V, io->responses, nullptr, p->temperature,
                                  io->logprob, io->entropy, nullptr, io->workspace, stream);
-    if (rc) return rc;
-    rc = ppo_logprob_entropy(io->ref_logits, dtype, rows, V, V, io->responses, nullptr, p->temperature,
-                             io->ref_logprob, nullptr, nullptr, io->workspace, stream);
+        if (rc) return rc;
+        rc = ppo_logprob_entropy(io->ref_logits, dtype, rows, V, V, io->responses, nullptr, p->temperature,
+                                 io->ref_logprob, nullptr, nullptr, io->workspace, stream);
+    }
     if (rc) return rc;
     rc = launch_rollout(io, B, T, p, s);
     if (rc) return rc;
