@@ -32,7 +32,7 @@ import torch  # noqa: E402
 
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the committed ncu capture of the same
 # configuration (profiles/loss_fwd_bwd_row_engine_config1.md); None where no capture of the current kernel exists.
-NCU_TRAFFIC_BYTES = {1: 161.627e6 + 288.077e6}
+NCU_TRAFFIC_BYTES = {1: 160.008e6 + 283.032e6}
 LAUNCHES_PER_STEP = 3   # ppo_step: logprob pair (policy + reference), rollout (token-level steps + loss prologue), row_engine (loss)
 
 
@@ -377,7 +377,7 @@ def run_ours(args, cfg):
                        "logprob_entropy_frac_of_peak": lp_gbs / peak, "loss_fwd_bwd_ms": loss_ms,
                        "launch": "cuda graph replay of ppo_step" if graph is not None else "eager ppo_step",
                        "device_status": status},
-            "roofline": {"bound": "hbm", "kernel": "loss_rows_kernel (ppo_loss_fwd_bwd)", "achieved": loss_gbs,
+            "roofline": {"bound": "hbm", "kernel": "row_engine_kernel (ppo_loss_fwd_bwd)", "achieved": loss_gbs,
                          "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": loss_gbs / peak,
                          "frac_of_8tbs": loss_gbs / 8000.0, "traffic": NCU_TRAFFIC_BYTES.get(cfg.index),
                          "algorithmic_bytes": loss_bytes,
