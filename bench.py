@@ -218,6 +218,10 @@ def run_ours(args, cfg):
     binding.lib()
 
     h = cfg.hyper
+    if args.whiten_rewards:   # optional reward whitening before GAE: one more token-level launch per step
+        import dataclasses
+        h = dataclasses.replace(h, whiten_rewards=1)
+    launches_per_step = LAUNCHES_PER_STEP + (1 if args.whiten_rewards else 0)
     B, T, V = cfg.B, cfg.T, cfg.V
     batch = make_batch(cfg, dev, seed=cfg.seed + 1000 * rank)
     hp = PPOHotPath(B, T, V, cfg.torch_dtype, binding.params_from(h), device=dev)
@@ -376,6 +380,7 @@ def run_ours(args, cfg):
                        "logprob_entropy_ms": lp_ms, "logprob_entropy_gbs": lp_gbs,
                        "logprob_entropy_frac_of_peak": lp_gbs / peak, "loss_fwd_bwd_ms": loss_ms,
                        "launch": "cuda graph replay of ppo_step" if graph is not None else "eager ppo_step",
+                       "whiten_rewards": bool(args.whiten_rewards),
                        "device_status": status},
             "roofline": {"bound": "hbm", "kernel": "row_engine_kernel (ppo_loss_fwd_bwd)", "achieved": loss_gbs,
                          "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": loss_gbs / peak,
@@ -386,7 +391,7 @@ def run_ours(args, cfg):
             "clocks": clk.summary(),
             "e2e": e2e,
             "cpu_baseline": cpu,
-            "gpu_launches": LAUNCHES_PER_STEP * K,
+            "gpu_launches": launches_per_step * K,
         }
         print(json.dumps(line), flush=True)
     if distributed:
@@ -510,6 +515,8 @@ def main():
     ap.add_argument("--lm-rows", type=int, default=None, help="config 4: rows of H (default 512*53)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--eager", action="store_true", help="launch every step call by call instead of replaying a CUDA graph")
+    ap.add_argument("--whiten-rewards", action="store_true",
+                    help="detail '(Optional) Reward whitening': whiten the rewards (mean kept) before GAE")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=10)

@@ -70,11 +70,16 @@ enum { PPO_LOSS_PG = 0, PPO_LOSS_VF = 1, PPO_LOSS_TOTAL = 2, PPO_LOSS_APPROX_KL 
  * "EOS trick"; whiten_eps 1e-8 from the whiten() listing; eos_id 0 (Pythia <|endoftext|>);
  * pad_id must be set by the caller to a [PAD] id different from eos_id (section "Dataset ->
  * ... do not use EOS synonymously as [PAD]"); the default 1 is only a placeholder.
+ * whiten_rewards (default 0 = off): detail "(Optional) Reward whitening" - when non-zero, ppo_step
+ * whitens the per-token rewards of the batch over its real tokens with shift_mean = 0 (mean kept)
+ * before GAE; callers of the separate entry points do the same with ppo_whiten between
+ * ppo_kl_rewards and ppo_gae.  Only ppo_step reads this field.
  */
 typedef struct ppo_params {
     float temperature, kl_coef, gamma, lam, cliprange, cliprange_value, vf_coef, no_eos_score,
         whiten_eps;
     int32_t eos_id, pad_id;
+    int32_t whiten_rewards;
 } ppo_params;
 
 void ppo_default_params(ppo_params *p /* host */);
@@ -277,7 +282,8 @@ int ppo_lmhead_logprob_entropy(const void *H, const void *W, int64_t M, int64_t 
  *            responses [B,T] i32; scores [B]; values, values_new [B,T];
  *            old_logprob [B,T] or NULL (= the log-probs this call computes: first PPO epoch, ratio 1)
  *   outputs  responses_out, eos_index, seq_len, mask, scores_out (step 2); logprob, entropy,
- *            ref_logprob (step 1); kl, rewards (step 3); advantages, returns (step 4);
+ *            ref_logprob (step 1); kl, rewards (step 3; with params.whiten_rewards the rewards
+ *            array holds the whitened rewards that GAE consumed); advantages, returns (step 4);
  *            advantages_whitened, whiten_stats[3] (step 5); losses[8], dlogits, dvalues and the
  *            nullable new_logprob, new_entropy, dlogprob (step 6); workspace (device only)
  *

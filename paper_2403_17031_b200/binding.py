@@ -34,7 +34,7 @@ class PPOParams(C.Structure):
     _fields_ = [("temperature", C.c_float), ("kl_coef", C.c_float), ("gamma", C.c_float), ("lam", C.c_float),
                 ("cliprange", C.c_float), ("cliprange_value", C.c_float), ("vf_coef", C.c_float),
                 ("no_eos_score", C.c_float), ("whiten_eps", C.c_float), ("eos_id", C.c_int32),
-                ("pad_id", C.c_int32)]
+                ("pad_id", C.c_int32), ("whiten_rewards", C.c_int32)]
 
 
 class PPOStepIO(C.Structure):
@@ -164,8 +164,8 @@ def default_params(pad_id: Optional[int] = None, **overrides) -> PPOParams:
 def params_from(h) -> PPOParams:
     """PPOParams from any object with the same attribute names (e.g. synthetic.PPOHyper)."""
     p = PPOParams()
-    for name, _ in PPOParams._fields_:
-        setattr(p, name, getattr(h, name))
+    for name, ctype in PPOParams._fields_:
+        setattr(p, name, int(getattr(h, name)) if ctype is C.c_int32 else getattr(h, name))
     return p
 
 

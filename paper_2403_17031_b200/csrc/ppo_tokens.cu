@@ -236,14 +236,21 @@ loss_prepare_kernel(const uint8_t *__restrict__ mask, int64_t rows, WorkspaceHea
 // runs the loss prologue (token count, row order) and whitens the advantages of the whole batch,
 // each with exactly the code and thread assignment of the stand-alone kernels, so the results are
 // bit-identical to calling the steps one by one.
+//
+// PHASE 0: all of it. With reward whitening (detail "(Optional) Reward whitening": the rewards of the
+// batch are whitened without shifting the mean BEFORE GAE) the advantages need batch-wide statistics of
+// the rewards first, so the work is split over two launches of the same kernel:
+// PHASE 1: EOS trick + KL rewards; the last block whitens the rewards in place (shift_mean = 0);
+// PHASE 2: GAE on the rewards array; the last block runs the loss prologue + advantage whitening.
+template <int PHASE>
 __global__ void __launch_bounds__(kWhitenThreads)
 rollout_kernel(const int32_t *responses, int B, int T, int eos_id, int pad_id, const float *__restrict__ scores,
-               float no_eos_score, int32_t *responses_out, int32_t *__restrict__ eos_index,
-               int32_t *__restrict__ seq_len, uint8_t *mask, float *__restrict__ scores_out,
-               const float *__restrict__ logprob, const float *__restrict__ ref_logprob,
-               const float *__restrict__ values, float kl_coef, double gamma, double c, float eps,
-               float *__restrict__ kl, float *__restrict__ rewards, float *advantages, float *__restrict__ returns,
-               float *whitened, float *__restrict__ stats3, WorkspaceHeader *hdr, int32_t *__restrict__ order)
+               float no_eos_score, int32_t *responses_out, int32_t *eos_index, int32_t *seq_len, uint8_t *mask,
+               float *__restrict__ scores_out, const float *__restrict__ logprob,
+               const float *__restrict__ ref_logprob, const float *__restrict__ values, float kl_coef, double gamma,
+               double c, float eps, float *__restrict__ kl, float *rewards, float *advantages,
+               float *__restrict__ returns, float *whitened, float *__restrict__ stats3, WorkspaceHeader *hdr,
+               int32_t *__restrict__ order)
 {
     static_assert(kWhitenThreads == kReduceThreads, "one block shape for both block-wide helpers");
     __shared__ double red[32];
@@ -252,24 +259,34 @@ rollout_kernel(const int32_t *responses, int B, int T, int eos_id, int pad_id, c
     const int lane = threadIdx.x & 31;
     const int b = blockIdx.x * (kWhitenThreads / 32) + (threadIdx.x >> 5);
     if (b < B) {
-        const int L = truncate_sequence(responses, b, T, eos_id, pad_id, scores, no_eos_score, responses_out, eos_index,
-                                        seq_len, mask, scores_out, lane);
-        int first_eos = 0;   // whether the sequence has an EOS decides the score that is used
-        {
-            const int32_t *r = responses + (int64_t)b * T;
-            first_eos = (L < T) || (r[T - 1] == eos_id);
+        if (PHASE == 2) {
+            const float *r = rewards + (int64_t)b * T;
+            gae_sequence([r](int t) { return r[t]; }, values + (int64_t)b * T, seq_len[b], T, gamma, c,
+                         advantages + (int64_t)b * T, returns + (int64_t)b * T, lane);
+        } else {
+            const int L = truncate_sequence(responses, b, T, eos_id, pad_id, scores, no_eos_score, responses_out,
+                                            eos_index, seq_len, mask, scores_out, lane);
+            int first_eos = 0;   // whether the sequence has an EOS decides the score that is used
+            {
+                const int32_t *r = responses + (int64_t)b * T;
+                first_eos = (L < T) || (r[T - 1] == eos_id);
+            }
+            const float score = first_eos ? scores[b] : no_eos_score;
+            const float *lp = logprob + (int64_t)b * T, *lr = ref_logprob + (int64_t)b * T;
+            for (int t = lane; t < T; t += 32) {
+                const bool real = t < L;
+                const float k = real ? __fsub_rn(lp[t], lr[t]) : 0.f;
+                kl[(int64_t)b * T + t] = k;
+                rewards[(int64_t)b * T + t] = kl_reward(k, real, kl_coef, t == L - 1, score);
+            }
+            if (PHASE == 0)
+                gae_sequence(
+                    [=](int t) {
+                        return kl_reward(t < L ? __fsub_rn(lp[t], lr[t]) : 0.f, t < L, kl_coef, t == L - 1, score);
+                    },
+                    values + (int64_t)b * T, L, T, gamma, c, advantages + (int64_t)b * T, returns + (int64_t)b * T,
+                    lane);
         }
-        const float score = first_eos ? scores[b] : no_eos_score;
-        const float *lp = logprob + (int64_t)b * T, *lr = ref_logprob + (int64_t)b * T;
-        for (int t = lane; t < T; t += 32) {
-            const bool real = t < L;
-            const float k = real ? __fsub_rn(lp[t], lr[t]) : 0.f;
-            kl[(int64_t)b * T + t] = k;
-            rewards[(int64_t)b * T + t] = kl_reward(k, real, kl_coef, t == L - 1, score);
-        }
-        gae_sequence(
-            [=](int t) { return kl_reward(t < L ? __fsub_rn(lp[t], lr[t]) : 0.f, t < L, kl_coef, t == L - 1, score); },
-            values + (int64_t)b * T, L, T, gamma, c, advantages + (int64_t)b * T, returns + (int64_t)b * T, lane);
     }
     __threadfence();
     __syncthreads();
@@ -282,6 +299,10 @@ rollout_kernel(const int32_t *responses, int B, int T, int eos_id, int pad_id, c
     if (!is_last) return;
     __threadfence();
     const int64_t rows = (int64_t)B * T;
+    if (PHASE == 1) {
+        whiten_block(rewards, mask, rows, 0, eps, rewards, nullptr, &hdr->status, red);
+        return;
+    }
     loss_prepare_block(mask, rows, hdr, order, warp_tot);
     __syncthreads();
     whiten_block(advantages, mask, rows, 1, eps, whitened, stats3, &hdr->status, red);
@@ -333,11 +354,20 @@ int launch_loss_prepare(const uint8_t *mask, int64_t rows, void *workspace, cuda
 int launch_rollout(const ppo_step_io *io, int B, int T, const ppo_params *p, cudaStream_t s)
 {
     const unsigned grid = (unsigned)((B + kWhitenThreads / 32 - 1) / (kWhitenThreads / 32));
-    rollout_kernel<<<grid, kWhitenThreads, 0, s>>>(
-        io->responses, B, T, p->eos_id, p->pad_id, io->scores, p->no_eos_score, io->responses_out, io->eos_index,
-        io->seq_len, io->mask, io->scores_out, io->logprob, io->ref_logprob, io->values, p->kl_coef, (double)p->gamma,
-        (double)p->gamma * (double)p->lam, p->whiten_eps, io->kl, io->rewards, io->advantages, io->returns,
-        io->advantages_whitened, io->whiten_stats, ws_header(io->workspace), ws_order(io->workspace, (int64_t)B * T));
+#define PPO_LAUNCH_ROLLOUT(PHASE)                                                                                    \
+    rollout_kernel<PHASE><<<grid, kWhitenThreads, 0, s>>>(                                                           \
+        io->responses, B, T, p->eos_id, p->pad_id, io->scores, p->no_eos_score, io->responses_out, io->eos_index,    \
+        io->seq_len, io->mask, io->scores_out, io->logprob, io->ref_logprob, io->values, p->kl_coef,                 \
+        (double)p->gamma, (double)p->gamma * (double)p->lam, p->whiten_eps, io->kl, io->rewards, io->advantages,     \
+        io->returns, io->advantages_whitened, io->whiten_stats, ws_header(io->workspace),                            \
+        ws_order(io->workspace, (int64_t)B * T))
+    if (p->whiten_rewards) {
+        PPO_LAUNCH_ROLLOUT(1);
+        PPO_LAUNCH_ROLLOUT(2);
+    } else {
+        PPO_LAUNCH_ROLLOUT(0);
+    }
+#undef PPO_LAUNCH_ROLLOUT
     return launch_status();
 }
 
@@ -366,6 +396,7 @@ extern "C" void ppo_default_params(ppo_params *p)
     p->whiten_eps = 1e-8f;
     p->eos_id = 0;
     p->pad_id = 1;
+    p->whiten_rewards = 0;
 }
 
 extern "C" int ppo_version(void) { return 100; }

@@ -53,6 +53,8 @@ class PPOHotPath:
                            out=(o["ref_logprob"], None, None))
         _b.kl_rewards(o["logprob"], o["ref_logprob"], o["mask"], o["seq_len"], o["scores_out"], p.kl_coef,
                       out=(o["kl"], o["rewards"]))
+        if p.whiten_rewards:   # optional reward whitening: mean kept, in place, before GAE
+            _b.whiten(o["rewards"], o["mask"], False, p.whiten_eps, workspace=self.workspace, out=o["rewards"])
         _b.gae(o["rewards"], values, o["seq_len"], p.gamma, p.lam, out=(o["advantages"], o["returns"]))
         _b.whiten(o["advantages"], o["mask"], True, p.whiten_eps, workspace=self.workspace,
                   out=o["advantages_whitened"], stats=o["whiten_stats"])

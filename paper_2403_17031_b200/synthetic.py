@@ -35,6 +35,7 @@ class PPOHyper:
     whiten_eps: float = 1e-8       # constant inside the paper's whiten()
     eos_id: int = 0                # Pythia <|endoftext|>
     pad_id: int = 1                # a [PAD] id distinct from EOS
+    whiten_rewards: int = 0        # detail "(Optional) Reward whitening": whiten(rewards, shift_mean=False) before GAE
 
 
 @dataclass(frozen=True)

@@ -80,6 +80,8 @@ def oracle_chain(O, batch, h, old_logprob=None, loss_logits=None, sel_rows=None,
     r["logprob"], r["entropy"], r["ref_logprob"] = lp.reshape(B, T), ent.reshape(B, T), rlp.reshape(B, T)
     r["kl"], r["rewards"] = O.kl_rewards(f32(r["logprob"]), f32(r["ref_logprob"]), r["mask"], r["seq_len"],
                                          f32(r["scores_out"]), np.float32(h.kl_coef))
+    if getattr(h, "whiten_rewards", 0):   # detail "(Optional) Reward whitening": before GAE, mean kept
+        r["rewards"], _ = O.whiten(f32(r["rewards"]), r["mask"], False, np.float32(h.whiten_eps))
     r["advantages"], r["returns"] = O.gae(f32(r["rewards"]), npy(batch["values"]), r["seq_len"],
                                           np.float32(h.gamma), np.float32(h.lam))
     r["advantages_whitened"], r["whiten_stats"] = O.whiten(f32(r["advantages"]), r["mask"], True,

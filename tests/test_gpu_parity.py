@@ -296,3 +296,50 @@ def test_single_call_step_and_host_step_match_the_separate_calls(P):
            batch["values_new"])
     torch.cuda.synchronize()
     assert float(b.out["losses"][3]) == 0.0 and float(b.out["losses"][4]) == 0.0
+
+
+@pytest.mark.parametrize("B,T,V", [(4, 16, 1000), (70, 53, 1000)])
+def test_reward_whitening_before_gae(P, oracle, B, T, V):
+    """Detail "(Optional) Reward whitening": whiten(rewards, shift_mean=False) over the batch's real tokens before
+    GAE. Stage-wise against the oracle, ppo_step against the separate calls (same bits) and against the oracle chain."""
+    import dataclasses
+    from paper_2403_17031_b200.pipeline import PPOHotPath
+    from paper_2403_17031_b200.synthetic import CONFIGS, make_batch
+    cfg = dataclasses.replace(CONFIGS[0], B=B, T=T, V=V,
+                              hyper=dataclasses.replace(CONFIGS[0].hyper, whiten_rewards=1))
+    h = cfg.hyper
+    batch = make_batch(cfg, "cuda")
+    ref = oracle_chain(oracle, batch, h, want_dlogits=False)
+    off = oracle_chain(oracle, batch, dataclasses.replace(h, whiten_rewards=0), want_dlogits=False)
+    assert np.abs(ref["rewards"] - off["rewards"]).max() > 1e-2      # the option changes the rewards ...
+    m = ref["mask"].astype(bool)
+    assert abs(ref["rewards"][m].mean() - off["rewards"][m].mean()) < 1e-7   # ... but not their mean (fp32 inputs)
+    assert abs(ref["rewards"][m].var() - 1.0) < 1e-5                          # and the variance becomes 1
+    # stage-wise: the whitening call on the oracle's raw rewards, GAE on the oracle's whitened rewards
+    rw, _ = P.whiten(dev(f32(off["rewards"])), dev(ref["mask"]), False, h.whiten_eps)
+    assert_rel(npy(rw), ref["rewards"], TOL_REL, "whitened rewards")
+    adv, ret = P.gae(dev(f32(ref["rewards"])), batch["values"], dev(ref["seq_len"]), h.gamma, h.lam)
+    assert_rel(npy(adv), ref["advantages"], TOL_REL, "advantages")
+    assert_rel(npy(ret), ref["returns"], TOL_REL, "returns")
+    # ppo_step == separate calls, bit for bit
+    pp = _params(P, h)
+    assert pp.whiten_rewards == 1
+    a = PPOHotPath(B, T, V, torch.float32, pp)
+    o = a.rollout_stats(batch["policy_logits"], batch["ref_logits"], batch["responses"], batch["scores"],
+                        batch["values"])
+    old = (o["logprob"] + batch["old_logprob_noise"]).contiguous()
+    a.loss(batch["policy_logits"], batch["responses"], old, batch["values_new"], batch["values"])
+    b = PPOHotPath(B, T, V, torch.float32, pp)
+    b.step(batch["policy_logits"], batch["ref_logits"], batch["responses"], batch["scores"], batch["values"],
+           batch["values_new"], old_logprob=old)
+    torch.cuda.synchronize()
+    for k in ("mask", "seq_len", "kl", "rewards", "advantages", "returns", "advantages_whitened", "losses", "dlogits",
+              "dvalues"):
+        assert torch.equal(a.out[k], b.out[k]), k
+    # chained against the oracle: fp32 log-prob errors (<= 1e-4, times kl_coef) are divided by the rewards'
+    # standard deviation and summed by GAE
+    assert_rel(npy(b.out["rewards"]), ref["rewards"], 1e-4, "rewards (chained)")
+    for k in ("advantages", "returns"):
+        assert_rel(npy(b.out[k]), ref[k], 5e-4, k + " (chained)")
+    assert_rel(npy(b.out["advantages_whitened"]), ref["advantages_whitened"], 5e-4, "advantages_whitened (chained)")
+    assert b.device_status() == 0
