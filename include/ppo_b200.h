@@ -237,6 +237,50 @@ int ppo_loss_from_logprob(const float *new_logprob, const float *entropy, int32_
                           float *dvalues, void *workspace, void *stream);
 
 /*
+ * Chain rule from token log-probs back to the logits (the backward half of ppo_logprob_entropy;
+ * used by losses that are functions of sequence log-probs, such as the DPO loss below):
+ *   dlogits[r, j] = dlogprob[r] * (1[j == tokens[r]] - softmax(logits[r, :] / temperature)[j]) / temperature
+ * for rows with mask[r] != 0; rows with mask 0 are zero-filled and their logits are never read.
+ *   logits   [rows, V] dtype, contiguous (row pitch V);  dlogits [rows, V] same dtype, != logits
+ *   tokens   [rows] i32;  mask [rows] u8;  dlogprob [rows] f32 (upstream gradient)
+ *   new_logprob, entropy  nullable [rows] f32 outputs: the row's log-prob / entropy, recomputed on the way
+ *   workspace  required, >= ppo_workspace_bytes(rows, 1, V), 256-byte aligned
+ * One read of the real rows and one write of all rows (same kernels as ppo_loss_fwd_bwd).  A token id
+ * outside [0, V) makes its row NaN and sets PPO_DEV_BAD_TOKEN.
+ */
+int ppo_logprob_bwd(const void *logits, int dtype, int64_t rows, int64_t V, const int32_t *tokens,
+                    const uint8_t *mask, const float *dlogprob, float temperature, void *dlogits,
+                    float *new_logprob, float *entropy, void *workspace, void *stream);
+
+/*
+ * Reward-model loss (section "Preliminaries", step 2): mean over the P pairs of
+ * -log sigma(r_chosen - r_rejected) = log(1 + e^(r_rejected - r_chosen)).
+ *   reward_chosen, reward_rejected  [P] f32
+ *   out4  [4] f32: loss, accuracy (share of pairs with r_chosen > r_rejected), mean r_chosen, mean r_rejected
+ *   dreward_chosen, dreward_rejected  nullable [P] f32: gradient of the mean loss
+ * One block, fp64 sums in a fixed order.  No workspace.
+ */
+int ppo_pairwise_loss(const float *reward_chosen, const float *reward_rejected, int64_t P, float *out4,
+                      float *dreward_chosen, float *dreward_rejected, void *stream);
+
+/*
+ * DPO loss (section "Preliminaries", "RL-free approaches") from token log-probs of the chosen and
+ * the rejected completion under the policy and under the frozen SFT reference:
+ *   reward = beta * (sum_t mask * logprob - sum_t mask * ref_logprob)       (the implicit reward)
+ *   loss   = mean over pairs of -log sigma(reward_chosen - reward_rejected)
+ *   logprob_*, ref_logprob_*  [P, T] f32;  mask_*  [P, T] u8 (1 on response tokens)
+ *   out4  [4] f32: loss, accuracy of the implicit rewards, mean reward_chosen, mean reward_rejected
+ *   reward_chosen, reward_rejected  nullable [P] f32
+ *   dlogprob_chosen, dlogprob_rejected  nullable [P, T] f32: gradient of the mean loss w.r.t. the
+ *       policy's token log-probs (0 outside the mask); feed them to ppo_logprob_bwd
+ * beta: Table "DPO hyperparameters" (0.05).  One block, one warp per pair, fp64 sums in a fixed order.
+ */
+int ppo_dpo_loss(const float *logprob_chosen, const float *logprob_rejected, const float *ref_logprob_chosen,
+                 const float *ref_logprob_rejected, const uint8_t *mask_chosen, const uint8_t *mask_rejected,
+                 int64_t P, int32_t T, float beta, float *out4, float *reward_chosen, float *reward_rejected,
+                 float *dlogprob_chosen, float *dlogprob_rejected, void *stream);
+
+/*
  * Allocation-free variant of ppo_loss_from_logprob (an addition of this library; the paper has no
  * counterpart).  It is meant for callers that cannot obtain device memory at the point of the call:
  * code running under a framework whose allocator must not be re-entered, inside a region where

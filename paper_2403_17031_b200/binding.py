@@ -91,6 +91,11 @@ _SIGS = {
                            C.c_void_p]),
     "ppo_step_host": (C.c_int, [C.POINTER(PPOStepIO), C.POINTER(PPOStepIO), C.c_int, C.c_int32, C.c_int32, C.c_int64,
                                 C.POINTER(PPOParams), C.c_void_p]),
+    "ppo_logprob_bwd": (C.c_int, [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                  C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "ppo_pairwise_loss": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                    C.c_void_p]),
+    "ppo_dpo_loss": (C.c_int, [C.c_void_p] * 6 + [C.c_int64, C.c_int32, C.c_float] + [C.c_void_p] * 6),
     "ppo_lmhead_logprob_entropy": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p,
                                              C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                              C.c_void_p]),
@@ -365,4 +370,53 @@ def lmhead_logprob_entropy(H, W, tokens, temperature: float, workspace, mask=Non
                                           float(temperature), _ptr(lp, torch.float32), _ptr(ent, torch.float32),
                                           _ptr(lse, torch.float32), _ptr(workspace), _stream())
     _check("ppo_lmhead_logprob_entropy", rc)
+    return out
+
+
+def logprob_bwd(logits, tokens, mask, dlogprob, temperature: float, workspace, dlogits=None, want_aux: bool = False):
+    """Gradient on token log-probs -> gradient on the logits [..., V] (rows with mask 0: zeros, never read).
+    Returns dict(dlogits[, new_logprob, entropy])."""
+    V = logits.shape[-1]
+    rows = logits.numel() // V
+    if dlogits is None:
+        dlogits = torch.empty_like(logits)
+    out = {"dlogits": dlogits}
+    if want_aux:
+        out["new_logprob"] = torch.empty(tokens.shape, dtype=torch.float32, device=logits.device)
+        out["entropy"] = torch.empty(tokens.shape, dtype=torch.float32, device=logits.device)
+    rc = lib().ppo_logprob_bwd(_ptr(logits), _logits_dtype(logits), rows, V, _ptr(tokens, torch.int32),
+                               _ptr(mask, torch.uint8), _ptr(dlogprob, torch.float32), float(temperature),
+                               _ptr(dlogits, logits.dtype), _ptr(out.get("new_logprob")), _ptr(out.get("entropy")),
+                               _ptr(workspace), _stream())
+    _check("ppo_logprob_bwd", rc)
+    return out
+
+
+def pairwise_loss(reward_chosen, reward_rejected, want_grad: bool = True):
+    """Reward-model loss of a batch of pairs. Returns dict(out4 = [loss, accuracy, mean r_c, mean r_r][, dr_c, dr_r])."""
+    P = reward_chosen.numel()
+    o = {"out4": torch.empty(4, dtype=torch.float32, device=reward_chosen.device)}
+    if want_grad:
+        o["dr_c"], o["dr_r"] = torch.empty_like(reward_chosen), torch.empty_like(reward_rejected)
+    rc = lib().ppo_pairwise_loss(_ptr(reward_chosen, torch.float32), _ptr(reward_rejected, torch.float32), P,
+                                 _ptr(o["out4"]), _ptr(o.get("dr_c")), _ptr(o.get("dr_r")), _stream())
+    _check("ppo_pairwise_loss", rc)
+    return o
+
+
+def dpo_loss(lp_c, lp_r, ref_c, ref_r, mask_c, mask_r, beta: float, out=None):
+    """DPO loss of P pairs from token log-probs [P,T]. Returns dict(out4 = [loss, accuracy, mean implicit reward
+    chosen, rejected], reward_c, reward_r [P], dlp_c, dlp_r [P,T])."""
+    P, T = lp_c.shape
+    if out is None:
+        dev = lp_c.device
+        out = {"out4": torch.empty(4, dtype=torch.float32, device=dev),
+               "reward_c": torch.empty(P, dtype=torch.float32, device=dev),
+               "reward_r": torch.empty(P, dtype=torch.float32, device=dev),
+               "dlp_c": torch.empty_like(lp_c), "dlp_r": torch.empty_like(lp_r)}
+    rc = lib().ppo_dpo_loss(_ptr(lp_c, torch.float32), _ptr(lp_r, torch.float32), _ptr(ref_c, torch.float32),
+                            _ptr(ref_r, torch.float32), _ptr(mask_c, torch.uint8), _ptr(mask_r, torch.uint8), P, T,
+                            float(beta), _ptr(out["out4"]), _ptr(out["reward_c"]), _ptr(out["reward_r"]),
+                            _ptr(out["dlp_c"]), _ptr(out["dlp_r"]), _stream())
+    _check("ppo_dpo_loss", rc)
     return out

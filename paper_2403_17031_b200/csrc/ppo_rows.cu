@@ -124,7 +124,7 @@ loss_rows_kernel(const LossArgs a)
         if (!a.mask[row]) {
             if (dst) fill_row_zero<T, VECTOR, THREADS>(dst, V);
             if (threadIdx.x == 0) {
-                a.dvalues[row] = 0.f;
+                if (a.dvalues) a.dvalues[row] = 0.f;
                 if (a.new_logprob) a.new_logprob[row] = 0.f;
                 if (a.entropy) a.entropy[row] = 0.f;
                 if (a.dlogprob) a.dlogprob[row] = 0.f;
@@ -140,11 +140,15 @@ loss_rows_kernel(const LossArgs a)
         float xtok = 0.f, t_old = 0.f, t_adv = 0.f, t_vn = 0.f, t_vo = 0.f, t_ret = 0.f;
         if (threadIdx.x == 0) {   // per-token scalars: fetched now, used after the row reduction
             if (!bad) xtok = Pack<T>::load1(src + tok);
-            t_old = a.old_logprob[row];
-            t_adv = a.advantages[row];
-            t_vn = a.values_new[row];
-            t_vo = a.values_old[row];
-            t_ret = a.returns[row];
+            if (a.g_ext) {
+                t_old = a.g_ext[row];
+            } else {
+                t_old = a.old_logprob[row];
+                t_adv = a.advantages[row];
+                t_vn = a.values_new[row];
+                t_vo = a.values_old[row];
+                t_ret = a.returns[row];
+            }
         }
         SoftmaxState st;
         if (VECTOR) {
@@ -163,8 +167,14 @@ loss_rows_kernel(const LossArgs a)
                 lp = H = __int_as_float(0x7fc00000);
                 if (a.status) atomicOr(a.status, PPO_DEV_BAD_TOKEN);
             }
-            const TokenLoss tl = token_loss(lp, t_old, t_adv, t_vn, t_vo, t_ret, a.eps, a.eps_v, a.c1, n);
-            a.dvalues[row] = tl.dvalue;
+            TokenLoss tl;
+            if (a.g_ext) {   // the gradient on the log-prob is an input (a bad token still poisons its row)
+                tl.g = bad ? lp : t_old;
+                tl.dvalue = tl.pg = tl.vf = tl.kl = tl.pg_clipped = tl.vf_clipped = 0.f;
+            } else {
+                tl = token_loss(lp, t_old, t_adv, t_vn, t_vo, t_ret, a.eps, a.eps_v, a.c1, n);
+            }
+            if (a.dvalues) a.dvalues[row] = tl.dvalue;
             if (a.new_logprob) a.new_logprob[row] = lp;
             if (a.entropy) a.entropy[row] = H;
             if (a.dlogprob) a.dlogprob[row] = tl.g;
@@ -384,6 +394,7 @@ int ppo::loss_fwd_bwd_prepared(const void *logits, int dtype, int32_t B, int32_t
     a.V = (int)V;
     a.tokens = tokens;
     a.mask = mask;
+    a.g_ext = nullptr;
     a.old_logprob = old_logprob;
     a.advantages = advantages;
     a.values_new = values_new;
@@ -409,4 +420,47 @@ int ppo::loss_fwd_bwd_prepared(const void *logits, int dtype, int32_t B, int32_t
     rc = dtype == PPO_F32 ? launch_loss<float>(a, s) : launch_loss<__nv_bfloat16>(a, s);
     if (rc) return rc;
     return launch_loss_finalize(rows, p->vf_coef, losses, workspace, s);
+}
+
+extern "C" int ppo_logprob_bwd(const void *logits, int dtype, int64_t rows, int64_t V, const int32_t *tokens,
+                               const uint8_t *mask, const float *dlogprob, float temperature, void *dlogits,
+                               float *new_logprob, float *entropy, void *workspace, void *stream)
+{
+    if (dtype != PPO_F32 && dtype != PPO_BF16) return PPO_ERR_DTYPE;
+    if (rows <= 0 || V <= 0 || V >= ((int64_t)1 << 31) || rows >= ((int64_t)1 << 31)) return PPO_ERR_SHAPE;
+    if (!logits || !tokens || !mask || !dlogprob || !dlogits || !workspace) return PPO_ERR_NULL;
+    if (!(temperature > 0.f) || !finite_f(temperature)) return PPO_ERR_PARAM;
+    const size_t es = dtype == PPO_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(logits) % es || reinterpret_cast<uintptr_t>(dlogits) % es ||
+        reinterpret_cast<uintptr_t>(workspace) % 256)
+        return PPO_ERR_ALIGN;
+    if (dlogits == logits) return PPO_ERR_PARAM;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    int rc = launch_loss_prepare(mask, rows, workspace, s);
+    if (rc) return rc;
+    LossArgs a = {};
+    a.logits = logits;
+    a.dlogits = dlogits;
+    a.rows = rows;
+    a.V = (int)V;
+    a.tokens = tokens;
+    a.mask = mask;
+    a.g_ext = dlogprob;
+    a.new_logprob = new_logprob;
+    a.entropy = entropy;
+    a.partials = ws_partials(workspace);
+    a.n_tokens = &ws_header(workspace)->n_tokens;
+    a.status = &ws_header(workspace)->status;
+    a.c = kLog2e / temperature;
+    a.inv_tau = 1.0f / temperature;
+    // the kernels end with the reduction of the (all-zero) loss partials; it lands in the header's spare words
+    float *sink = reinterpret_cast<float *>(ws_header(workspace)->reserved);
+    rc = PPO_ERR_UNSUPPORTED;
+    if (option_value(PPO_OPT_ROW_ENGINE) != 1) {
+        rc = launch_loss_bulk(a, dtype, workspace, sink, 0.f, s);
+        if (rc != PPO_ERR_UNSUPPORTED) return rc;
+    }
+    rc = dtype == PPO_F32 ? launch_loss<float>(a, s) : launch_loss<__nv_bfloat16>(a, s);
+    if (rc) return rc;
+    return launch_loss_finalize(rows, 0.f, sink, workspace, s);
 }

@@ -228,6 +228,9 @@ struct LossArgs {
     const int32_t *tokens;
     const uint8_t *mask;
     const float *old_logprob, *advantages, *values_new, *values_old, *returns;
+    // log-prob backward only (ppo_logprob_bwd): the gradient on each token's log-prob is given; the five
+    // PPO inputs above and dvalues are null, and no loss term is computed
+    const float *g_ext;
     float *dvalues, *new_logprob, *entropy, *dlogprob;
     float *partials;
     const int *n_tokens;

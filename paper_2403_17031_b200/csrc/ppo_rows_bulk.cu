@@ -342,7 +342,7 @@ row_engine_kernel(const EngineArgs a)
                              : "memory");
             }
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-            la.dvalues[row] = 0.f;
+            if (la.dvalues) la.dvalues[row] = 0.f;
             if (la.new_logprob) la.new_logprob[row] = 0.f;
             if (la.entropy) la.entropy[row] = 0.f;
             if (la.dlogprob) la.dlogprob[row] = 0.f;
@@ -469,10 +469,14 @@ row_engine_kernel(const EngineArgs a)
     if (row_c >= 0) {
         tok_c = a.tokens[row_c];
         if (MODE == 1) {
-            in_c[0] = a.loss.old_logprob[row_c];
-            in_c[1] = a.loss.advantages[row_c];
+            if (a.loss.g_ext) {
+                in_c[0] = a.loss.g_ext[row_c];
+            } else {
+                in_c[0] = a.loss.old_logprob[row_c];
+                in_c[1] = a.loss.advantages[row_c];
+            }
         }
-        if (MODE == 1 && ct == 0) {
+        if (MODE == 1 && ct == 0 && !a.loss.g_ext) {
             in_c[2] = a.loss.values_new[row_c];
             in_c[3] = a.loss.values_old[row_c];
             in_c[4] = a.loss.returns[row_c];
@@ -501,10 +505,14 @@ row_engine_kernel(const EngineArgs a)
                 if (row_n >= 0) {
                     tok_n = a.tokens[row_n];
                     if (MODE == 1) {   // every thread derives the gradient scale itself, so every thread needs these two
-                        in_n[0] = a.loss.old_logprob[row_n];
-                        in_n[1] = a.loss.advantages[row_n];
+                        if (a.loss.g_ext) {
+                            in_n[0] = a.loss.g_ext[row_n];
+                        } else {
+                            in_n[0] = a.loss.old_logprob[row_n];
+                            in_n[1] = a.loss.advantages[row_n];
+                        }
                     }
-                    if (MODE == 1 && ct == 0) {
+                    if (MODE == 1 && ct == 0 && !a.loss.g_ext) {
                         in_n[2] = a.loss.values_new[row_n];
                         in_n[3] = a.loss.values_old[row_n];
                         in_n[4] = a.loss.returns[row_n];
@@ -545,7 +553,13 @@ row_engine_kernel(const EngineArgs a)
             // section between the two passes over the row.
             float lp = (fmaf(xtok, a.c, -st.m) - l2s) * kLn2;
             if (bad) lp = __int_as_float(0x7fc00000);
-            const PolicyTerm pt = policy_term(lp, t_old, t_adv, la.eps, inv_n_f);
+            PolicyTerm pt;
+            if (la.g_ext) {   // the gradient on the log-prob is an input (a bad token still poisons its row)
+                pt.g = bad ? lp : t_old;
+                pt.pg = pt.kl = pt.pg_clipped = 0.f;
+            } else {
+                pt = policy_term(lp, t_old, t_adv, la.eps, inv_n_f);
+            }
             const float Y = st.m + l2s;           // log2-sum-exp
             const float gs = pt.g * la.inv_tau;   // gradient scale
             if (ct == 0) {   // per-token outputs; the other warps are already in pass 2
@@ -554,8 +568,10 @@ row_engine_kernel(const EngineArgs a)
                     H = lp;
                     if (status) atomicOr(status, PPO_DEV_BAD_TOKEN);
                 }
-                const ValueTerm vt = value_term(t_vn, t_vo, t_ret, la.eps_v, la.c1, inv_n);
-                la.dvalues[row] = vt.dvalue;
+                ValueTerm vt;
+                vt.dvalue = vt.vf = vt.vf_clipped = 0.f;
+                if (!la.g_ext) vt = value_term(t_vn, t_vo, t_ret, la.eps_v, la.c1, inv_n);
+                if (la.dvalues) la.dvalues[row] = vt.dvalue;
                 if (la.new_logprob) la.new_logprob[row] = lp;
                 if (la.entropy) la.entropy[row] = H;
                 if (la.dlogprob) la.dlogprob[row] = pt.g;
@@ -618,7 +634,7 @@ row_engine_kernel(const EngineArgs a)
             uint4 *dst4 = reinterpret_cast<uint4 *>(reinterpret_cast<T *>(la.dlogits) + row * (int64_t)V);
             for (int i = ct; i < nvec; i += kConsumers) st_stream(dst4 + i, z);
             if (ct == 0) {
-                la.dvalues[row] = 0.f;
+                if (la.dvalues) la.dvalues[row] = 0.f;
                 if (la.new_logprob) la.new_logprob[row] = 0.f;
                 if (la.entropy) la.entropy[row] = 0.f;
                 if (la.dlogprob) la.dlogprob[row] = 0.f;

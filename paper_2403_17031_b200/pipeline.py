@@ -106,3 +106,40 @@ class PPOHotPath:
 
     def device_status(self) -> int:
         return _b.last_device_status(self.workspace)
+
+
+class DPOStep:
+    """One DPO step on materialised logits (section "Preliminaries", "RL-free approaches"), all on the
+    current CUDA stream: token log-probs of the policy and of the frozen SFT reference on the response
+    rows (prompt and padding rows are skipped, never read), the DPO loss with its implicit rewards, and
+    the gradient back to the policy's logits. Leading axis of every tensor: 0 = chosen, 1 = rejected.
+    Temperature is 1 (the loss is defined on the model's own distribution)."""
+
+    def __init__(self, P: int, T: int, V: int, dtype: torch.dtype, beta: float, device="cuda"):
+        dev = torch.device(device)
+        self.P, self.T, self.V, self.beta = P, T, V, float(beta)
+        f32 = torch.float32
+        self.workspace = _b.new_workspace(_b.workspace_bytes(2 * P * T, 1, V), dev)
+        self.out = {
+            "logprob": torch.empty((2, P, T), dtype=f32, device=dev),
+            "ref_logprob": torch.empty((2, P, T), dtype=f32, device=dev),
+            "out4": torch.empty(4, dtype=f32, device=dev),
+            "reward_c": torch.empty(P, dtype=f32, device=dev), "reward_r": torch.empty(P, dtype=f32, device=dev),
+            "dlogprob": torch.empty((2, P, T), dtype=f32, device=dev),
+            "dlogits": torch.empty((2, P, T, V), dtype=dtype, device=dev),
+        }
+
+    def step(self, policy_logits, ref_logits, tokens, mask):
+        o = self.out
+        _b.logprob_entropy(policy_logits, tokens, 1.0, mask=mask, workspace=self.workspace, want_entropy=False,
+                           out=(o["logprob"], None, None))
+        _b.logprob_entropy(ref_logits, tokens, 1.0, mask=mask, workspace=self.workspace, want_entropy=False,
+                           out=(o["ref_logprob"], None, None))
+        _b.dpo_loss(o["logprob"][0], o["logprob"][1], o["ref_logprob"][0], o["ref_logprob"][1], mask[0], mask[1],
+                    self.beta, out={"out4": o["out4"], "reward_c": o["reward_c"], "reward_r": o["reward_r"],
+                                    "dlp_c": o["dlogprob"][0], "dlp_r": o["dlogprob"][1]})
+        _b.logprob_bwd(policy_logits, tokens, mask, o["dlogprob"], 1.0, self.workspace, dlogits=o["dlogits"])
+        return o
+
+    def device_status(self) -> int:
+        return _b.last_device_status(self.workspace)

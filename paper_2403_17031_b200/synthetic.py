@@ -245,3 +245,68 @@ def make_lmhead_batch(cfg: WorkloadConfig, device="cpu", M: Optional[int] = None
         out["old_logprob_noise"] = 0.15 * torch.randn((Bn, cfg.T), generator=g, device=dev,
                                                        dtype=torch.float32)
     return out
+
+
+# ---------------------------------------------------------------- preference batches (RM / DPO losses)
+@dataclass(frozen=True)
+class PrefConfig:
+    """A batch of preference pairs in the paper's pre-tokenised layout (section "Dataset": query and
+    response concatenated and right-padded to 638 tokens; queries fill the first 512 positions)."""
+    name: str
+    P: int                 # pairs; Table "DPO hyperparameters": batch 64 over 8 GPUs = 8 pairs per GPU
+    T: int = 638
+    V: int = 50304
+    dtype: str = "bf16"
+    query_len: int = 512   # positions [0, query_len) are the prompt: not part of the loss
+    resp_lo: int = 20      # response lengths ~ U[resp_lo, resp_hi]
+    resp_hi: int = 126
+    logit_std: float = 2.0
+    ref_noise: float = 0.5
+    beta: float = 0.05     # Table "DPO hyperparameters"
+    seed: int = BASE_SEED + 5
+
+    @property
+    def torch_dtype(self) -> torch.dtype:
+        return torch.float32 if self.dtype == "f32" else torch.bfloat16
+
+
+PREF_CONFIGS: Dict[str, PrefConfig] = {
+    "tiny": PrefConfig("tiny-pref", P=3, T=24, V=1000, dtype="f32", query_len=10, resp_lo=2, resp_hi=14),
+    "dpo": PrefConfig("dpo-tldr-per-gpu", P=8),
+}
+
+
+def make_pref_batch(cfg: PrefConfig, device="cpu", seed: Optional[int] = None,
+                    chunk_rows: int = 2048) -> Dict[str, torch.Tensor]:
+    """Index 0 of the leading axis = chosen completions, 1 = rejected.
+      policy_logits, ref_logits [2,P,T,V] cfg dtype: N(0, logit_std^2) on response rows (reference = policy
+                                 + N(0, ref_noise^2)), zeros elsewhere (those rows are never read)
+      tokens [2,P,T] int32       labels, uniform over the vocabulary
+      mask   [2,P,T] uint8       1 on the response tokens (query_len <= t < query_len + length)
+      rm_rewards [2,P] float32   stand-in reward-model outputs ~ N(0,1) (+0.5 for chosen)"""
+    seed = cfg.seed if seed is None else seed
+    dev = torch.device(device)
+    g = _gen(dev, seed)
+    gc = _gen("cpu", seed + 7919)
+    P, T, V = cfg.P, cfg.T, cfg.V
+    length = torch.randint(cfg.resp_lo, cfg.resp_hi + 1, (2, P), generator=gc)
+    length = torch.minimum(length, torch.tensor(T - cfg.query_len))
+    t = torch.arange(T)[None, None, :]
+    mask = ((t >= cfg.query_len) & (t < cfg.query_len + length[:, :, None])).to(torch.uint8)
+    tokens = torch.randint(2, V, (2, P, T), generator=gc, dtype=torch.int32)
+    dt = cfg.torch_dtype
+    policy = torch.zeros((2 * P * T, V), dtype=dt, device=dev)
+    ref = torch.zeros((2 * P * T, V), dtype=dt, device=dev)
+    rows = torch.nonzero(mask.reshape(-1)).reshape(-1).to(dev)
+    for r0 in range(0, rows.numel(), chunk_rows):
+        idx = rows[r0:r0 + chunk_rows]
+        x = cfg.logit_std * torch.randn((idx.numel(), V), generator=g, device=dev, dtype=torch.float32)
+        p = x.to(dt)
+        policy[idx] = p
+        ref[idx] = (p.float() + cfg.ref_noise * torch.randn((idx.numel(), V), generator=g, device=dev,
+                                                            dtype=torch.float32)).to(dt)
+        del x, p
+    rm = torch.randn((2, P), generator=g, device=dev, dtype=torch.float32)
+    rm[0] += 0.5
+    return {"policy_logits": policy.view(2, P, T, V), "ref_logits": ref.view(2, P, T, V),
+            "tokens": tokens.to(dev), "mask": mask.to(dev).contiguous(), "rm_rewards": rm}
