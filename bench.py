@@ -31,8 +31,9 @@ if ROOT not in sys.path:
 import torch  # noqa: E402
 
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the committed ncu capture of the same
-# configuration (profiles/loss_fwd_bwd_row_engine_config1.md); None where no capture of the current kernel exists.
-NCU_TRAFFIC_BYTES = {1: 160.008e6 + 283.032e6}
+# configuration (profiles/loss_fwd_bwd_row_engine_config1.md, profiles/dpo_step_config5.md); None where no capture
+# of the current kernel exists.
+NCU_TRAFFIC_BYTES = {1: 160.008e6 + 283.032e6, 5: 109.9e6 + 967.3e6}
 LAUNCHES_PER_STEP = 3   # ppo_step: logprob pair (policy + reference), rollout (token-level steps + loss prologue), row_engine (loss)
 
 
@@ -506,12 +507,123 @@ def run_lmhead(args, cfg):
         dist.destroy_process_group()
 
 
+def run_dpo(args):
+    """Config 5: one DPO step on a batch of preference pairs in the paper's (B, 638) layout: token log-probs of
+    policy and reference on the response rows, DPO loss + implicit rewards, gradient back to the policy's logits."""
+    rank, world, local = _dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    distributed = world > 1
+    if distributed:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2403_17031_b200 import binding, build
+    from paper_2403_17031_b200.pipeline import DPOStep
+    from paper_2403_17031_b200.synthetic import PREF_CONFIGS, make_pref_batch
+    if rank == 0:
+        build.build()
+    if distributed:
+        dist.barrier()
+    binding.lib()
+    cfg = PREF_CONFIGS["dpo"]
+    b = make_pref_batch(cfg, dev, seed=cfg.seed + 1000 * rank)
+    P, T, V = cfg.P, cfg.T, cfg.V
+    st = DPOStep(P, T, V, cfg.torch_dtype, cfg.beta, device=dev)
+    run = lambda: st.step(b["policy_logits"], b["ref_logits"], b["tokens"], b["mask"])
+    for _ in range(max(args.warmup, 3)):
+        run()
+    torch.cuda.synchronize()
+    K = args.steps
+    n_real = int(b["mask"].sum().item())
+    rows = 2 * P * T
+    es = 2 if cfg.dtype == "bf16" else 4
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if distributed:
+        dist.barrier()
+    torch.cuda.synchronize()
+    with ClockSampler(local) as clk:
+        ev0.record()
+        for _ in range(K):
+            run()
+        ev1.record()
+        torch.cuda.synchronize()
+        # the dominant call alone, same workload, right after the timed region
+        bw = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(20)]
+        for e0, e1 in bw:
+            e0.record()
+            binding.logprob_bwd(b["policy_logits"], b["tokens"], b["mask"], st.out["dlogprob"], 1.0, st.workspace,
+                                dlogits=st.out["dlogits"])
+            e1.record()
+        torch.cuda.synchronize()
+    total_ms = ev0.elapsed_time(ev1)
+    if distributed:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / K
+    bwd_ms = statistics.mean(a.elapsed_time(c) for a, c in bw)
+    bwd_bytes = (n_real + rows) * V * es
+    bwd_gbs = bwd_bytes / (bwd_ms * 1e-3) / 1e9
+    path_bytes = (3 * n_real + rows) * V * es     # two log-prob passes + backward read, backward write of all rows
+    peak, kind = _peaks("hbm_gbs", 6650.0)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import numpy as np
+        from oracle import ppo_oracle as O, pref_oracle as R
+        O.build()
+        m = b["mask"].cpu().numpy()
+        idx = np.flatnonzero(m.reshape(-1))
+        tok = b["tokens"].cpu().numpy().reshape(-1)
+        pl = b["policy_logits"].reshape(-1, V)[torch.from_numpy(idx).to(dev)].cpu()
+        rl = b["ref_logits"].reshape(-1, V)[torch.from_numpy(idx).to(dev)].cpu()
+        to_np = lambda t: t.view(torch.int16).numpy().view(np.uint16) if t.dtype == torch.bfloat16 else t.numpy()
+        t0 = time.perf_counter()
+        lp = np.zeros(rows)
+        rlp = np.zeros(rows)
+        lp[idx] = O.logprob_entropy(to_np(pl), tok[idx], 1.0)[0]
+        rlp[idx] = O.logprob_entropy(to_np(rl), tok[idx], 1.0)[0]
+        lp, rlp = lp.reshape(2, P, T), rlp.reshape(2, P, T)
+        d = R.dpo_loss(lp[0], lp[1], rlp[0], rlp[1], m[0], m[1], cfg.beta)
+        g = np.stack([d["dlp_c"], d["dlp_r"]]).reshape(-1)[idx]
+        R.logprob_bwd(pl.double().numpy(), tok[idx], g, 1.0)
+        dt_s = time.perf_counter() - t0
+        cpu = {"value": n_real / dt_s, "unit": "tokens/s", "cores": O.num_threads(), "kind": "oracle",
+               "sample": "the whole batch once: %d response rows of V=%d (log-probs x2 in C/OpenMP, loss and "
+                         "backward in numpy), %.1f s" % (n_real, V, dt_s)}
+    if rank == 0:
+        line = {
+            "metric": "response tokens/s", "value": n_real * world / (ms_per_step * 1e-3), "unit": "tokens/s",
+            "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "config5 %s (DPO step)" % cfg.name, "pairs_per_gpu": P, "T": T, "V": V,
+                       "logits_dtype": cfg.dtype, "response_tokens": n_real, "rows": rows,
+                       "l2": "inputs larger than L2 (%.0f MB of logits read, %.0f MB of gradient written per step)" %
+                             (3 * n_real * V * es / 1e6, rows * V * es / 1e6),
+                       "path_hbm_gbs": path_bytes / (ms_per_step * 1e-3) / 1e9, "logprob_bwd_ms": bwd_ms,
+                       "launch": "eager: 2 x ppo_logprob_entropy, ppo_dpo_loss, ppo_logprob_bwd",
+                       "device_status": st.device_status()},
+            "roofline": {"bound": "hbm", "kernel": "row_engine_kernel (ppo_logprob_bwd)", "achieved": bwd_gbs,
+                         "peak": peak, "peak_kind": kind, "unit": "GB/s", "frac": bwd_gbs / peak,
+                         "frac_of_8tbs": bwd_gbs / 8000.0, "traffic": NCU_TRAFFIC_BYTES.get(5),
+                         "algorithmic_bytes": bwd_bytes,
+                         "timing": "CUDA events around the ppo_logprob_bwd call (prologue + row engine launches), "
+                                   "right after the timed region"},
+            "clocks": clk.summary(), "e2e": None, "cpu_baseline": cpu, "gpu_launches": 5 * K,
+        }
+        print(json.dumps(line), flush=True)
+    if distributed:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--config", type=int, default=1, choices=[1, 2, 3, 4])
+    ap.add_argument("--config", type=int, default=1, choices=[1, 2, 3, 4, 5],
+                    help="1-3: PPO path on stored logits; 4: fused LM head; 5: DPO step on preference pairs")
     ap.add_argument("--lm-rows", type=int, default=None, help="config 4: rows of H (default 512*53)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--eager", action="store_true", help="launch every step call by call instead of replaying a CUDA graph")
@@ -525,7 +637,10 @@ def main():
     ap.add_argument("--ref-seconds", type=float, default=150.0, help="time budget of the reference arm")
     args = ap.parse_args()
     from paper_2403_17031_b200.synthetic import CONFIGS
-    cfg = CONFIGS[args.config]
+    if args.config == 5 and args.impl != "reference":
+        run_dpo(args)
+        return
+    cfg = CONFIGS[1 if args.config == 5 else args.config]
     if args.impl == "reference":
         run_reference(args, CONFIGS[1] if args.config == 4 else cfg)
     elif args.config == 4:
