@@ -320,6 +320,26 @@ int ppo_lmhead_logprob_entropy(const void *H, const void *W, int64_t M, int64_t 
                                void *stream);
 
 /*
+ * Backward of the fused LM head (the step after ppo_loss_from_logprob when the logits were never
+ * materialised): with z = H W / temperature and the gradient g = dlogprob on each token's log-prob,
+ *   dlogits = g * (onehot(token) - softmax(z)) / temperature   [M, V]
+ *   dH = dlogits W^T  [M, K],   dW = H^T dlogits  [K, V]
+ * Three tensor-core passes: the logits are recomputed tile by tile and turned into dlogits in the
+ * epilogue (using the log-sum-exp saved by ppo_lmhead_logprob_entropy), then two contractions.
+ *   H [M,K], W [K,V]  bf16 as in ppo_lmhead_logprob_entropy;  tokens [M] i32;  mask nullable [M] u8
+ *   lse [M] f32       the `lse` output of ppo_lmhead_logprob_entropy for the same H, W, temperature
+ *   dlogprob [M] f32  upstream gradient (rows with mask 0 or dlogprob 0 give zero rows)
+ *   dlogits [M,V] bf16  required scratch AND output: the only intermediate written to memory
+ *   dH [M,K], dW [K,V]  bf16 outputs, each nullable (its pass is skipped)
+ *   workspace  required (status word only), 256-byte aligned
+ * Requirements: K % 8 == 0, V % 8 == 0, all matrices 16-byte aligned; else PPO_ERR_UNSUPPORTED /
+ * PPO_ERR_ALIGN.  Token ids are assumed valid (the forward call reports bad ones).
+ */
+int ppo_lmhead_bwd(const void *H, const void *W, int64_t M, int64_t K, int64_t V, const int32_t *tokens,
+                   const uint8_t *mask, const float *lse, const float *dlogprob, float temperature,
+                   void *dlogits, void *dH, void *dW, void *workspace, void *stream);
+
+/*
  * The whole path in one call.  ppo_step_io names every buffer of one PPO iteration over a batch of
  * B responses x T tokens; all pointers of one struct live in the same memory space.
  *   inputs   policy_logits, ref_logits [B,T,V] (dtype); loss_logits [B,T,V] or NULL (= policy_logits);

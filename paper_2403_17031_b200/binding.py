@@ -91,6 +91,9 @@ _SIGS = {
                            C.c_void_p]),
     "ppo_step_host": (C.c_int, [C.POINTER(PPOStepIO), C.POINTER(PPOStepIO), C.c_int, C.c_int32, C.c_int32, C.c_int64,
                                 C.POINTER(PPOParams), C.c_void_p]),
+    "ppo_lmhead_bwd": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
+                                 C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                 C.c_void_p]),
     "ppo_logprob_bwd": (C.c_int, [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                   C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ppo_pairwise_loss": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -419,4 +422,20 @@ def dpo_loss(lp_c, lp_r, ref_c, ref_r, mask_c, mask_r, beta: float, out=None):
                             float(beta), _ptr(out["out4"]), _ptr(out["reward_c"]), _ptr(out["reward_r"]),
                             _ptr(out["dlp_c"]), _ptr(out["dlp_r"]), _stream())
     _check("ppo_dpo_loss", rc)
+    return out
+
+
+def lmhead_bwd(H, W, tokens, lse, dlogprob, temperature: float, workspace, mask=None, dlogits=None,
+               want_dH: bool = True, want_dW: bool = True, out=None):
+    """Backward of the fused LM head. Returns dict(dlogits [M,V], dH [M,K] | None, dW [K,V] | None), all bf16."""
+    M, K = H.shape
+    V = W.shape[1]
+    if out is None:
+        out = {"dlogits": dlogits if dlogits is not None else torch.empty((M, V), dtype=torch.bfloat16, device=H.device),
+               "dH": torch.empty_like(H) if want_dH else None, "dW": torch.empty_like(W) if want_dW else None}
+    rc = lib().ppo_lmhead_bwd(_ptr(H, torch.bfloat16), _ptr(W, torch.bfloat16), M, K, V, _ptr(tokens, torch.int32),
+                              _ptr(mask, torch.uint8), _ptr(lse, torch.float32), _ptr(dlogprob, torch.float32),
+                              float(temperature), _ptr(out["dlogits"], torch.bfloat16), _ptr(out["dH"]),
+                              _ptr(out["dW"]), _ptr(workspace), _stream())
+    _check("ppo_lmhead_bwd", rc)
     return out

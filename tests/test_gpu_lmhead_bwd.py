@@ -1,0 +1,75 @@
+"""GPU parity of the LM-head backward (ppo_lmhead_bwd) against oracle/lmhead_bwd_oracle.py, through the C ABI.
+
+Tolerance (derived from the arithmetic): dlogits is stored in bf16 (relative rounding 2^-9, the logits behind it
+carry fp32-accumulation error ~1e-5); dH and dW contract that bf16 dlogits with fp32 accumulation and are rounded
+to bf16 once more, so |error| <= 2^-9 * sum|D||W| (worst case over the contraction) + 2^-9 |result|. The tests
+allow twice that plus a small absolute term."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import lmhead_bwd_oracle as B
+
+pytestmark = pytest.mark.gpu
+
+REL = 2.0 ** -8
+
+
+@pytest.fixture(scope="module")
+def P():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    import paper_2403_17031_b200 as pkg
+    from paper_2403_17031_b200 import build
+    build.build()
+    pkg.lib()
+    return pkg
+
+
+def _wide(t):
+    return t.detach().double().cpu().numpy()
+
+
+def _check(P, M, K, V, seed, with_mask=True, tau=0.7):
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    H = torch.randn((M, K), generator=g, device="cuda").to(torch.bfloat16)
+    W = (torch.randn((K, V), generator=g, device="cuda") * (2.0 / K ** 0.5)).to(torch.bfloat16)
+    tok = torch.randint(0, V, (M,), generator=g, device="cuda", dtype=torch.int32)
+    up = torch.randn((M,), generator=g, device="cuda")
+    up[0] = 0.0
+    mask = (torch.rand((M,), generator=g, device="cuda") < 0.8).to(torch.uint8) if with_mask else None
+    ws = P.new_workspace(P.lmhead_workspace_bytes(M, K, V))
+    _, _, lse = P.lmhead_logprob_entropy(H, W, tok, tau, ws, want_lse=True)
+    o = P.lmhead_bwd(H, W, tok, lse, up, tau, ws, mask=mask)
+    torch.cuda.synchronize()
+    assert P.last_device_status(ws) == 0
+    ref = B.lmhead_bwd(_wide(H), _wide(W), tok.cpu().numpy(), up.cpu().numpy().astype(np.float64), tau,
+                       mask=None if mask is None else mask.cpu().numpy())
+    D, dH, dW = _wide(o["dlogits"]), _wide(o["dH"]), _wide(o["dW"])
+    assert np.isfinite(D).all() and np.isfinite(dH).all() and np.isfinite(dW).all()
+    bad = np.abs(D - ref["D"]) > REL * np.abs(ref["D"]) + 1e-6
+    assert not bad.any(), "dlogits: %d off, worst %.3e" % (bad.sum(), np.abs(D - ref["D"])[bad].max())
+    if mask is not None:
+        assert not D[mask.cpu().numpy() == 0].any()
+    assert not D[0].any()
+    for name, got, want, scale in (("dH", dH, ref["dH"], ref["dH_abs"]), ("dW", dW, ref["dW"], ref["dW_abs"])):
+        bad = np.abs(got - want) > REL * scale + REL * np.abs(want) + 1e-6
+        assert not bad.any(), "%s: %d of %d off, worst %.3e (|want| max %.3e)" % (
+            name, bad.sum(), bad.size, np.abs(got - want)[bad].max(), np.abs(want).max())
+
+
+@pytest.mark.parametrize("M,K,V", [(128, 64, 256), (200, 128, 1000), (300, 192, 2056), (64, 64, 520),
+                                   (1000, 256, 4096)])
+def test_lmhead_bwd_small_shapes(P, M, K, V):
+    _check(P, M, K, V, seed=M + K + V)
+
+
+def test_lmhead_bwd_without_mask_and_partial_outputs(P):
+    _check(P, 256, 128, 512, seed=5, with_mask=False, tau=1.0)
+    M, K, V = 128, 64, 256
+    H = torch.randn((M, K), device="cuda").to(torch.bfloat16)
+    W = torch.randn((K, V), device="cuda").to(torch.bfloat16)
+    tok = torch.zeros(M, dtype=torch.int32, device="cuda")
+    ws = P.new_workspace(P.lmhead_workspace_bytes(M, K, V))
+    _, _, lse = P.lmhead_logprob_entropy(H, W, tok, 1.0, ws, want_lse=True)
+    o = P.lmhead_bwd(H, W, tok, lse, torch.ones(M, device="cuda"), 1.0, ws, want_dH=False, want_dW=False)
+    assert o["dH"] is None and o["dW"] is None and torch.isfinite(o["dlogits"].float()).all()
