@@ -73,3 +73,57 @@ def test_lmhead_bwd_without_mask_and_partial_outputs(P):
     _, _, lse = P.lmhead_logprob_entropy(H, W, tok, 1.0, ws, want_lse=True)
     o = P.lmhead_bwd(H, W, tok, lse, torch.ones(M, device="cuda"), 1.0, ws, want_dH=False, want_dW=False)
     assert o["dH"] is None and o["dW"] is None and torch.isfinite(o["dlogits"].float()).all()
+
+
+def test_lmhead_bwd_full_width_1024_rows(P):
+    """Full K and V of config 4 (many vocabulary tiles, 64 contraction blocks), rows cut to what the dense oracle
+    handles in seconds: every element of dlogits, dH and dW is compared."""
+    _check(P, 1024, 4096, 50304, seed=11)
+
+
+def test_lmhead_bwd_config4_full_size_sampled(P):
+    """Config 4 in the launch configuration the benchmark times. Row-local results (dlogits and dH rows) are checked
+    on sampled rows, which the oracle computes one by one; dW mixes all rows, so it is checked through properties:
+    every row of dW sums to ~0 over the vocabulary (each row of dlogits does), and a random projection
+    u^T dW equals (H u)^T D restricted to sampled vocabulary columns computed from the oracle-checked dlogits."""
+    from paper_2403_17031_b200.synthetic import CONFIGS, make_lmhead_batch
+    cfg = CONFIGS[4]
+    b = make_lmhead_batch(cfg, "cuda")
+    H, W, tok = b["H"], b["W"], b["tokens"]
+    M, K = H.shape
+    V = W.shape[1]
+    tau = cfg.hyper.temperature
+    g = torch.Generator(device="cuda").manual_seed(3)
+    up = torch.randn((M,), generator=g, device="cuda") / M
+    mask = (torch.rand((M,), generator=g, device="cuda") < 0.55).to(torch.uint8)
+    ws = P.new_workspace(P.lmhead_workspace_bytes(M, K, V))
+    _, _, lse = P.lmhead_logprob_entropy(H, W, tok, tau, ws, want_lse=True)
+    o = P.lmhead_bwd(H, W, tok, lse, up, tau, ws, mask=mask)
+    torch.cuda.synchronize()
+    assert P.last_device_status(ws) == 0
+    rng = np.random.default_rng(4)
+    real = np.flatnonzero(mask.cpu().numpy())
+    rows = np.unique(np.concatenate([[real[0], real[-1]], rng.choice(real, 10, replace=False),
+                                     np.flatnonzero(mask.cpu().numpy() == 0)[:2]]))
+    Wd = _wide(W)
+    idx = torch.from_numpy(rows).cuda()
+    ref = B.lmhead_bwd(_wide(H[idx]), Wd, tok[idx].cpu().numpy(), up[idx].cpu().numpy().astype(np.float64), tau,
+                       mask=mask[idx].cpu().numpy())
+    D, dH = _wide(o["dlogits"][idx]), _wide(o["dH"][idx])
+    bad = np.abs(D - ref["D"]) > REL * np.abs(ref["D"]) + 1e-9
+    assert not bad.any(), "dlogits rows: %d off, worst %.3e" % (bad.sum(), np.abs(D - ref["D"])[bad].max())
+    bad = np.abs(dH - ref["dH"]) > REL * ref["dH_abs"] + REL * np.abs(ref["dH"]) + 1e-9
+    assert not bad.any(), "dH rows: %d off, worst %.3e" % (bad.sum(), np.abs(dH - ref["dH"])[bad].max())
+    assert not _wide(o["dlogits"][mask == 0][:64]).any()
+    dW = o["dW"].float()
+    assert torch.isfinite(dW).all()
+    # rows of dW sum to zero up to the bf16 rounding of its 50304 entries
+    assert float((dW.double().sum(1).abs() / dW.double().abs().sum(1).clamp_min(1e-30)).max()) < 2.0 ** -8
+    # projection check against the dlogits that this call wrote (its rows were checked above): fp64 on the GPU
+    cols = torch.from_numpy(np.sort(rng.choice(V, 64, replace=False))).cuda()
+    u = torch.randn((K,), generator=g, device="cuda", dtype=torch.float64)
+    lhs = u @ dW.double()[:, cols]
+    Dc = o["dlogits"][:, cols].double()
+    rhs = (H.double() @ u) @ Dc
+    scale = (H.double().abs() @ u.abs()) @ Dc.abs()      # sum_k |u_k| (|H|^T |D|)[k, v]: the scale of dW's rounding
+    assert float(((lhs - rhs).abs() / scale.clamp_min(1e-30)).max()) < 2.0 ** -8
