@@ -432,6 +432,14 @@ def run_lmhead(args, cfg):
          "kl": bt(), "rew": bt(), "adv": bt(), "ret": bt(), "aw": bt(), "st": torch.empty(3, dtype=f32, device=dev)}
     loss_out = {"losses": torch.empty(8, dtype=f32, device=dev), "dlogprob": bt(), "dvalues": bt()}
     tok = b["responses"].reshape(-1)
+    bwd_out = None
+    if args.lm_backward:   # the step after the loss: gradient on the log-probs back to H and W
+        bwd_out = {"dlogits": torch.empty((M, V), dtype=torch.bfloat16, device=dev),
+                   "dH": torch.empty_like(b["H"]), "dW": torch.empty_like(b["W"])}
+
+    def backward():
+        binding.lmhead_bwd(b["H"], b["W"], tok, o["lse"].view(-1), loss_out["dlogprob"].view(-1), p.temperature, ws,
+                           mask=o["mask"].view(-1), out=bwd_out)
 
     def step(old):
         binding.truncate_and_score(b["responses"], b["scores"], p.eos_id, p.pad_id, p.no_eos_score,
@@ -445,6 +453,8 @@ def run_lmhead(args, cfg):
         binding.whiten(o["adv"], o["mask"], True, p.whiten_eps, workspace=ws, out=o["aw"], stats=o["st"])
         binding.loss_from_logprob(o["lp"], o["ent"], o["mask"], o["lp"] if old is None else old, o["aw"],
                                   b["values_new"], b["values"], o["ret"], p, ws, out=loss_out)
+        if bwd_out is not None:
+            backward()
     step(None)
     old = (o["lp"] + b["old_logprob_noise"]).contiguous()
     for _ in range(max(args.warmup, 3)):
@@ -453,6 +463,7 @@ def run_lmhead(args, cfg):
     K_steps = args.steps
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     lm_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K_steps)]
+    bw_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K_steps)]
     if distributed:
         dist.barrier()
     torch.cuda.synchronize()
@@ -472,6 +483,10 @@ def run_lmhead(args, cfg):
             binding.whiten(o["adv"], o["mask"], True, p.whiten_eps, workspace=ws, out=o["aw"], stats=o["st"])
             binding.loss_from_logprob(o["lp"], o["ent"], o["mask"], old, o["aw"], b["values_new"], b["values"],
                                       o["ret"], p, ws, out=loss_out)
+            if bwd_out is not None:
+                bw_ev[i][0].record()
+                backward()
+                bw_ev[i][1].record()
         ev1.record()
         torch.cuda.synchronize()
     total_ms = ev0.elapsed_time(ev1)
@@ -482,6 +497,7 @@ def run_lmhead(args, cfg):
     ms_per_step = total_ms / K_steps
     lm_ms = statistics.mean(a.elapsed_time(c) for a, c in lm_ev)
     status = binding.last_device_status(ws)
+    bwd_ms = statistics.mean(a.elapsed_time(c) for a, c in bw_ev) if bwd_out is not None else None
     flops = 2.0 * M * K * V
     tf = flops / (lm_ms * 1e-3) / 1e12
     # the kernel runs back to back for the whole timed region: compare with the sustained figure
@@ -495,12 +511,15 @@ def run_lmhead(args, cfg):
             "config": {"workload": "config4 %s" % cfg.name, "M_per_gpu": M, "K": K, "V": V,
                        "l2": "inputs larger than L2 (H %.0f MB + 2 x W %.0f MB per step)" %
                              (M * K * 2 / 1e6, K * V * 2 / 1e6),
-                       "lmhead_ms": lm_ms, "device_status": status},
+                       "lmhead_ms": lm_ms, "lmhead_bwd_ms": bwd_ms,
+                       "lmhead_bwd_tflops": None if bwd_ms is None else 3.0 * flops / (bwd_ms * 1e-3) / 1e12,
+                       "device_status": status},
             "roofline": {"bound": "tensor", "kernel": "lmhead_kernel (ppo_lmhead_logprob_entropy)", "achieved": tf,
                          "peak": peak, "peak_kind": kind + " (sustained)", "unit": "TFLOP/s", "frac": tf / peak,
                          "frac_of_burst": tf / burst, "traffic": None,
                          "timing": "CUDA events around the C-ABI call (GEMM kernel + finalize kernel)"},
-            "clocks": clk.summary(), "e2e": None, "cpu_baseline": None, "gpu_launches": 9 * K_steps,
+            "clocks": clk.summary(), "e2e": None, "cpu_baseline": None,
+            "gpu_launches": (9 + (3 if bwd_out is not None else 0)) * K_steps,
         }
         print(json.dumps(line), flush=True)
     if distributed:
@@ -625,6 +644,8 @@ def main():
     ap.add_argument("--config", type=int, default=1, choices=[1, 2, 3, 4, 5],
                     help="1-3: PPO path on stored logits; 4: fused LM head; 5: DPO step on preference pairs")
     ap.add_argument("--lm-rows", type=int, default=None, help="config 4: rows of H (default 512*53)")
+    ap.add_argument("--lm-backward", action="store_true",
+                    help="config 4: the step also runs the LM-head backward (dlogits, dH, dW)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--eager", action="store_true", help="launch every step call by call instead of replaying a CUDA graph")
     ap.add_argument("--whiten-rewards", action="store_true",
