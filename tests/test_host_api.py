@@ -132,6 +132,64 @@ def test_argument_errors_are_returned_before_any_launch(L):
     assert L.ppo_workspace_init(P(FAKE + 8), 1024, None) == -4
 
 
+def test_argument_errors_of_the_widened_entry_points(L):
+    """ppo_step, the preference losses, the log-prob backward and the LM-head forward/backward validate their
+    arguments on the host before anything is launched (no GPU needed to see the error codes)."""
+    from paper_2403_17031_b200 import binding as b
+    P = C.c_void_p
+    p = b.default_params()
+
+    def call(fn, args, **repl):
+        a = list(args)
+        for k, v in repl.items():
+            a[int(k[1:])] = v
+        return fn(*a)
+
+    lb = L.ppo_logprob_bwd
+    ok = [P(FAKE), b.PPO_BF16, 64, 1000, P(FAKE), P(FAKE), P(FAKE), 1.0, P(2 * FAKE), None, None, P(FAKE), None]
+    assert call(lb, ok, _1=9) == -5
+    assert call(lb, ok, _2=0) == -2 and call(lb, ok, _3=0) == -2
+    assert call(lb, ok, _6=None) == -1 and call(lb, ok, _8=None) == -1 and call(lb, ok, _11=None) == -1
+    assert call(lb, ok, _7=0.0) == -3
+    assert call(lb, ok, _8=P(FAKE)) == -3                 # in place is not supported
+    assert call(lb, ok, _11=P(FAKE + 64)) == -4
+
+    pw = L.ppo_pairwise_loss
+    okp = [P(FAKE), P(FAKE), 8, P(FAKE), None, None, None]
+    assert call(pw, okp, _2=0) == -2 and call(pw, okp, _0=None) == -1 and call(pw, okp, _3=None) == -1
+
+    dp = L.ppo_dpo_loss
+    okd = [P(FAKE)] * 6 + [8, 638, 0.05, P(FAKE), None, None, None, None, None]
+    assert call(dp, okd, _6=0) == -2 and call(dp, okd, _7=0) == -2
+    assert call(dp, okd, _3=None) == -1 and call(dp, okd, _9=None) == -1
+    assert call(dp, okd, _8=float("nan")) == -3
+
+    lm = L.ppo_lmhead_logprob_entropy
+    okm = [P(FAKE), P(FAKE), 128, 4096, 50304, P(FAKE), None, 0.7, P(FAKE), None, None, P(FAKE), None]
+    assert call(lm, okm, _3=4100) == -6                   # K must be a multiple of 64
+    assert call(lm, okm, _4=50305) == -6                  # V must be a multiple of 8
+    assert call(lm, okm, _7=-1.0) == -3 and call(lm, okm, _11=None) == -1 and call(lm, okm, _2=0) == 0
+    assert call(lm, okm, _0=P(FAKE + 2)) == -4
+
+    bw = L.ppo_lmhead_bwd
+    okb = [P(FAKE), P(FAKE), 128, 4096, 50304, P(FAKE), None, P(FAKE), P(FAKE), 0.7, P(FAKE), None, None, P(FAKE),
+           None]
+    assert call(bw, okb, _2=0) == -2
+    assert call(bw, okb, _3=4100) == -6 and call(bw, okb, _4=50306) == -6
+    assert call(bw, okb, _7=None) == -1 and call(bw, okb, _10=None) == -1 and call(bw, okb, _13=None) == -1
+    assert call(bw, okb, _9=0.0) == -3
+    assert call(bw, okb, _10=P(FAKE + 8)) == -4
+
+    io = b.PPOStepIO()
+    st = L.ppo_step
+    assert st(None, b.PPO_BF16, 4, 16, 1000, C.byref(p), None) == -1
+    assert st(C.byref(io), b.PPO_BF16, 4, 16, 1000, C.byref(p), None) == -1      # every required buffer is NULL
+    assert st(C.byref(io), b.PPO_BF16, 0, 16, 1000, C.byref(p), None) == -2
+    sh = L.ppo_step_host
+    assert sh(C.byref(io), None, b.PPO_BF16, 4, 16, 1000, C.byref(p), None) == -1
+    assert sh(C.byref(io), C.byref(io), 5, 4, 16, 1000, C.byref(p), None) == -5
+
+
 def test_binding_rejects_cpu_tensors():
     import torch
     from paper_2403_17031_b200 import binding as b
