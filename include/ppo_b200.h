@@ -58,6 +58,7 @@ extern "C" {
 #define PPO_DEV_BAD_TOKEN 1      /* a token id was outside [0, V): that row's outputs are NaN */
 #define PPO_DEV_EMPTY_MASK 2     /* mask selected no element: statistics / losses are 0 */
 #define PPO_DEV_TIMEOUT 4        /* a bounded wait inside a kernel gave up; outputs are invalid */
+#define PPO_DEV_BAD_ROW 8        /* ppo_sample_logprob_entropy: a row had a NaN / +inf or no finite logit: token -1 */
 
 /* indices into the losses[8] output of ppo_loss_fwd_bwd */
 enum { PPO_LOSS_PG = 0, PPO_LOSS_VF = 1, PPO_LOSS_TOTAL = 2, PPO_LOSS_APPROX_KL = 3,
@@ -235,6 +236,25 @@ int ppo_loss_from_logprob(const float *new_logprob, const float *entropy, int32_
                           const float *values_new, const float *values_old, const float *returns,
                           const ppo_params *p /* host */, float *losses, float *dlogprob,
                           float *dvalues, void *workspace, void *stream);
+
+/*
+ * Temperature sampling fused with step 1 (Table "PPO hyperparameters": temperature): draws one token
+ * per row from softmax(logits / temperature) and returns its log-prob, the row's entropy and
+ * log-sum-exp from the same single pass over HBM.  The draw is reproducible and defined as follows:
+ *   word(j)  = Philox4x32-10 with key = seed, counter = (j / 4, row, offset low, offset high), output j % 4
+ *   u_j      = (floor(word(j) / 2^9) + 1/2) * 2^-23            (an fp32 number in (0, 1))
+ *   token    = argmax_j [ logit_j * log2(e) / temperature - log2(-log2 u_j) ], ties to the lowest j
+ * Use a new `offset` for every call that must be independent of the previous ones with the same seed.
+ *   logits [rows, V] dtype, row pitch row_stride >= V elements
+ *   tokens_out [rows] i32; logprob, entropy, lse nullable [rows] f32 (as in ppo_logprob_entropy)
+ *   workspace  nullable (status word: PPO_DEV_BAD_ROW when a row has a NaN, a +inf or no finite logit;
+ *              that row gets token -1 and NaN outputs)
+ * The kernel evaluates the rule in fp32 with hardware exp2/log2 approximations: where two candidates'
+ * scores differ by less than ~1e-5 it may pick the other one than an exact evaluation would.
+ */
+int ppo_sample_logprob_entropy(const void *logits, int dtype, int64_t rows, int64_t V, int64_t row_stride,
+                               float temperature, uint64_t seed, uint64_t offset, int32_t *tokens_out,
+                               float *logprob, float *entropy, float *lse, void *workspace, void *stream);
 
 /*
  * Chain rule from token log-probs back to the logits (the backward half of ppo_logprob_entropy;

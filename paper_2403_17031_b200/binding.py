@@ -91,6 +91,9 @@ _SIGS = {
                            C.c_void_p]),
     "ppo_step_host": (C.c_int, [C.POINTER(PPOStepIO), C.POINTER(PPOStepIO), C.c_int, C.c_int32, C.c_int32, C.c_int64,
                                 C.POINTER(PPOParams), C.c_void_p]),
+    "ppo_sample_logprob_entropy": (C.c_int, [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_float,
+                                             C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                             C.c_void_p, C.c_void_p]),
     "ppo_lmhead_bwd": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
                                  C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                  C.c_void_p]),
@@ -439,3 +442,29 @@ def lmhead_bwd(H, W, tokens, lse, dlogprob, temperature: float, workspace, mask=
                               _ptr(out["dW"]), _ptr(workspace), _stream())
     _check("ppo_lmhead_bwd", rc)
     return out
+
+
+def sample_logprob_entropy(logits: torch.Tensor, temperature: float, seed: int, offset: int = 0, workspace=None,
+                           want_entropy: bool = True, want_lse: bool = False, out=None):
+    """Draw one token per row of logits [..., V] at the given temperature; returns (tokens, logprob, entropy, lse)."""
+    V = logits.shape[-1]
+    rows = logits.numel() // V
+    lg2 = logits.reshape(rows, V) if logits.is_contiguous() else logits
+    if lg2.dim() != 2 or lg2.stride(1) != 1:
+        raise TypeError("logits rows must be contiguous")
+    stride = lg2.stride(0) if rows > 1 else V
+    shape = logits.shape[:-1]
+    if out is None:
+        dev = logits.device
+        out = (torch.empty(shape, dtype=torch.int32, device=dev), torch.empty(shape, dtype=torch.float32, device=dev),
+               torch.empty(shape, dtype=torch.float32, device=dev) if want_entropy else None,
+               torch.empty(shape, dtype=torch.float32, device=dev) if want_lse else None)
+    tok, lp, ent, lse = out
+    if not lg2.is_cuda:
+        raise TypeError("logits must be a CUDA tensor")
+    rc = lib().ppo_sample_logprob_entropy(C.c_void_p(lg2.data_ptr()), _logits_dtype(lg2), rows, V, stride,
+                                          float(temperature), int(seed) & (2 ** 64 - 1), int(offset) & (2 ** 64 - 1),
+                                          _ptr(tok, torch.int32), _ptr(lp, torch.float32), _ptr(ent, torch.float32),
+                                          _ptr(lse, torch.float32), _ptr(workspace), _stream())
+    _check("ppo_sample_logprob_entropy", rc)
+    return tok, lp, ent, lse

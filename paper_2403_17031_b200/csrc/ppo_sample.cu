@@ -1,0 +1,240 @@
+// Temperature sampling fused into the log-prob / entropy pass (the step before step 1: Table "PPO
+// hyperparameters", temperature 0.7): one kernel draws the token of every row from
+// softmax(logits / tau) and returns its log-prob, the row's entropy and log-sum-exp, so the logits are
+// streamed from HBM once for both.
+//
+// The draw is defined so that it can be reproduced on a CPU token by token:
+//   * Philox4x32-10 (counter-based; Salmon et al., SC'11): key = seed, counter = (j / 4, row, offset low,
+//     offset high), word j % 4 belongs to element j of the row;
+//   * u_j = (floor(word / 2^9) + 1/2) * 2^-23, an fp32 number strictly inside (0, 1);
+//   * the token is the j that minimises E_j / 2^(y_j) with E_j = -log2(u_j) (an exponential race; the
+//     same as the Gumbel-max rule argmax_j [y_j - log2(-log2 u_j)]), y_j = logit_j * log2(e) / tau.
+//     Candidates are compared by cross-multiplication (E_j * e_best < E_best * e_j with e = 2^(y - max)),
+//     so the race costs no division and reuses the exponential that the softmax sums need anyway;
+//     exact ties go to the lowest index.
+// One block per row, two passes over the row: the maximum (second pass then needs no rescaling; the row
+// is re-read through L2), then sums and race. The generator dominates: ~10 integer instructions per
+// logit next to ~12 for everything else, so this kernel is bound by instruction issue, not by HBM.
+#include "ppo_rows.cuh"
+
+namespace ppo {
+
+constexpr uint32_t kPhiloxM0 = 0xD2511F53u, kPhiloxM1 = 0xCD9E8D57u;
+constexpr uint32_t kPhiloxW0 = 0x9E3779B9u, kPhiloxW1 = 0xBB67AE85u;
+
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                              uint32_t k1, uint32_t (&o)[4])
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(kPhiloxM0, c0), lo0 = kPhiloxM0 * c0;
+        const uint32_t hi1 = __umulhi(kPhiloxM1, c2), lo1 = kPhiloxM1 * c2;
+        c0 = hi1 ^ c1 ^ k0;
+        c1 = lo1;
+        c2 = hi0 ^ c3 ^ k1;
+        c3 = lo0;
+        k0 += kPhiloxW0;
+        k1 += kPhiloxW1;
+    }
+    o[0] = c0; o[1] = c1; o[2] = c2; o[3] = c3;
+}
+
+// 32-bit word -> E = -log2(u), u = (word >> 9 + 1/2) * 2^-23 (built in the mantissa: no int->float convert)
+__device__ __forceinline__ float exponential_variate(uint32_t w)
+{
+    const float u = __uint_as_float(0x3f800000u | (w >> 9)) - 0.99999994f;   // 1 + k 2^-23 - (1 - 2^-24): exact
+    float l;
+    asm("lg2.approx.f32 %0, %1;" : "=f"(l) : "f"(u));
+    return -l;
+}
+
+struct Race {
+    float e, E, t;   // best candidate so far: 2^(y - max), its exponential variate, y - max
+    int j;
+    __device__ __forceinline__ void init() { e = 0.f; E = 1.f; t = 0.f; j = 0x7fffffff; }
+    // element with a larger index than everything offered to this thread before
+    __device__ __forceinline__ void offer(float e1, float E1, float t1, int j1)
+    {
+        if (E1 * e < E * e1) { e = e1; E = E1; t = t1; j = j1; }
+    }
+    __device__ __forceinline__ void merge(const Race &o)
+    {
+        const float l = o.E * e, r = E * o.e;
+        if (l < r || (l == r && o.j < j)) *this = o;
+    }
+};
+
+struct SampleArgs {
+    const void *logits;
+    int V;
+    int64_t row_stride;
+    float c;
+    uint32_t k0, k1, off_lo, off_hi;
+    int32_t *tokens;
+    float *logprob, *entropy, *lse;
+    int *status;
+};
+
+template <typename T, bool VECTOR, int THREADS>
+__global__ void __launch_bounds__(THREADS)
+sample_kernel(const SampleArgs a)
+{
+    constexpr int N = Pack<T>::N;
+    __shared__ float red[3 * 32];
+    __shared__ int redj[32];
+    const int64_t row = blockIdx.x;
+    const T *src = reinterpret_cast<const T *>(a.logits) + row * a.row_stride;
+    const int V = a.V;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int WARPS = THREADS / 32;
+
+    // ---- pass 1: the row maximum (NaN-blind here; a NaN shows up in the sums of pass 2)
+    float mx = kNegBig;
+    if (VECTOR) {
+        const uint4 *src4 = reinterpret_cast<const uint4 *>(src);
+        const int nvec = V / N;
+        for (int i = threadIdx.x; i < nvec; i += THREADS) {
+            float x[N], xm;
+            Pack<T>::unpack(src4[i], x, xm);
+            mx = fmaxf(mx, xm);
+        }
+    } else {
+        for (int j = threadIdx.x; j < V; j += THREADS) mx = fmaxf(mx, fmaxf(Pack<T>::load1(src + j), kNegBig));
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+    if (lane == 0) red[warp] = mx;
+    __syncthreads();
+    mx = red[lane < WARPS ? lane : 0];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+    __syncthreads();
+    const float m = mx * a.c, nm = -m;
+
+    // ---- pass 2: softmax sums and the race
+    float s0 = 0.f, s1 = 0.f, u0 = 0.f, u1 = 0.f;
+    Race best;
+    best.init();
+    const uint32_t rlo = (uint32_t)row;
+    if (VECTOR) {
+        const uint4 *src4 = reinterpret_cast<const uint4 *>(src);
+        const int nvec = V / N;
+        for (int i = threadIdx.x; i < nvec; i += THREADS) {
+            float x[N];
+            Pack<T>::unpack_clamped(src4[i], x);
+#pragma unroll
+            for (int h = 0; h < N / 4; ++h) {
+                uint32_t w[4];
+                philox4x32_10((uint32_t)(i * (N / 4) + h), rlo, a.off_lo, a.off_hi, a.k0, a.k1, w);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float t = fmaf(x[h * 4 + q], a.c, nm);
+                    const float e = ex2(t);
+                    if (q & 1) { s1 += e; u1 = fmaf(e, t, u1); } else { s0 += e; u0 = fmaf(e, t, u0); }
+                    best.offer(e, exponential_variate(w[q]), t, i * N + h * 4 + q);
+                }
+            }
+        }
+    } else {
+        for (int j = threadIdx.x; j < V; j += THREADS) {
+            float x = Pack<T>::load1(src + j);
+            x = (x != x) ? x : fmaxf(x, kNegBig);
+            uint32_t w[4];
+            philox4x32_10((uint32_t)(j >> 2), rlo, a.off_lo, a.off_hi, a.k0, a.k1, w);
+            const float t = fmaf(x, a.c, nm);
+            const float e = ex2(t);
+            s0 += e;
+            u0 = fmaf(e, t, u0);
+            best.offer(e, exponential_variate(w[j & 3]), t, j);
+        }
+    }
+    // ---- block merge: sums by addition, race by comparison (fixed order: lanes, then warps)
+    float s = s0 + s1, u = u0 + u1;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        s += __shfl_xor_sync(0xffffffffu, s, off);
+        u += __shfl_xor_sync(0xffffffffu, u, off);
+        Race o;
+        o.e = __shfl_xor_sync(0xffffffffu, best.e, off);
+        o.E = __shfl_xor_sync(0xffffffffu, best.E, off);
+        o.t = __shfl_xor_sync(0xffffffffu, best.t, off);
+        o.j = __shfl_xor_sync(0xffffffffu, best.j, off);
+        best.merge(o);
+    }
+    __shared__ float rs[32], ru[32];
+    if (lane == 0) {
+        rs[warp] = s; ru[warp] = u;
+        red[warp] = best.e; red[32 + warp] = best.E; red[64 + warp] = best.t; redj[warp] = best.j;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        s = 0.f; u = 0.f;
+        best.init();
+        for (int w = 0; w < WARPS; ++w) {
+            s += rs[w]; u += ru[w];
+            Race o;
+            o.e = red[w]; o.E = red[32 + w]; o.t = red[64 + w]; o.j = redj[w];
+            best.merge(o);
+        }
+        const float l2s = log2f(s);
+        float lp = (best.t - l2s) * kLn2;
+        float H = (l2s - u / s) * kLn2;
+        float L = (m + l2s) * kLn2;
+        int tok = best.j;
+        // no finite maximum, a NaN or +inf in the row, or no candidate: nothing is drawn
+        if (!(mx > -1.0e29f) || !(s == s) || !(fabsf(u) < 3.0e38f) || tok == 0x7fffffff) {
+            tok = -1;
+            lp = H = L = __int_as_float(0x7fc00000);
+            if (a.status) atomicOr(a.status, PPO_DEV_BAD_ROW);
+        }
+        a.tokens[row] = tok;
+        if (a.logprob) a.logprob[row] = lp;
+        if (a.entropy) a.entropy[row] = H;
+        if (a.lse) a.lse[row] = L;
+    }
+}
+
+}   // namespace ppo
+
+using namespace ppo;
+
+extern "C" int ppo_sample_logprob_entropy(const void *logits, int dtype, int64_t rows, int64_t V, int64_t row_stride,
+                                          float temperature, uint64_t seed, uint64_t offset, int32_t *tokens_out,
+                                          float *logprob, float *entropy, float *lse, void *workspace, void *stream)
+{
+    if (dtype != PPO_F32 && dtype != PPO_BF16) return PPO_ERR_DTYPE;
+    if (rows < 0 || rows >= ((int64_t)1 << 31) || V <= 0 || V >= ((int64_t)1 << 31) || row_stride < V)
+        return PPO_ERR_SHAPE;
+    if (!(temperature > 0.f) || !finite_f(temperature)) return PPO_ERR_PARAM;
+    if (rows == 0) return PPO_OK;
+    if (!logits || !tokens_out) return PPO_ERR_NULL;
+    const size_t es = dtype == PPO_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(logits) % es) return PPO_ERR_ALIGN;
+    SampleArgs a;
+    a.logits = logits;
+    a.V = (int)V;
+    a.row_stride = row_stride;
+    a.c = kLog2e / temperature;
+    a.k0 = (uint32_t)seed;
+    a.k1 = (uint32_t)(seed >> 32);
+    a.off_lo = (uint32_t)offset;
+    a.off_hi = (uint32_t)(offset >> 32);
+    a.tokens = tokens_out;
+    a.logprob = logprob;
+    a.entropy = entropy;
+    a.lse = lse;
+    a.status = workspace ? &ws_header(workspace)->status : nullptr;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    constexpr int THREADS = 256;
+    const int n = dtype == PPO_F32 ? 4 : 8;
+    const bool vec = aligned16(logits) && (row_stride * es) % 16 == 0 && V % n == 0;
+    const unsigned grid = (unsigned)rows;
+    if (dtype == PPO_F32) {
+        if (vec) sample_kernel<float, true, THREADS><<<grid, THREADS, 0, s>>>(a);
+        else sample_kernel<float, false, THREADS><<<grid, THREADS, 0, s>>>(a);
+    } else {
+        if (vec) sample_kernel<__nv_bfloat16, true, THREADS><<<grid, THREADS, 0, s>>>(a);
+        else sample_kernel<__nv_bfloat16, false, THREADS><<<grid, THREADS, 0, s>>>(a);
+    }
+    return launch_status();
+}

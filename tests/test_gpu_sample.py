@@ -1,0 +1,95 @@
+"""GPU parity of ppo_sample_logprob_entropy against oracle/sample_oracle.py (Philox4x32-10 + Gumbel-max in base 2).
+
+The token is an integer decided by floating point. The kernel evaluates the rule in fp32 with hardware exp2 / log2
+approximations (relative error ~2^-22 on scores of magnitude <= ~60), the oracle in fp64; so the comparison is:
+identical token wherever the oracle's best and second-best scores are more than GAP apart, and otherwise a token
+whose score is within GAP of the best."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import sample_oracle as S
+from parity import TOL_LOGPROB, assert_abs, host_logits, npy
+
+pytestmark = pytest.mark.gpu
+GAP = 1e-4
+
+
+@pytest.fixture(scope="module")
+def P():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    import paper_2403_17031_b200 as pkg
+    from paper_2403_17031_b200 import build
+    build.build()
+    pkg.lib()
+    return pkg
+
+
+def _compare(P, oracle, x, tau, seed, offset=0):
+    rows, V = x.shape
+    ws = P.new_workspace(P.workspace_bytes(rows, 1, V))
+    tok, lp, ent, lse = P.sample_logprob_entropy(x, tau, seed, offset, workspace=ws, want_lse=True)
+    torch.cuda.synchronize()
+    assert P.last_device_status(ws) == 0
+    tok = npy(tok).astype(np.int64)
+    want, keys = S.sample(x.detach().double().cpu().numpy(), tau, seed, offset)
+    top2 = np.partition(keys, -2, axis=1)[:, -2:]
+    clear = top2[:, 1] - top2[:, 0] > GAP
+    assert clear.mean() > 0.98
+    assert np.array_equal(tok[clear], want[clear]), "%d clear rows differ" % (tok[clear] != want[clear]).sum()
+    chosen = keys[np.arange(rows), tok]
+    assert (keys.max(axis=1) - chosen <= GAP).all()
+    # log-prob of the token that was drawn, entropy and lse: the forward oracle
+    o_lp, o_ent, o_lse = oracle.logprob_entropy(host_logits(x), tok.astype(np.int32), tau)
+    assert_abs(npy(lp), o_lp, TOL_LOGPROB, "logprob of the drawn token")
+    assert_abs(npy(ent), o_ent, TOL_LOGPROB, "entropy")
+    assert_abs(npy(lse), o_lse, TOL_LOGPROB, "lse")
+    return tok
+
+
+@pytest.mark.parametrize("dtype,rows,V", [(torch.float32, 64, 1000), (torch.float32, 33, 1001), (torch.bfloat16, 128, 2048),
+                                          (torch.bfloat16, 40, 50304), (torch.bfloat16, 17, 1004), (torch.float32, 12, 50304)])
+def test_sample_matches_oracle(P, oracle, dtype, rows, V):
+    g = torch.Generator(device="cuda").manual_seed(rows + V)
+    x = (2.0 * torch.randn((rows, V), generator=g, device="cuda")).to(dtype)
+    _compare(P, oracle, x, 0.7, seed=0x1234567890abcdef, offset=3)
+
+
+def test_strided_rows_seed_and_offset(P, oracle):
+    g = torch.Generator(device="cuda").manual_seed(1)
+    big = torch.randn((50, 1536), generator=g, device="cuda")
+    x = big[:, :1000]                                     # row pitch 1536 > V
+    t0 = _compare(P, oracle, x, 1.0, seed=11)
+    t1 = _compare(P, oracle, x, 1.0, seed=12)
+    t2 = _compare(P, oracle, x, 1.0, seed=11, offset=2 ** 33 + 5)
+    assert (t0 != t1).mean() > 0.5 and (t0 != t2).mean() > 0.5
+    again, _, _, _ = P.sample_logprob_entropy(x, 1.0, 11)
+    assert np.array_equal(npy(again), t0)                 # same seed and offset: same draw
+
+
+def test_distribution_of_draws(P):
+    """20000 rows with the same logits: token frequencies follow softmax(logits / tau) (chi-square)."""
+    rng = np.random.default_rng(3)
+    V, n, tau = 16, 20000, 0.7
+    row = (rng.normal(size=V) * 1.5).astype(np.float32)
+    x = torch.from_numpy(np.tile(row, (n, 1))).cuda()
+    tok, _, _, _ = P.sample_logprob_entropy(x, tau, seed=2024)
+    p = np.exp(row.astype(np.float64) / tau)
+    p /= p.sum()
+    counts = np.bincount(npy(tok), minlength=V)
+    assert ((counts - n * p) ** 2 / (n * p)).sum() < 50.0          # 15 degrees of freedom: P(> 50) ~ 1e-5
+
+
+def test_minus_infinity_never_drawn_and_bad_rows(P):
+    V = 512
+    x = torch.randn((6, V), device="cuda")
+    x[:, ::2] = float("-inf")
+    x[3, 7] = float("nan")
+    x[4, :] = float("-inf")
+    x[5, 9] = float("inf")
+    ws = P.new_workspace(P.workspace_bytes(6, 1, V))
+    tok, lp, ent, _ = P.sample_logprob_entropy(x, 0.7, 5, workspace=ws)
+    tok = npy(tok)
+    assert (tok[:3] % 2 == 1).all() and np.isfinite(npy(lp)[:3]).all() and np.isfinite(npy(ent)[:3]).all()
+    assert (tok[3:] == -1).all() and np.isnan(npy(lp)[3:]).all()
+    assert P.last_device_status(ws) == 8
