@@ -636,13 +636,95 @@ def run_dpo(args):
         dist.destroy_process_group()
 
 
+def run_sample(args):
+    """Config 6: temperature sampling fused with the log-prob / entropy pass on the config-1 logits."""
+    rank, world, local = _dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    distributed = world > 1
+    if distributed:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2403_17031_b200 import binding, build
+    from paper_2403_17031_b200.synthetic import CONFIGS, make_batch
+    if rank == 0:
+        build.build()
+    if distributed:
+        dist.barrier()
+    binding.lib()
+    cfg = CONFIGS[1]
+    x = make_batch(cfg, dev, seed=cfg.seed + 1000 * rank, with_ref=False)["policy_logits"]
+    B, T, V = x.shape
+    ws = binding.new_workspace(binding.workspace_bytes(B, T, V), dev)
+    out = binding.sample_logprob_entropy(x, cfg.hyper.temperature, 20240317, 0, workspace=ws)
+    for i in range(max(args.warmup, 3)):
+        binding.sample_logprob_entropy(x, cfg.hyper.temperature, 20240317, i + 1, workspace=ws, out=out)
+    torch.cuda.synchronize()
+    K = args.steps
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if distributed:
+        dist.barrier()
+    torch.cuda.synchronize()
+    with ClockSampler(local) as clk:
+        ev0.record()
+        for i in range(K):
+            binding.sample_logprob_entropy(x, cfg.hyper.temperature, 20240317, 100 + i, workspace=ws, out=out)
+        ev1.record()
+        torch.cuda.synchronize()
+    total_ms = ev0.elapsed_time(ev1)
+    if distributed:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms = total_ms / K
+    logits = B * T * V
+    # instructions the method needs per logit (stated in DESIGN.md): Philox4x32-10 10, uniform 2, log2 1, widen 1,
+    # scale 1, exp2 1, two sums 2, race 3, maximum pass 2
+    ops_per_logit = 23
+    clocks = clk.summary()
+    sm_ghz = (clocks.get("sm_max_mhz") or 1965) / 1e3
+    peak = 148 * 4 * 32 * sm_ghz          # Ginstr/s: one warp instruction per scheduler and clock
+    achieved = ops_per_logit * logits / (ms * 1e-3) / 1e9
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import sample_oracle as S
+        n = 48
+        xs = x.reshape(-1, V)[:n].double().cpu().numpy()
+        t0 = time.perf_counter()
+        S.sample(xs, cfg.hyper.temperature, 20240317, 0)
+        dt_s = time.perf_counter() - t0
+        cpu = {"value": n / dt_s, "unit": "tokens/s", "cores": 1, "kind": "oracle",
+               "sample": "%d rows of V=%d (numpy Philox + Gumbel-max, draw only), %.1f s" % (n, V, dt_s)}
+    if rank == 0:
+        line = {
+            "metric": "response tokens/s", "value": B * T * world / (ms * 1e-3), "unit": "tokens/s", "n_gpus": world,
+            "steps": K, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "config6 fused sampling + log-prob on config1 logits", "B_per_gpu": B, "T": T, "V": V,
+                       "logits_dtype": cfg.dtype, "l2": "inputs larger than L2 (%.0f MB of logits per step)" %
+                       (logits * 2 / 1e6), "hbm_gbs": logits * 2 / (ms * 1e-3) / 1e9,
+                       "device_status": binding.last_device_status(ws)},
+            "roofline": {"bound": "alu", "kernel": "sample_kernel (ppo_sample_logprob_entropy)", "achieved": achieved,
+                         "peak": peak, "peak_kind": "derived: 148 SMs x 4 schedulers x 32 lanes x max SM clock",
+                         "unit": "Ginstr/s", "frac": achieved / peak, "traffic": None,
+                         "ops_per_logit": ops_per_logit},
+            "clocks": clocks, "e2e": None, "cpu_baseline": cpu, "gpu_launches": K,
+        }
+        print(json.dumps(line), flush=True)
+    if distributed:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--config", type=int, default=1, choices=[1, 2, 3, 4, 5],
-                    help="1-3: PPO path on stored logits; 4: fused LM head; 5: DPO step on preference pairs")
+    ap.add_argument("--config", type=int, default=1, choices=[1, 2, 3, 4, 5, 6],
+                    help="1-3: PPO path on stored logits; 4: fused LM head; 5: DPO step on preference pairs; "
+                         "6: fused sampling + log-prob")
     ap.add_argument("--lm-rows", type=int, default=None, help="config 4: rows of H (default 512*53)")
     ap.add_argument("--lm-backward", action="store_true",
                     help="config 4: the step also runs the LM-head backward (dlogits, dH, dW)")
@@ -661,7 +743,10 @@ def main():
     if args.config == 5 and args.impl != "reference":
         run_dpo(args)
         return
-    cfg = CONFIGS[1 if args.config == 5 else args.config]
+    if args.config == 6 and args.impl != "reference":
+        run_sample(args)
+        return
+    cfg = CONFIGS[1 if args.config in (5, 6) else args.config]
     if args.impl == "reference":
         run_reference(args, CONFIGS[1] if args.config == 4 else cfg)
     elif args.config == 4:

@@ -22,19 +22,29 @@ namespace ppo {
 constexpr uint32_t kPhiloxM0 = 0xD2511F53u, kPhiloxM1 = 0xCD9E8D57u;
 constexpr uint32_t kPhiloxW0 = 0x9E3779B9u, kPhiloxW1 = 0xBB67AE85u;
 
-__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
-                                              uint32_t k1, uint32_t (&o)[4])
+// the ten round keys depend on the seed only: computed once per thread (uniform across the grid)
+struct PhiloxKeys {
+    uint32_t k0[10], k1[10];
+    __device__ __forceinline__ void init(uint32_t a, uint32_t b)
+    {
+#pragma unroll
+        for (int r = 0; r < 10; ++r) {
+            k0[r] = a + (uint32_t)r * kPhiloxW0;
+            k1[r] = b + (uint32_t)r * kPhiloxW1;
+        }
+    }
+};
+
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, const PhiloxKeys &k,
+                                              uint32_t (&o)[4])
 {
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
-        const uint32_t hi0 = __umulhi(kPhiloxM0, c0), lo0 = kPhiloxM0 * c0;
-        const uint32_t hi1 = __umulhi(kPhiloxM1, c2), lo1 = kPhiloxM1 * c2;
-        c0 = hi1 ^ c1 ^ k0;
-        c1 = lo1;
-        c2 = hi0 ^ c3 ^ k1;
-        c3 = lo0;
-        k0 += kPhiloxW0;
-        k1 += kPhiloxW1;
+        const uint64_t p0 = (uint64_t)kPhiloxM0 * c0, p1 = (uint64_t)kPhiloxM1 * c2;   // one wide multiply each
+        c0 = (uint32_t)(p1 >> 32) ^ c1 ^ k.k0[r];
+        c1 = (uint32_t)p1;
+        c2 = (uint32_t)(p0 >> 32) ^ c3 ^ k.k1[r];
+        c3 = (uint32_t)p0;
     }
     o[0] = c0; o[1] = c1; o[2] = c2; o[3] = c3;
 }
@@ -116,6 +126,8 @@ sample_kernel(const SampleArgs a)
     Race best;
     best.init();
     const uint32_t rlo = (uint32_t)row;
+    PhiloxKeys keys;
+    keys.init(a.k0, a.k1);
     if (VECTOR) {
         const uint4 *src4 = reinterpret_cast<const uint4 *>(src);
         const int nvec = V / N;
@@ -125,7 +137,7 @@ sample_kernel(const SampleArgs a)
 #pragma unroll
             for (int h = 0; h < N / 4; ++h) {
                 uint32_t w[4];
-                philox4x32_10((uint32_t)(i * (N / 4) + h), rlo, a.off_lo, a.off_hi, a.k0, a.k1, w);
+                philox4x32_10((uint32_t)(i * (N / 4) + h), rlo, a.off_lo, a.off_hi, keys, w);
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     const float t = fmaf(x[h * 4 + q], a.c, nm);
@@ -140,7 +152,7 @@ sample_kernel(const SampleArgs a)
             float x = Pack<T>::load1(src + j);
             x = (x != x) ? x : fmaxf(x, kNegBig);
             uint32_t w[4];
-            philox4x32_10((uint32_t)(j >> 2), rlo, a.off_lo, a.off_hi, a.k0, a.k1, w);
+            philox4x32_10((uint32_t)(j >> 2), rlo, a.off_lo, a.off_hi, keys, w);
             const float t = fmaf(x, a.c, nm);
             const float e = ex2(t);
             s0 += e;
