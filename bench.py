@@ -681,8 +681,8 @@ def run_sample(args):
     ms = total_ms / K
     logits = B * T * V
     # instructions the method needs per logit (stated in the design doc): Philox4x32-10 10, uniform 2, log2 1, widen 1,
-    # scale 1, exp2 1, two sums 2, race 3, maximum pass 2
-    ops_per_logit = 23
+    # scale 1, exp2 1, two sums 2, race 3
+    ops_per_logit = 21
     clocks = clk.summary()
     sm_ghz = (clocks.get("sm_max_mhz") or 1965) / 1e3
     peak = 148 * 4 * 32 * sm_ghz          # Ginstr/s: one warp instruction per scheduler and clock

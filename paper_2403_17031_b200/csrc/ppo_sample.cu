@@ -12,8 +12,9 @@
 //     Candidates are compared by cross-multiplication (E_j * e_best < E_best * e_j with e = 2^(y - max)),
 //     so the race costs no division and reuses the exponential that the softmax sums need anyway;
 //     exact ties go to the lowest index.
-// One block per row, two passes over the row: the maximum (second pass then needs no rescaling; the row
-// is re-read through L2), then sums and race. The generator dominates: ~10 integer instructions per
+// One block per row, one pass: the exponentials are taken relative to the maximum of the row's first pack
+// (any reference serves the race and the sums); a row whose sums overflow that way, or that holds a NaN or
+// an infinity, is repeated with its exact maximum. The generator dominates: ~10 integer instructions per
 // logit next to ~12 for everything else, so this kernel is bound by instruction issue, not by HBM.
 #include "ppo_rows.cuh"
 
@@ -49,28 +50,30 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
     o[0] = c0; o[1] = c1; o[2] = c2; o[3] = c3;
 }
 
-// 32-bit word -> E = -log2(u), u = (word >> 9 + 1/2) * 2^-23 (built in the mantissa: no int->float convert)
-__device__ __forceinline__ float exponential_variate(uint32_t w)
+// 32-bit word -> log2(u) < 0, u = (word >> 9 + 1/2) * 2^-23 (built in the mantissa: no int->float convert).
+// The exponential variate of the race is E = -log2(u); the sign stays folded into the comparisons.
+__device__ __forceinline__ float log2_uniform(uint32_t w)
 {
     const float u = __uint_as_float(0x3f800000u | (w >> 9)) - 0.99999994f;   // 1 + k 2^-23 - (1 - 2^-24): exact
     float l;
     asm("lg2.approx.f32 %0, %1;" : "=f"(l) : "f"(u));
-    return -l;
+    return l;
 }
 
 struct Race {
-    float e, E, t;   // best candidate so far: 2^(y - max), its exponential variate, y - max
+    float e, L;   // best candidate so far: e = 2^(y - reference), L = log2(u) = -E
     int j;
-    __device__ __forceinline__ void init() { e = 0.f; E = 1.f; t = 0.f; j = 0x7fffffff; }
-    // element with a larger index than everything offered to this thread before
-    __device__ __forceinline__ void offer(float e1, float E1, float t1, int j1)
+    __device__ __forceinline__ void init() { e = 0.f; L = -1.f; j = 0x7fffffff; }
+    // candidate (e1, L1) beats the best when E1 / e1 < E / e, i.e. L1 * e > L * e1 (both sides <= 0);
+    // offered in increasing index order, so a strict comparison leaves ties with the lowest index
+    __device__ __forceinline__ void offer(float e1, float L1, int j1)
     {
-        if (E1 * e < E * e1) { e = e1; E = E1; t = t1; j = j1; }
+        if (L1 * e > L * e1) { e = e1; L = L1; j = j1; }
     }
     __device__ __forceinline__ void merge(const Race &o)
     {
-        const float l = o.E * e, r = E * o.e;
-        if (l < r || (l == r && o.j < j)) *this = o;
+        const float l = o.L * e, r = L * o.e;
+        if (l > r || (l == r && o.j < j)) *this = o;
     }
 };
 
@@ -85,49 +88,26 @@ struct SampleArgs {
     int *status;
 };
 
+struct SampleSmem {
+    float rs[32], ru[32], re[32], rl[32];
+    int rj[32];
+    float bs, bu;
+    int redo;
+};
+
+// softmax sums and race of one row relative to the reference m (base-2 units); result in thread 0
 template <typename T, bool VECTOR, int THREADS>
-__global__ void __launch_bounds__(THREADS)
-sample_kernel(const SampleArgs a)
+__device__ __forceinline__ void sums_and_race(const T *src, int V, float c, float m, uint32_t row, const SampleArgs &a,
+                                              const PhiloxKeys &keys, SampleSmem &sm, float &s_out, float &u_out,
+                                              Race &best_out)
 {
     constexpr int N = Pack<T>::N;
-    __shared__ float red[3 * 32];
-    __shared__ int redj[32];
-    const int64_t row = blockIdx.x;
-    const T *src = reinterpret_cast<const T *>(a.logits) + row * a.row_stride;
-    const int V = a.V;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int WARPS = THREADS / 32;
-
-    // ---- pass 1: the row maximum (NaN-blind here; a NaN shows up in the sums of pass 2)
-    float mx = kNegBig;
-    if (VECTOR) {
-        const uint4 *src4 = reinterpret_cast<const uint4 *>(src);
-        const int nvec = V / N;
-        for (int i = threadIdx.x; i < nvec; i += THREADS) {
-            float x[N], xm;
-            Pack<T>::unpack(src4[i], x, xm);
-            mx = fmaxf(mx, xm);
-        }
-    } else {
-        for (int j = threadIdx.x; j < V; j += THREADS) mx = fmaxf(mx, fmaxf(Pack<T>::load1(src + j), kNegBig));
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-    if (lane == 0) red[warp] = mx;
-    __syncthreads();
-    mx = red[lane < WARPS ? lane : 0];
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-    __syncthreads();
-    const float m = mx * a.c, nm = -m;
-
-    // ---- pass 2: softmax sums and the race
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const float nm = -m;
     float s0 = 0.f, s1 = 0.f, u0 = 0.f, u1 = 0.f;
     Race best;
     best.init();
-    const uint32_t rlo = (uint32_t)row;
-    PhiloxKeys keys;
-    keys.init(a.k0, a.k1);
     if (VECTOR) {
         const uint4 *src4 = reinterpret_cast<const uint4 *>(src);
         const int nvec = V / N;
@@ -137,13 +117,13 @@ sample_kernel(const SampleArgs a)
 #pragma unroll
             for (int h = 0; h < N / 4; ++h) {
                 uint32_t w[4];
-                philox4x32_10((uint32_t)(i * (N / 4) + h), rlo, a.off_lo, a.off_hi, keys, w);
+                philox4x32_10((uint32_t)(i * (N / 4) + h), row, a.off_lo, a.off_hi, keys, w);
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    const float t = fmaf(x[h * 4 + q], a.c, nm);
+                    const float t = fmaf(x[h * 4 + q], c, nm);
                     const float e = ex2(t);
                     if (q & 1) { s1 += e; u1 = fmaf(e, t, u1); } else { s0 += e; u0 = fmaf(e, t, u0); }
-                    best.offer(e, exponential_variate(w[q]), t, i * N + h * 4 + q);
+                    best.offer(e, log2_uniform(w[q]), i * N + h * 4 + q);
                 }
             }
         }
@@ -152,15 +132,15 @@ sample_kernel(const SampleArgs a)
             float x = Pack<T>::load1(src + j);
             x = (x != x) ? x : fmaxf(x, kNegBig);
             uint32_t w[4];
-            philox4x32_10((uint32_t)(j >> 2), rlo, a.off_lo, a.off_hi, keys, w);
-            const float t = fmaf(x, a.c, nm);
+            philox4x32_10((uint32_t)(j >> 2), row, a.off_lo, a.off_hi, keys, w);
+            const float t = fmaf(x, c, nm);
             const float e = ex2(t);
             s0 += e;
             u0 = fmaf(e, t, u0);
-            best.offer(e, exponential_variate(w[j & 3]), t, j);
+            best.offer(e, log2_uniform(w[j & 3]), j);
         }
     }
-    // ---- block merge: sums by addition, race by comparison (fixed order: lanes, then warps)
+    // block merge: sums by addition, race by comparison (fixed order: lanes, then warps)
     float s = s0 + s1, u = u0 + u1;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
@@ -168,36 +148,91 @@ sample_kernel(const SampleArgs a)
         u += __shfl_xor_sync(0xffffffffu, u, off);
         Race o;
         o.e = __shfl_xor_sync(0xffffffffu, best.e, off);
-        o.E = __shfl_xor_sync(0xffffffffu, best.E, off);
-        o.t = __shfl_xor_sync(0xffffffffu, best.t, off);
+        o.L = __shfl_xor_sync(0xffffffffu, best.L, off);
         o.j = __shfl_xor_sync(0xffffffffu, best.j, off);
         best.merge(o);
     }
-    __shared__ float rs[32], ru[32];
+    __syncthreads();   // the arrays below may still be read from an earlier call
     if (lane == 0) {
-        rs[warp] = s; ru[warp] = u;
-        red[warp] = best.e; red[32 + warp] = best.E; red[64 + warp] = best.t; redj[warp] = best.j;
+        sm.rs[warp] = s; sm.ru[warp] = u; sm.re[warp] = best.e; sm.rl[warp] = best.L; sm.rj[warp] = best.j;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
         s = 0.f; u = 0.f;
         best.init();
         for (int w = 0; w < WARPS; ++w) {
-            s += rs[w]; u += ru[w];
+            s += sm.rs[w]; u += sm.ru[w];
             Race o;
-            o.e = red[w]; o.E = red[32 + w]; o.t = red[64 + w]; o.j = redj[w];
+            o.e = sm.re[w]; o.L = sm.rl[w]; o.j = sm.rj[w];
             best.merge(o);
         }
-        const float l2s = log2f(s);
-        float lp = (best.t - l2s) * kLn2;
-        float H = (l2s - u / s) * kLn2;
-        float L = (m + l2s) * kLn2;
+    }
+    s_out = s; u_out = u; best_out = best;
+}
+
+template <typename T, bool VECTOR, int THREADS>
+__global__ void __launch_bounds__(THREADS)
+sample_kernel(const SampleArgs a)
+{
+    constexpr int N = Pack<T>::N;
+    constexpr int WARPS = THREADS / 32;
+    __shared__ SampleSmem sm;
+    const int64_t row = blockIdx.x;
+    const T *src = reinterpret_cast<const T *>(a.logits) + row * a.row_stride;
+    const int V = a.V;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    PhiloxKeys keys;
+    keys.init(a.k0, a.k1);
+
+    // First attempt with the maximum of the row's first pack as the reference of the exponentials (any
+    // reference works for the race and the sums as long as nothing overflows): one pass over the row.
+    float m = VECTOR ? row_reference<T>(src, a.c) : safe_reference(fmaxf(Pack<T>::load1(src), kNegBig), a.c);
+    float s, u;
+    Race best;
+    sums_and_race<T, VECTOR, THREADS>(src, V, a.c, m, (uint32_t)row, a, keys, sm, s, u, best);
+    if (threadIdx.x == 0) sm.redo = !(s < 1.0e37f) || !(fabsf(u) < 1.0e37f);
+    __syncthreads();
+    if (sm.redo) {
+        // a sum overflowed (an element lies more than ~2^127 above the reference) or the row holds a NaN or
+        // +inf: take the exact maximum (NaN-blind; a NaN then shows up in the sums again) and repeat
+        float mx = kNegBig;
+        if (VECTOR) {
+            const uint4 *src4 = reinterpret_cast<const uint4 *>(src);
+            const int nvec = V / N;
+            for (int i = threadIdx.x; i < nvec; i += THREADS) {
+                float x[N], xm;
+                Pack<T>::unpack(src4[i], x, xm);
+                mx = fmaxf(mx, xm);
+            }
+        } else {
+            for (int j = threadIdx.x; j < V; j += THREADS) mx = fmaxf(mx, fmaxf(Pack<T>::load1(src + j), kNegBig));
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+        __syncthreads();
+        if (lane == 0) sm.rs[warp] = mx;
+        __syncthreads();
+        mx = sm.rs[lane < WARPS ? lane : 0];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+        m = safe_reference(mx, a.c);
+        sums_and_race<T, VECTOR, THREADS>(src, V, a.c, m, (uint32_t)row, a, keys, sm, s, u, best);
+    }
+    if (threadIdx.x == 0) {
         int tok = best.j;
-        // no finite maximum, a NaN or +inf in the row, or no candidate: nothing is drawn
-        if (!(mx > -1.0e29f) || !(s == s) || !(fabsf(u) < 3.0e38f) || tok == 0x7fffffff) {
+        float lp, H, L;
+        // a NaN or +inf in the row, or no element with non-zero probability: nothing is drawn
+        if (!(s < 3.0e38f) || !(fabsf(u) < 3.0e38f) || tok == 0x7fffffff) {
             tok = -1;
             lp = H = L = __int_as_float(0x7fc00000);
             if (a.status) atomicOr(a.status, PPO_DEV_BAD_ROW);
+        } else {
+            float x = Pack<T>::load1(src + tok);          // the winner's own logit, for its log-prob
+            x = fmaxf(x, kNegBig);
+            const float l2s = log2f(s);
+            lp = (fmaf(x, a.c, -m) - l2s) * kLn2;
+            H = (l2s - u / s) * kLn2;
+            L = (m + l2s) * kLn2;
         }
         a.tokens[row] = tok;
         if (a.logprob) a.logprob[row] = lp;

@@ -93,3 +93,14 @@ def test_minus_infinity_never_drawn_and_bad_rows(P):
     assert (tok[:3] % 2 == 1).all() and np.isfinite(npy(lp)[:3]).all() and np.isfinite(npy(ent)[:3]).all()
     assert (tok[3:] == -1).all() and np.isnan(npy(lp)[3:]).all()
     assert P.last_device_status(ws) == 8
+
+
+def test_rows_far_above_their_first_pack_take_the_exact_maximum(P, oracle):
+    """The one-pass path uses the row's first pack as reference; a row whose other logits lie hundreds above it
+    overflows there and must come out the same through the exact-maximum repeat."""
+    g = torch.Generator(device="cuda").manual_seed(9)
+    x = 2.0 * torch.randn((24, 4096), generator=g, device="cuda")
+    x[::2, :8] = -300.0
+    _compare(P, oracle, x, 0.7, seed=77)
+    xb = x.to(torch.bfloat16)
+    _compare(P, oracle, xb, 0.7, seed=78)
