@@ -370,7 +370,9 @@ row_engine_kernel(const EngineArgs a)
             int64_t it_static = blockIdx.x;
             const auto fetch = [&]() -> int {
                 if constexpr (MODE == 1) {
-                    const int64_t item = atomicAdd(&a.hdr->real_next, 1);
+                    // the first two items of a block are fixed (no counter round trip before the first copy
+                    // can be issued); everything after them is drawn from the counter
+                    const int64_t item = 2 * (int64_t)gridDim.x + atomicAdd(&a.hdr->real_next, 1);
                     return item < n_items ? a.order[item] : -1;
                 } else {
                     while (it_static < n_items) {
@@ -386,8 +388,15 @@ row_engine_kernel(const EngineArgs a)
             };
             // the block's rows reach the consumers through sm.ring; the entry for item k + 1 is written
             // before the first copy of item k is armed, and read after that copy has landed
-            int row_c = fetch();
-            int row_n = row_c >= 0 ? fetch() : -1;
+            int row_c, row_n;
+            if (MODE == 1) {
+                const int64_t i0 = blockIdx.x, i1 = i0 + gridDim.x;
+                row_c = i0 < n_items ? a.order[i0] : -1;
+                row_n = i1 < n_items ? a.order[i1] : -1;
+            } else {
+                row_c = fetch();
+                row_n = row_c >= 0 ? fetch() : -1;
+            }
             sm.ring[0] = row_c;
             if (row_c < 0) mbar_arrive(&sm.full[0]);   // no row at all: complete the phase the consumers wait for
             int64_t prev_row = -1;
