@@ -680,7 +680,7 @@ def run_sample(args):
         total_ms = float(t.item())
     ms = total_ms / K
     logits = B * T * V
-    # instructions the method needs per logit (stated in the design doc): Philox4x32-10 10, uniform 2, log2 1, widen 1,
+    # instructions the method needs per logit: Philox4x32-10 10, uniform 2, log2 1, widen 1,
     # scale 1, exp2 1, two sums 2, race 3
     ops_per_logit = 21
     clocks = clk.summary()
