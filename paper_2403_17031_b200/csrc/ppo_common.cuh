@@ -22,7 +22,10 @@ struct WorkspaceHeader {
     int done_blocks;   // blocks of the loss kernel that have retired (reset by every loss call)
     int step_blocks;   // blocks of ppo_step's token-level kernel that have finished (resets itself)
     int real_next;     // work counter of the loss kernel's mask==1 rows (reset by every loss call)
-    int reserved[58];
+    int order_ready;   // n_tokens + 1 once token count, counters and row order of the loss call in flight are written
+    int adv_ready;     // 1 once the advantages / returns that the loss call reads are written
+    int step_blocks2;  // second ticket of ppo_step's token-level kernel (resets itself)
+    int reserved[55];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header is one 256-byte block");
 
@@ -331,9 +334,61 @@ __device__ __forceinline__ void reduce_loss_partials(const float *partials, int6
     }
 }
 
+// Hand-over of results between two kernels that overlap in time (the loss kernel of ppo_step is launched
+// while the token-level kernel before it is still running, see launch_dependent): the writer publishes
+// with flag_set after its data, the reader polls with flag_wait before it touches them. The wait is
+// bounded (~1 s); when it runs out the status word gets PPO_DEV_TIMEOUT and the caller carries on.
+__device__ __forceinline__ void flag_set(int *flag, int value = 1 /* non-zero */)
+{
+    __threadfence();
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(flag), "r"(value) : "memory");
+}
+
+// returns the flag's (non-zero) value, or 0 after the wait ran out
+__device__ __forceinline__ int flag_wait(const int *flag, int *status)
+{
+    for (uint32_t it = 0; it < (1u << 20); ++it) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+        if (v) return v;
+        __nanosleep(200);
+    }
+    if (status) atomicOr(status, PPO_DEV_TIMEOUT);
+    return 0;
+}
+
+// Programmatic dependent launch: a kernel launched with launch_dependent() may be scheduled while the
+// kernel before it in the stream is still running, but only once every block of that kernel has executed
+// grid_dependents_may_launch() or has exited - so the earlier kernel is resident and will finish, and the
+// later one may wait (flag_wait) for what it produces. The instruction does nothing when no dependent
+// launch follows.
+__device__ __forceinline__ void grid_dependents_may_launch() { asm volatile("griddepcontrol.launch_dependents;"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                    Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+    if (e != cudaSuccess) {   // attribute not accepted in this context: ordinary launch (same results, no overlap)
+        (void)cudaGetLastError();
+        cfg.numAttrs = 0;
+        e = cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+    }
+    return e;
+}
+
 // launchers shared between translation units
 // all token-level steps of ppo_step in one launch (EOS trick, KL rewards, GAE, loss prologue, whitening)
-int launch_rollout(const ppo_step_io *io, int B, int T, const ppo_params *p, cudaStream_t s);
 // ppo_loss_fwd_bwd without its prologue launch (the caller has already run the prologue on this mask)
 int loss_fwd_bwd_prepared(const void *logits, int dtype, int32_t B, int32_t T, int64_t V, const int32_t *tokens,
                           const uint8_t *mask, const float *old_logprob, const float *advantages,
@@ -342,9 +397,12 @@ int loss_fwd_bwd_prepared(const void *logits, int dtype, int32_t B, int32_t T, i
                           float *dlogprob, void *workspace, void *stream, bool prepared);
 int launch_loss_prepare(const uint8_t *mask, int64_t rows, void *workspace, cudaStream_t s);
 // step 1 for policy and reference logits in one launch; PPO_ERR_UNSUPPORTED if the layout rules it out
+// (also clears the two hand-over flags of the header for the kernels that follow in ppo_step)
 int launch_logprob_pair(const void *policy_logits, const void *ref_logits, int dtype, int64_t rows, int V,
                         const int32_t *tokens, float c, float *logprob, float *entropy, float *ref_logprob,
-                        int *status, cudaStream_t s);
+                        WorkspaceHeader *hdr, cudaStream_t s);
+// flags_cleared: the launch before this one has cleared the header's hand-over flags already
+int launch_rollout(const ppo_step_io *io, int B, int T, const ppo_params *p, bool flags_cleared, cudaStream_t s);
 int launch_loss_finalize(int64_t rows, float vf_coef, float *losses, void *workspace, cudaStream_t s);
 
 // tuning options (ppo_set_option)

@@ -77,9 +77,12 @@ template <typename T, int THREADS>
 __global__ void __launch_bounds__(THREADS)
 logprob_pair_kernel(const T *__restrict__ policy_logits, const T *__restrict__ ref_logits, int V,
                     const int32_t *__restrict__ tokens, float c, float *__restrict__ logprob,
-                    float *__restrict__ entropy, float *__restrict__ ref_logprob, int *status)
+                    float *__restrict__ entropy, float *__restrict__ ref_logprob, int *status, int *flags2)
 {
     __shared__ float red[96];
+    // the hand-over flags between the two kernels that follow in ppo_step start at 0 (nothing runs beside this
+    // kernel on the stream, and the next kernel starts after it has ended)
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) { flags2[0] = 0; flags2[1] = 0; }
     if (blockIdx.y == 0)
         logprob_entropy_row<T, true, true, THREADS>(policy_logits, V, V, tokens, nullptr, c, logprob, entropy, nullptr,
                                                     status, red);
@@ -263,8 +266,11 @@ static int launch_logprob(const void *logits, int64_t rows, int V, int64_t row_s
 // PPO_ERR_UNSUPPORTED when the pointers or the shape do not allow 16-byte packs (the caller then makes two calls)
 int launch_logprob_pair(const void *policy_logits, const void *ref_logits, int dtype, int64_t rows, int V,
                         const int32_t *tokens, float c, float *logprob, float *entropy, float *ref_logprob,
-                        int *status, cudaStream_t s)
+                        WorkspaceHeader *hdr, cudaStream_t s)
 {
+    int *status = &hdr->status, *flags2 = &hdr->order_ready;
+    static_assert(offsetof(WorkspaceHeader, adv_ready) == offsetof(WorkspaceHeader, order_ready) + sizeof(int),
+                  "the two flags are cleared as a pair");
     constexpr int THREADS = 256;
     const size_t es = dtype == PPO_F32 ? 4 : 2;
     const int N = dtype == PPO_F32 ? 4 : 8;
@@ -274,11 +280,11 @@ int launch_logprob_pair(const void *policy_logits, const void *ref_logits, int d
     if (dtype == PPO_F32)
         logprob_pair_kernel<float, THREADS><<<grid, THREADS, 0, s>>>(
             reinterpret_cast<const float *>(policy_logits), reinterpret_cast<const float *>(ref_logits), V, tokens, c,
-            logprob, entropy, ref_logprob, status);
+            logprob, entropy, ref_logprob, status, flags2);
     else
         logprob_pair_kernel<__nv_bfloat16, THREADS><<<grid, THREADS, 0, s>>>(
             reinterpret_cast<const __nv_bfloat16 *>(policy_logits), reinterpret_cast<const __nv_bfloat16 *>(ref_logits),
-            V, tokens, c, logprob, entropy, ref_logprob, status);
+            V, tokens, c, logprob, entropy, ref_logprob, status, flags2);
     return launch_status();
 }
 
@@ -414,7 +420,7 @@ int ppo::loss_fwd_bwd_prepared(const void *logits, int dtype, int32_t B, int32_t
     a.c1 = p->vf_coef;
     rc = PPO_ERR_UNSUPPORTED;
     if (option_value(PPO_OPT_ROW_ENGINE) != 1) {
-        rc = launch_loss_bulk(a, dtype, workspace, losses, p->vf_coef, s);
+        rc = launch_loss_bulk(a, dtype, workspace, losses, p->vf_coef, prepared, s);
         if (rc != PPO_ERR_UNSUPPORTED) return rc;      // the engine reduces the partials itself
     }
     rc = dtype == PPO_F32 ? launch_loss<float>(a, s) : launch_loss<__nv_bfloat16>(a, s);
@@ -457,7 +463,7 @@ extern "C" int ppo_logprob_bwd(const void *logits, int dtype, int64_t rows, int6
     float *sink = reinterpret_cast<float *>(ws_header(workspace)->reserved);
     rc = PPO_ERR_UNSUPPORTED;
     if (option_value(PPO_OPT_ROW_ENGINE) != 1) {
-        rc = launch_loss_bulk(a, dtype, workspace, sink, 0.f, s);
+        rc = launch_loss_bulk(a, dtype, workspace, sink, 0.f, false, s);
         if (rc != PPO_ERR_UNSUPPORTED) return rc;
     }
     rc = dtype == PPO_F32 ? launch_loss<float>(a, s) : launch_loss<__nv_bfloat16>(a, s);

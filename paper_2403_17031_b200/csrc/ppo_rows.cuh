@@ -248,6 +248,9 @@ int launch_logprob_bulk(const void *logits, int dtype, int64_t rows, int V, int6
                         const int32_t *tokens, const uint8_t *mask, float c, float *logprob, float *entropy,
                         float *lse, int *status, cudaStream_t s);
 // (the engine's loss kernel also reduces the partials and writes `losses` itself)
-int launch_loss_bulk(const LossArgs &a, int dtype, void *workspace, float *losses, float vf_coef, cudaStream_t s);
+// `dependent`: launch so that the kernel may start while the kernel before it in the stream still runs (it
+// waits for the workspace header's flags before it reads that kernel's results)
+int launch_loss_bulk(const LossArgs &a, int dtype, void *workspace, float *losses, float vf_coef, bool dependent,
+                     cudaStream_t s);
 
 }   // namespace ppo

@@ -39,6 +39,7 @@ struct EngineSmem {
     int next_item;
     int is_last;
     int ring[4];           // row of the block's k-th item at [k % 4], -1 = no further item
+    int n_tokens;          // step 6: number of mask==1 rows of the call
     double lred[6 * 32];
     alignas(128) unsigned char zeros[kZeroBytes];
 };
@@ -241,6 +242,7 @@ struct EngineArgs {
     WorkspaceHeader *hdr;
     float *losses;
     float vf_coef;
+    int wait_flags;         // the launch overlaps the kernel that produces order / advantages: poll the header's flags
 };
 
 template <int CONS>
@@ -262,7 +264,7 @@ __device__ __forceinline__ void engine_epilogue(const EngineArgs &a, EngineSmem 
     block_sync_all<CONS>();
     if (!sm.is_last) return;
     __threadfence();
-    reduce_loss_partials<CONS + 64>(a.loss.partials, a.loss.rows, a.hdr->n_tokens, a.vf_coef, a.losses, sm.lred,
+    reduce_loss_partials<CONS + 64>(a.loss.partials, a.loss.rows, sm.n_tokens, a.vf_coef, a.losses, sm.lred,
                                     (int)threadIdx.x, [] { block_sync_all<CONS>(); });
 }
 
@@ -304,8 +306,6 @@ row_engine_kernel(const EngineArgs a)
     const int nch = (nvec + kChunkPacks - 1) / kChunkPacks;
     const T *logits = reinterpret_cast<const T *>(a.logits);
     const int64_t stride = MODE == 0 ? a.row_stride : (int64_t)V;
-    // number of work items of the streaming phase and how an item maps to a row
-    const int64_t n_items = MODE == 0 ? a.rows : (int64_t)a.hdr->n_tokens;
     int *status = a.status;
 
     if (threadIdx.x == 0) {
@@ -321,7 +321,14 @@ row_engine_kernel(const EngineArgs a)
             reinterpret_cast<uint4 *>(sm.zeros)[i] = make_uint4(0u, 0u, 0u, 0u);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // zeros are read by bulk copies
     }
+    // step 6 inside ppo_step: this kernel may have been launched while the token-level kernel is still at
+    // work; everything above touched shared memory only, from here on it reads what that kernel publishes
+    // (the first flag carries the token count)
+    if (MODE == 1 && threadIdx.x == 0)
+        sm.n_tokens = a.wait_flags ? max(flag_wait(&a.hdr->order_ready, status) - 1, 0) : a.hdr->n_tokens;
     __syncthreads();
+    // number of work items of the streaming phase
+    const int64_t n_items = MODE == 0 ? a.rows : (int64_t)sm.n_tokens;
 
     if (threadIdx.x >= kConsumers + 32) {
         // ------------------------------------------------------------ filler (step 6 only)
@@ -464,7 +471,7 @@ row_engine_kernel(const EngineArgs a)
     const int ct = threadIdx.x;
     const uint4 *buf = reinterpret_cast<const uint4 *>(smem_raw);
     const T *buf_elems = reinterpret_cast<const T *>(smem_raw);
-    const double inv_n = MODE == 1 ? 1.0 / (double)a.hdr->n_tokens : 0.0;
+    const double inv_n = MODE == 1 ? 1.0 / (double)sm.n_tokens : 0.0;
     const float inv_n_f = (float)inv_n;
     uint32_t k = 0;
     // The block's rows come from sm.ring (see the producer). Per-row scalars are dependent loads
@@ -473,7 +480,10 @@ row_engine_kernel(const EngineArgs a)
     int row_c, row_n = -1;
     int tok_c = -1, tok_n = -1;
     float in_c[5] = {0.f, 0.f, 0.f, 0.f, 0.f}, in_n[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
+    // advantages and returns of this step: polled while the first row's bytes are on their way
+    if (MODE == 1 && a.wait_flags && ct == 0) flag_wait(&a.hdr->adv_ready, status);
     mbar_wait(&sm.full[0], 0, status);
+    if (MODE == 1) consumer_sync<CONS>();
     row_c = sm.ring[0];
     if (row_c >= 0) {
         tok_c = a.tokens[row_c];
@@ -671,7 +681,7 @@ static int sm_count()
 }
 
 template <typename T, int MODE, bool ENTROPY>
-static int launch_engine(const EngineArgs &a, int64_t max_items, cudaStream_t s)
+static int launch_engine(const EngineArgs &a, int64_t max_items, bool dependent, cudaStream_t s)
 {
     const size_t row_bytes = (size_t)a.V * sizeof(T);
     if (row_bytes > kMaxRowBytes) return PPO_ERR_UNSUPPORTED;
@@ -684,12 +694,14 @@ static int launch_engine(const EngineArgs &a, int64_t max_items, cudaStream_t s)
         // two blocks per SM: 16 consumer warps each, 16 KB chunks
         auto kern = row_engine_kernel<T, MODE, ENTROPY, 2, 512>;
         PPO_RETURN_IF_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        kern<<<(unsigned)grid, 512 + 64, smem, s>>>(a);
+        if (dependent) PPO_RETURN_IF_CUDA(launch_dependent(kern, dim3((unsigned)grid), dim3(512 + 64), smem, s, a));
+        else kern<<<(unsigned)grid, 512 + 64, smem, s>>>(a);
     } else {
         // one block per SM: 30 consumer warps (a block holds at most 1024 threads), 30 KB chunks
         auto kern = row_engine_kernel<T, MODE, ENTROPY, 1, 960>;
         PPO_RETURN_IF_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        kern<<<(unsigned)grid, 960 + 64, smem, s>>>(a);
+        if (dependent) PPO_RETURN_IF_CUDA(launch_dependent(kern, dim3((unsigned)grid), dim3(960 + 64), smem, s, a));
+        else kern<<<(unsigned)grid, 960 + 64, smem, s>>>(a);
     }
     return launch_status();
 }
@@ -719,14 +731,15 @@ int launch_logprob_bulk(const void *logits, int dtype, int64_t rows, int V, int6
     a.status = status;
     if (dtype == PPO_F32) {
         if (!bulk_ok<float>(logits, row_stride, V)) return PPO_ERR_UNSUPPORTED;
-        return entropy ? launch_engine<float, 0, true>(a, rows, s) : launch_engine<float, 0, false>(a, rows, s);
+        return entropy ? launch_engine<float, 0, true>(a, rows, false, s) : launch_engine<float, 0, false>(a, rows, false, s);
     }
     if (!bulk_ok<__nv_bfloat16>(logits, row_stride, V)) return PPO_ERR_UNSUPPORTED;
-    return entropy ? launch_engine<__nv_bfloat16, 0, true>(a, rows, s)
-                   : launch_engine<__nv_bfloat16, 0, false>(a, rows, s);
+    return entropy ? launch_engine<__nv_bfloat16, 0, true>(a, rows, false, s)
+                   : launch_engine<__nv_bfloat16, 0, false>(a, rows, false, s);
 }
 
-int launch_loss_bulk(const LossArgs &la, int dtype, void *workspace, float *losses, float vf_coef, cudaStream_t s)
+int launch_loss_bulk(const LossArgs &la, int dtype, void *workspace, float *losses, float vf_coef, bool dependent,
+                     cudaStream_t s)
 {
     if (!la.dlogits || !aligned16(la.dlogits)) return PPO_ERR_UNSUPPORTED;
     EngineArgs a = {};
@@ -743,12 +756,13 @@ int launch_loss_bulk(const LossArgs &la, int dtype, void *workspace, float *loss
     a.hdr = ws_header(workspace);
     a.losses = losses;
     a.vf_coef = vf_coef;
+    a.wait_flags = dependent ? 1 : 0;
     if (dtype == PPO_F32) {
         if (!bulk_ok<float>(la.logits, la.V, la.V)) return PPO_ERR_UNSUPPORTED;
-        return launch_engine<float, 1, true>(a, la.rows, s);
+        return launch_engine<float, 1, true>(a, la.rows, dependent, s);
     }
     if (!bulk_ok<__nv_bfloat16>(la.logits, la.V, la.V)) return PPO_ERR_UNSUPPORTED;
-    return launch_engine<__nv_bfloat16, 1, true>(a, la.rows, s);
+    return launch_engine<__nv_bfloat16, 1, true>(a, la.rows, dependent, s);
 }
 
 }   // namespace ppo

@@ -30,7 +30,8 @@ extern "C" int ppo_step(const ppo_step_io *io, int dtype, int32_t B, int32_t T, 
         finite_f(p->temperature) && option_value(PPO_OPT_ROW_ENGINE) != 2)
         rc = launch_logprob_pair(io->policy_logits, io->ref_logits, dtype, rows, (int)V, io->responses,
                                  kLog2e / p->temperature, io->logprob, io->entropy, io->ref_logprob,
-                                 &ws_header(io->workspace)->status, s);
+                                 ws_header(io->workspace), s);
+    const bool flags_cleared = rc == PPO_OK;
     if (rc == PPO_ERR_UNSUPPORTED) {   // layout without 16-byte packs (or the row engine was asked for): two calls
         rc = ppo_logprob_entropy(io->policy_logits, dtype, rows, V, V, io->responses, nullptr, p->temperature,
                                  io->logprob, io->entropy, nullptr, io->workspace, stream);
@@ -39,7 +40,7 @@ extern "C" int ppo_step(const ppo_step_io *io, int dtype, int32_t B, int32_t T, 
                                  io->ref_logprob, nullptr, nullptr, io->workspace, stream);
     }
     if (rc) return rc;
-    rc = launch_rollout(io, B, T, p, s);
+    rc = launch_rollout(io, B, T, p, flags_cleared, s);
     if (rc) return rc;
     return loss_fwd_bwd_prepared(io->loss_logits ? io->loss_logits : io->policy_logits, dtype, B, T, V, io->responses,
                                  io->mask, io->old_logprob ? io->old_logprob : io->logprob, io->advantages_whitened,

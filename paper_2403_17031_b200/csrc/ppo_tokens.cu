@@ -182,7 +182,8 @@ constexpr int kReduceThreads = 1024;
 // the row order: indices of real rows ascending from the front, masked rows from the back. Each
 // thread owns one contiguous segment of rows, so the order is deterministic.
 __device__ __forceinline__ void loss_prepare_block(const uint8_t *mask, int64_t rows, WorkspaceHeader *hdr,
-                                                   int32_t *__restrict__ order, int *warp_tot /* 32 ints */)
+                                                   int32_t *__restrict__ order, int *warp_tot /* 32 ints */,
+                                                   bool publish /* a loss kernel may be waiting for the result */)
 {
     const int64_t seg = (rows + kReduceThreads - 1) / kReduceThreads;
     const int64_t r0 = min(rows, (int64_t)threadIdx.x * seg), r1 = min(rows, r0 + seg);
@@ -221,13 +222,17 @@ __device__ __forceinline__ void loss_prepare_block(const uint8_t *mask, int64_t 
         if (mask[r]) order[real_pos++] = (int32_t)r;
         else order[rows - 1 - masked_pos++] = (int32_t)r;
     }
+    if (!publish) return;
+    __syncthreads();
+    // a loss kernel that is already running may go on; the flag carries the token count (+1) it needs first
+    if (threadIdx.x == 0) flag_set(&hdr->order_ready, *reinterpret_cast<volatile int *>(&hdr->n_tokens) + 1);
 }
 
 __global__ void __launch_bounds__(kReduceThreads)
 loss_prepare_kernel(const uint8_t *__restrict__ mask, int64_t rows, WorkspaceHeader *hdr, int32_t *__restrict__ order)
 {
     __shared__ int warp_tot[32];
-    loss_prepare_block(mask, rows, hdr, order, warp_tot);
+    loss_prepare_block(mask, rows, hdr, order, warp_tot, false);
 }
 
 // ---------------------------------------------------------------- fused launch of ppo_step
@@ -250,7 +255,7 @@ rollout_kernel(const int32_t *responses, int B, int T, int eos_id, int pad_id, c
                const float *__restrict__ ref_logprob, const float *__restrict__ values, float kl_coef, double gamma,
                double c, float eps, float *__restrict__ kl, float *rewards, float *advantages,
                float *__restrict__ returns, float *whitened, float *__restrict__ stats3, WorkspaceHeader *hdr,
-               int32_t *__restrict__ order)
+               int32_t *__restrict__ order, int clear_flags)
 {
     static_assert(kWhitenThreads == kReduceThreads, "one block shape for both block-wide helpers");
     __shared__ double red[32];
@@ -258,54 +263,108 @@ rollout_kernel(const int32_t *responses, int B, int T, int eos_id, int pad_id, c
     __shared__ int is_last;
     const int lane = threadIdx.x & 31;
     const int b = blockIdx.x * (kWhitenThreads / 32) + (threadIdx.x >> 5);
-    if (b < B) {
-        if (PHASE == 2) {
+    const int64_t rows = (int64_t)B * T;
+    // The loss kernel of this step may start while this kernel runs (launch_dependent) and waits on the two
+    // flags. They are 0 by now: cleared by the launch before this one, or here before any block lets the loss
+    // kernel launch (it launches once ALL blocks have said so).
+    if (clear_flags) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            hdr->order_ready = 0;
+            hdr->adv_ready = 0;
+            __threadfence();
+        }
+        __syncthreads();
+    }
+    if (PHASE == 0) grid_dependents_may_launch();
+
+    // tickets: the block that draws the last one continues with the batch-wide step
+    const auto last_block = [&](int *counter, int n_blocks) {
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const int ticket = atomicAdd(counter, 1);
+            is_last = ticket == n_blocks - 1;
+            if (is_last) *counter = 0;   // ready for the next call
+        }
+        __syncthreads();
+        const bool last = is_last != 0;
+        if (last) __threadfence();
+        return last;
+    };
+
+    if (PHASE == 2) {
+        if (b < B) {
             const float *r = rewards + (int64_t)b * T;
             gae_sequence([r](int t) { return r[t]; }, values + (int64_t)b * T, seq_len[b], T, gamma, c,
                          advantages + (int64_t)b * T, returns + (int64_t)b * T, lane);
-        } else {
-            const int L = truncate_sequence(responses, b, T, eos_id, pad_id, scores, no_eos_score, responses_out,
-                                            eos_index, seq_len, mask, scores_out, lane);
-            int first_eos = 0;   // whether the sequence has an EOS decides the score that is used
-            {
-                const int32_t *r = responses + (int64_t)b * T;
-                first_eos = (L < T) || (r[T - 1] == eos_id);
-            }
-            const float score = first_eos ? scores[b] : no_eos_score;
-            const float *lp = logprob + (int64_t)b * T, *lr = ref_logprob + (int64_t)b * T;
-            for (int t = lane; t < T; t += 32) {
-                const bool real = t < L;
-                const float k = real ? __fsub_rn(lp[t], lr[t]) : 0.f;
-                kl[(int64_t)b * T + t] = k;
-                rewards[(int64_t)b * T + t] = kl_reward(k, real, kl_coef, t == L - 1, score);
-            }
-            if (PHASE == 0)
-                gae_sequence(
-                    [=](int t) {
-                        return kl_reward(t < L ? __fsub_rn(lp[t], lr[t]) : 0.f, t < L, kl_coef, t == L - 1, score);
-                    },
-                    values + (int64_t)b * T, L, T, gamma, c, advantages + (int64_t)b * T, returns + (int64_t)b * T,
-                    lane);
         }
+        if (!last_block(&hdr->step_blocks, (int)gridDim.x)) return;
+        loss_prepare_block(mask, rows, hdr, order, warp_tot, true);
+        __syncthreads();
+        whiten_block(advantages, mask, rows, 1, eps, whitened, stats3, &hdr->status, red);
+        __syncthreads();
+        if (threadIdx.x == 0) flag_set(&hdr->adv_ready);
+        return;
     }
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const int ticket = atomicAdd(&hdr->step_blocks, 1);
-        is_last = ticket == (int)gridDim.x - 1;
-        if (is_last) hdr->step_blocks = 0;   // ready for the next call
+
+    // PHASE 0 has one block more than the sequences need: it waits until every other block has done the EOS
+    // trick (the mask is all the loss prologue needs), then writes token count and row order and publishes
+    // them, while the other blocks go on with rewards and advantages.
+    const int n_seq_blocks = PHASE == 0 ? (int)gridDim.x - 1 : (int)gridDim.x;
+    if (PHASE == 0 && (int)blockIdx.x == n_seq_blocks) {
+        if (threadIdx.x == 0) {
+            bool done = false;
+            for (uint32_t it = 0; it < (1u << 20) && !done; ++it) {
+                int v;
+                asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(&hdr->step_blocks) : "memory");
+                done = v >= n_seq_blocks;
+                if (!done) __nanosleep(100);
+            }
+            if (!done) atomicOr(&hdr->status, PPO_DEV_TIMEOUT);
+            hdr->step_blocks = 0;   // ready for the next call
+        }
+        __syncthreads();
+        loss_prepare_block(mask, rows, hdr, order, warp_tot, true);
+        return;
     }
-    __syncthreads();
-    if (!is_last) return;
-    __threadfence();
-    const int64_t rows = (int64_t)B * T;
+    int L = 0;
+    if (b < B)
+        L = truncate_sequence(responses, b, T, eos_id, pad_id, scores, no_eos_score, responses_out, eos_index, seq_len,
+                              mask, scores_out, lane);
+    if (PHASE == 0) {   // tell the prologue block
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) atomicAdd(&hdr->step_blocks, 1);
+    }
+    if (b < B) {
+        int first_eos = 0;   // whether the sequence has an EOS decides the score that is used
+        {
+            const int32_t *r = responses + (int64_t)b * T;
+            first_eos = (L < T) || (r[T - 1] == eos_id);
+        }
+        const float score = first_eos ? scores[b] : no_eos_score;
+        const float *lp = logprob + (int64_t)b * T, *lr = ref_logprob + (int64_t)b * T;
+        for (int t = lane; t < T; t += 32) {
+            const bool real = t < L;
+            const float k = real ? __fsub_rn(lp[t], lr[t]) : 0.f;
+            kl[(int64_t)b * T + t] = k;
+            rewards[(int64_t)b * T + t] = kl_reward(k, real, kl_coef, t == L - 1, score);
+        }
+        if (PHASE == 0)
+            gae_sequence(
+                [=](int t) {
+                    return kl_reward(t < L ? __fsub_rn(lp[t], lr[t]) : 0.f, t < L, kl_coef, t == L - 1, score);
+                },
+                values + (int64_t)b * T, L, T, gamma, c, advantages + (int64_t)b * T, returns + (int64_t)b * T, lane);
+    }
+    if (!last_block(PHASE == 0 ? &hdr->step_blocks2 : &hdr->step_blocks, n_seq_blocks)) return;
     if (PHASE == 1) {
         whiten_block(rewards, mask, rows, 0, eps, rewards, nullptr, &hdr->status, red);
         return;
     }
-    loss_prepare_block(mask, rows, hdr, order, warp_tot);
-    __syncthreads();
     whiten_block(advantages, mask, rows, 1, eps, whitened, stats3, &hdr->status, red);
+    __syncthreads();
+    if (threadIdx.x == 0) flag_set(&hdr->adv_ready);
 }
 
 // Sum the per-token partials (fixed thread assignment, fp64) and write the eight loss scalars.
@@ -351,21 +410,21 @@ int launch_loss_prepare(const uint8_t *mask, int64_t rows, void *workspace, cuda
     return launch_status();
 }
 
-int launch_rollout(const ppo_step_io *io, int B, int T, const ppo_params *p, cudaStream_t s)
+int launch_rollout(const ppo_step_io *io, int B, int T, const ppo_params *p, bool flags_cleared, cudaStream_t s)
 {
-    const unsigned grid = (unsigned)((B + kWhitenThreads / 32 - 1) / (kWhitenThreads / 32));
-#define PPO_LAUNCH_ROLLOUT(PHASE)                                                                                    \
-    rollout_kernel<PHASE><<<grid, kWhitenThreads, 0, s>>>(                                                           \
+    const unsigned nb = (unsigned)((B + kWhitenThreads / 32 - 1) / (kWhitenThreads / 32));
+#define PPO_LAUNCH_ROLLOUT(PHASE, GRID, CLEAR)                                                                       \
+    rollout_kernel<PHASE><<<GRID, kWhitenThreads, 0, s>>>(                                                           \
         io->responses, B, T, p->eos_id, p->pad_id, io->scores, p->no_eos_score, io->responses_out, io->eos_index,    \
         io->seq_len, io->mask, io->scores_out, io->logprob, io->ref_logprob, io->values, p->kl_coef,                 \
         (double)p->gamma, (double)p->gamma * (double)p->lam, p->whiten_eps, io->kl, io->rewards, io->advantages,     \
         io->returns, io->advantages_whitened, io->whiten_stats, ws_header(io->workspace),                            \
-        ws_order(io->workspace, (int64_t)B * T))
+        ws_order(io->workspace, (int64_t)B * T), CLEAR)
     if (p->whiten_rewards) {
-        PPO_LAUNCH_ROLLOUT(1);
-        PPO_LAUNCH_ROLLOUT(2);
+        PPO_LAUNCH_ROLLOUT(1, nb, flags_cleared ? 0 : 1);
+        PPO_LAUNCH_ROLLOUT(2, nb, 0);
     } else {
-        PPO_LAUNCH_ROLLOUT(0);
+        PPO_LAUNCH_ROLLOUT(0, nb + 1, flags_cleared ? 0 : 1);   // + the block that runs the loss prologue
     }
 #undef PPO_LAUNCH_ROLLOUT
     return launch_status();
