@@ -176,12 +176,37 @@ __device__ __forceinline__ SoftmaxState consumer_merge_common(SoftmaxState st, f
     return r;
 }
 
+// The sums of one thread as two-wide fp32 vectors: even elements of a pack in .x, odd ones in .y. The
+// packed fp32 instructions of sm_100 (two fused multiply-adds or adds per issue slot, each lane rounded
+// like the scalar instruction) halve the issue slots of the arithmetic around the exponentials: fewer
+// instructions for the same bytes, which matters for the clocks under the board's power cap.
+struct PairAcc {
+    float2 s, u;
+    __device__ __forceinline__ void init() { s = u = make_float2(0.f, 0.f); }
+};
+
+template <typename T, bool ENTROPY, bool CLAMP = false>
+__device__ __forceinline__ void accumulate_pairs(const uint4 &v, float c, float nm, PairAcc &a)
+{
+    float x[Pack<T>::N];
+    if (CLAMP) Pack<T>::unpack_clamped(v, x);
+    else Pack<T>::unpack_raw(v, x);
+    const float2 cc = make_float2(c, c), nn = make_float2(nm, nm);
+#pragma unroll
+    for (int k = 0; k < Pack<T>::N; k += 2) {
+        const float2 t = __ffma2_rn(make_float2(x[k], x[k + 1]), cc, nn);
+        const float2 e = make_float2(ex2(t.x), ex2(t.y));
+        a.s = __fadd2_rn(a.s, e);
+        if (ENTROPY) a.u = __ffma2_rn(e, t, a.u);
+    }
+}
+
 // per-thread statistics with a fixed reference (the same for all threads of the row: the maximum of
 // the row's first pack) that is only moved when a chunk overflows
 template <typename T, bool ENTROPY>
 struct ThreadStats {
     float m;          // reference, base-2 units
-    FixedAcc acc;
+    PairAcc acc;
     __device__ __forceinline__ void init(float m_common)
     {
         m = m_common;
@@ -190,37 +215,46 @@ struct ThreadStats {
     __device__ __forceinline__ void rebase(float nm)
     {
         const float d = m - nm, a = ex2(d);
-        acc.u0 = a * fmaf(d, acc.s0, acc.u0);
-        acc.u1 = a * fmaf(d, acc.s1, acc.u1);
-        acc.s0 *= a;
-        acc.s1 *= a;
+        acc.u.x = a * fmaf(d, acc.s.x, acc.u.x);
+        acc.u.y = a * fmaf(d, acc.s.y, acc.u.y);
+        acc.s.x *= a;
+        acc.s.y *= a;
         m = nm;
+    }
+    // the sums left fp32 range, or a -inf/NaN logit turned the entropy sum into NaN
+    __device__ __forceinline__ bool broken() const
+    {
+        return !(acc.s.x + acc.s.y < 1.0e35f) || !(fabsf(acc.u.x + acc.u.y) < 1.0e35f);
+    }
+    // slow path for one pack: clamped values, reference moved up to the pack maximum when needed
+    __device__ __forceinline__ void pack_safe(const uint4 &v, float c)
+    {
+        float x[Pack<T>::N], xm;
+        Pack<T>::unpack(v, x, xm);
+        const float nm = safe_reference(xm, c);
+        if (nm > m) rebase(nm);
+        accumulate_pairs<T, ENTROPY, true>(v, c, -m, acc);
     }
     // fold up to two packs of one chunk
     __device__ __forceinline__ void chunk(const uint4 &v0, bool h0, const uint4 &v1, bool h1, float c)
     {
         if (!h0) return;                      // h1 implies h0
-        const FixedAcc save = acc;
-        accumulate_fixed<T, ENTROPY>(v0, c, -m, acc);
-        if (h1) accumulate_fixed<T, ENTROPY>(v1, c, -m, acc);
-        if (!(acc.s0 + acc.s1 < 1.0e35f) || !(fabsf(acc.u0 + acc.u1) < 1.0e35f)) {
-            // overflow, or -inf/NaN logits: move the reference up and redo the chunk with clamped values
+        const PairAcc save = acc;
+        accumulate_pairs<T, ENTROPY>(v0, c, -m, acc);
+        if (h1) accumulate_pairs<T, ENTROPY>(v1, c, -m, acc);
+        if (broken()) {
+            // overflow, or -inf/NaN logits: redo the chunk with clamped values and a moving reference
             acc = save;
-            float x[Pack<T>::N], xm0, xm1 = kNegBig;
-            Pack<T>::unpack(v0, x, xm0);
-            if (h1) Pack<T>::unpack(v1, x, xm1);
-            const float nm = safe_reference(fmaxf(xm0, xm1), c);
-            if (nm > m) rebase(nm);
-            accumulate_fixed<T, ENTROPY, true>(v0, c, -m, acc);
-            if (h1) accumulate_fixed<T, ENTROPY, true>(v1, c, -m, acc);
+            pack_safe(v0, c);
+            if (h1) pack_safe(v1, c);
         }
     }
     __device__ __forceinline__ SoftmaxState state() const
     {
         SoftmaxState st;
         st.m = m;
-        st.s = acc.s0 + acc.s1;
-        st.u = ENTROPY ? acc.u0 + acc.u1 : 0.f;
+        st.s = acc.s.x + acc.s.y;
+        st.u = ENTROPY ? acc.u.x + acc.u.y : 0.f;
         return st;
     }
 };
@@ -268,6 +302,13 @@ __device__ __forceinline__ void engine_epilogue(const EngineArgs &a, EngineSmem 
                                     (int)threadIdx.x, [] { block_sync_all<CONS>(); });
 }
 
+// sign flip of a packed gradient (both bf16 halves of each word, or each fp32 word)
+template <typename T> __device__ __forceinline__ uint4 negate_pack(uint4 v)
+{
+    const uint32_t m = sizeof(T) == 2 ? 0x80008000u : 0x80000000u;
+    return make_uint4(v.x ^ m, v.y ^ m, v.z ^ m, v.w ^ m);
+}
+
 // pass 2 of the loss for one thread's two packs of a chunk: d = -+ 2^(x*c + off), packed and stored
 template <typename T, bool NEG, int CONS>
 __device__ __forceinline__ void gradient_packs(const uint4 *buf, uint4 *dst4, int i0, int nvec, float c, float off)
@@ -275,6 +316,7 @@ __device__ __forceinline__ void gradient_packs(const uint4 *buf, uint4 *dst4, in
     constexpr int kConsumers = CONS;
     // (dst4 is the shared-memory row itself in the loss kernel: the gradient replaces the logits in place)
     constexpr int N = Pack<T>::N;
+    const float2 cc = make_float2(c, c), oo = make_float2(off, off);
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const int i = i0 + h * kConsumers;
@@ -282,11 +324,13 @@ __device__ __forceinline__ void gradient_packs(const uint4 *buf, uint4 *dst4, in
             float x[N], d[N];
             Pack<T>::unpack_raw(buf[i], x);
 #pragma unroll
-            for (int q = 0; q < N; ++q) {
-                const float e = ex2(fmaf(x[q], c, off));
-                d[q] = NEG ? -e : e;
+            for (int q = 0; q < N; q += 2) {
+                const float2 t = __ffma2_rn(make_float2(x[q], x[q + 1]), cc, oo);
+                d[q] = ex2(t.x);
+                d[q + 1] = ex2(t.y);
             }
-            dst4[i] = Pack<T>::pack(d);
+            const uint4 g = Pack<T>::pack(d);
+            dst4[i] = NEG ? negate_pack<T>(g) : g;
         }
     }
 }
