@@ -185,10 +185,21 @@ __device__ __forceinline__ void loss_prepare_block(const uint8_t *mask, int64_t 
                                                    int32_t *__restrict__ order, int *warp_tot /* 32 ints */,
                                                    bool publish /* a loss kernel may be waiting for the result */)
 {
-    const int64_t seg = (rows + kReduceThreads - 1) / kReduceThreads;
+    // segments are multiples of 16 rows so that a 16-byte aligned mask is read 16 rows per load (the result does
+    // not depend on the segment length: segments are contiguous and ascending)
+    const bool vec = (reinterpret_cast<uintptr_t>(mask) & 15) == 0;
+    int64_t seg = (rows + kReduceThreads - 1) / kReduceThreads;
+    if (vec) seg = (seg + 15) & ~(int64_t)15;
     const int64_t r0 = min(rows, (int64_t)threadIdx.x * seg), r1 = min(rows, r0 + seg);
+    const int64_t rv = vec ? r0 + ((r1 - r0) & ~(int64_t)15) : r0;   // [r0, rv): whole groups of 16 rows
     int c = 0;
-    for (int64_t r = r0; r < r1; ++r) c += mask[r] ? 1 : 0;
+#pragma unroll 4
+    for (int64_t r = r0; r < rv; r += 16) {
+        const uint4 v = *reinterpret_cast<const uint4 *>(mask + r);
+        c += (__popc(__vcmpne4(v.x, 0u)) + __popc(__vcmpne4(v.y, 0u)) + __popc(__vcmpne4(v.z, 0u)) +
+              __popc(__vcmpne4(v.w, 0u))) >> 3;
+    }
+    for (int64_t r = rv; r < r1; ++r) c += mask[r] ? 1 : 0;
     // block exclusive scan of c
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int incl = c;
@@ -218,7 +229,16 @@ __device__ __forceinline__ void loss_prepare_block(const uint8_t *mask, int64_t 
     __syncthreads();
     int real_pos = warp_tot[warp] + incl - c;            // real rows before this segment
     int64_t masked_pos = r0 - real_pos;                   // masked rows before this segment
-    for (int64_t r = r0; r < r1; ++r) {
+    for (int64_t r = r0; r < rv; r += 16) {
+        const uint4 v = *reinterpret_cast<const uint4 *>(mask + r);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+            if ((w[q >> 2] >> ((q & 3) * 8)) & 0xffu) order[real_pos++] = (int32_t)(r + q);
+            else order[rows - 1 - masked_pos++] = (int32_t)(r + q);
+        }
+    }
+    for (int64_t r = rv; r < r1; ++r) {
         if (mask[r]) order[real_pos++] = (int32_t)r;
         else order[rows - 1 - masked_pos++] = (int32_t)r;
     }
