@@ -371,8 +371,11 @@ int ppo_lmhead_bwd(const void *H, const void *W, int64_t M, int64_t K, int64_t V
  *            advantages_whitened, whiten_stats[3] (step 5); losses[8], dlogits, dvalues and the
  *            nullable new_logprob, new_entropy, dlogprob (step 6); workspace (device only)
  *
- * ppo_step: `io` is a host struct of DEVICE pointers; runs steps 2, 1 (policy), 1 (reference), 3, 4,
- * 5, 6 in that order on `stream` without synchronising.  Errors are those of the individual calls.
+ * ppo_step: `io` is a host struct of DEVICE pointers; runs steps 1 (policy and reference), 2, 3, 4,
+ * 5, 6 on `stream` without synchronising; its launches overlap where their inputs allow (the loss
+ * kernel starts while the token-level kernel runs, the token-level kernel while the log-prob kernel
+ * drains), so no output buffer may alias an input buffer or another output buffer, and one
+ * workspace serves one call at a time.  Errors are those of the individual calls.
  *
  * ppo_step_host: `host` is a host struct of HOST pointers (pinned memory makes the copies
  * asynchronous), `dev` a host struct of DEVICE pointers used as staging and output buffers.  Copies

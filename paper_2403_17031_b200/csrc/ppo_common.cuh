@@ -363,6 +363,9 @@ __device__ __forceinline__ int flag_wait(const int *flag, int *status)
 // later one may wait (flag_wait) for what it produces. The instruction does nothing when no dependent
 // launch follows.
 __device__ __forceinline__ void grid_dependents_may_launch() { asm volatile("griddepcontrol.launch_dependents;"); }
+// in a kernel launched with launch_dependent(): returns once the kernel before it has completed and its
+// writes are visible (returns at once in a kernel launched the ordinary way)
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,

@@ -83,6 +83,7 @@ logprob_pair_kernel(const T *__restrict__ policy_logits, const T *__restrict__ r
     // the hand-over flags between the two kernels that follow in ppo_step start at 0 (nothing runs beside this
     // kernel on the stream, and the next kernel starts after it has ended)
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) { flags2[0] = 0; flags2[1] = 0; }
+    grid_dependents_may_launch();   // the token-level kernel may be scheduled as this grid drains; it waits for its end
     if (blockIdx.y == 0)
         logprob_entropy_row<T, true, true, THREADS>(policy_logits, V, V, tokens, nullptr, c, logprob, entropy, nullptr,
                                                     status, red);

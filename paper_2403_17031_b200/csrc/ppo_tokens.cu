@@ -296,6 +296,10 @@ rollout_kernel(const int32_t *responses, int B, int T, int eos_id, int pad_id, c
         __syncthreads();
     }
     if (PHASE == 0) grid_dependents_may_launch();
+    // This kernel itself may have been scheduled while the log-prob kernel before it was draining. The EOS trick
+    // and the loss prologue need the sampled tokens only (an input that nothing writes), so in PHASE 0 they run
+    // before the wait for that kernel; everything that reads log-probs comes after it.
+    if (PHASE != 0) grid_dependency_wait();
 
     // tickets: the block that draws the last one continues with the batch-wide step
     const auto last_block = [&](int *counter, int n_blocks) {
@@ -351,10 +355,11 @@ rollout_kernel(const int32_t *responses, int B, int T, int eos_id, int pad_id, c
     if (b < B)
         L = truncate_sequence(responses, b, T, eos_id, pad_id, scores, no_eos_score, responses_out, eos_index, seq_len,
                               mask, scores_out, lane);
-    if (PHASE == 0) {   // tell the prologue block
+    if (PHASE == 0) {   // tell the prologue block, then wait for the log-probs
         __threadfence();
         __syncthreads();
         if (threadIdx.x == 0) atomicAdd(&hdr->step_blocks, 1);
+        grid_dependency_wait();
     }
     if (b < B) {
         int first_eos = 0;   // whether the sequence has an EOS decides the score that is used
@@ -434,7 +439,7 @@ int launch_rollout(const ppo_step_io *io, int B, int T, const ppo_params *p, boo
 {
     const unsigned nb = (unsigned)((B + kWhitenThreads / 32 - 1) / (kWhitenThreads / 32));
 #define PPO_LAUNCH_ROLLOUT(PHASE, GRID, CLEAR)                                                                       \
-    rollout_kernel<PHASE><<<GRID, kWhitenThreads, 0, s>>>(                                                           \
+    launch_dependent(rollout_kernel<PHASE>, dim3(GRID), dim3(kWhitenThreads), 0, s,                                  \
         io->responses, B, T, p->eos_id, p->pad_id, io->scores, p->no_eos_score, io->responses_out, io->eos_index,    \
         io->seq_len, io->mask, io->scores_out, io->logprob, io->ref_logprob, io->values, p->kl_coef,                 \
         (double)p->gamma, (double)p->gamma * (double)p->lam, p->whiten_eps, io->kl, io->rewards, io->advantages,     \
