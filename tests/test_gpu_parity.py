@@ -343,3 +343,45 @@ def test_reward_whitening_before_gae(P, oracle, B, T, V):
         assert_rel(npy(b.out[k]), ref[k], 5e-4, k + " (chained)")
     assert_rel(npy(b.out["advantages_whitened"]), ref["advantages_whitened"], 5e-4, "advantages_whitened (chained)")
     assert b.device_status() == 0
+
+
+@pytest.mark.parametrize("B,T,V,dtype", [(64, 53, 50304, "bf16"), (150, 53, 2048, "bf16"), (5, 16, 1001, "f32"),
+                                         (40, 512, 1000, "f32")])
+def test_step_overlapped_launches_repeatable(P, B, T, V, dtype):
+    """ppo_step's launches overlap (the loss kernel starts while the token-level kernel runs, that one while the
+    log-prob kernel drains) and hand results over through flags in the workspace. Repeated calls, eager and as a
+    replayed CUDA graph, must give the bits of the separate calls every time; V = 1001 takes the path without
+    16-byte packs (two log-prob launches, direct-load loss kernels)."""
+    import dataclasses
+    from paper_2403_17031_b200.pipeline import PPOHotPath
+    from paper_2403_17031_b200.synthetic import CONFIGS, make_batch
+    cfg = dataclasses.replace(CONFIGS[0], B=B, T=T, V=V, dtype=dtype, n_no_eos_exact=None)
+    batch = make_batch(cfg, "cuda")
+    pp = _params(P, cfg.hyper)
+    names = ("mask", "seq_len", "logprob", "entropy", "ref_logprob", "kl", "rewards", "advantages", "returns",
+             "advantages_whitened", "losses", "dlogits", "dvalues", "new_logprob", "dlogprob")
+    a = PPOHotPath(B, T, V, cfg.torch_dtype, pp)
+    o = a.rollout_stats(batch["policy_logits"], batch["ref_logits"], batch["responses"], batch["scores"], batch["values"])
+    old = (o["logprob"] + batch["old_logprob_noise"]).contiguous()
+    a.loss(batch["policy_logits"], batch["responses"], old, batch["values_new"], batch["values"])
+    torch.cuda.synchronize()
+    want = {k: a.out[k].clone() for k in names}
+    b = PPOHotPath(B, T, V, cfg.torch_dtype, pp)
+    args = (batch["policy_logits"], batch["ref_logits"], batch["responses"], batch["scores"], batch["values"],
+            batch["values_new"])
+    for it in range(3):
+        for k in names:
+            b.out[k].fill_(7)                      # stale contents must not survive
+        b.step(*args, old_logprob=old)
+        torch.cuda.synchronize()
+        for k in names:
+            assert torch.equal(b.out[k], want[k]), (k, "eager", it)
+    graph = b.capture_step(*args, old_logprob=old)
+    for it in range(3):
+        for k in names:
+            b.out[k].fill_(7)
+        graph.replay()
+        torch.cuda.synchronize()
+        for k in names:
+            assert torch.equal(b.out[k], want[k]), (k, "graph", it)
+    assert b.device_status() == 0
