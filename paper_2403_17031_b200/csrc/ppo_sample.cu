@@ -68,7 +68,8 @@ struct Race {
     // offered in increasing index order, so a strict comparison leaves ties with the lowest index
     __device__ __forceinline__ void offer(float e1, float L1, int j1)
     {
-        if (L1 * e > L * e1) { e = e1; L = L1; j = j1; }
+        const float2 pr = __fmul2_rn(make_float2(L1, L), make_float2(e, e1));   // both products in one instruction
+        if (pr.x > pr.y) { e = e1; L = L1; j = j1; }
     }
     __device__ __forceinline__ void merge(const Race &o)
     {
@@ -119,11 +120,15 @@ __device__ __forceinline__ void sums_and_race(const T *src, int V, float c, floa
                 uint32_t w[4];
                 philox4x32_10((uint32_t)(i * (N / 4) + h), row, a.off_lo, a.off_hi, keys, w);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const float t = fmaf(x[h * 4 + q], c, nm);
-                    const float e = ex2(t);
-                    if (q & 1) { s1 += e; u1 = fmaf(e, t, u1); } else { s0 += e; u0 = fmaf(e, t, u0); }
-                    best.offer(e, log2_uniform(w[q]), i * N + h * 4 + q);
+                for (int q = 0; q < 4; q += 2) {   // packed fp32x2 arithmetic: two elements per instruction
+                    const float2 t = __ffma2_rn(make_float2(x[h * 4 + q], x[h * 4 + q + 1]), make_float2(c, c),
+                                                make_float2(nm, nm));
+                    const float2 e = make_float2(ex2(t.x), ex2(t.y));
+                    const float2 sn = __fadd2_rn(make_float2(s0, s1), e);
+                    const float2 un = __ffma2_rn(e, t, make_float2(u0, u1));
+                    s0 = sn.x; s1 = sn.y; u0 = un.x; u1 = un.y;
+                    best.offer(e.x, log2_uniform(w[q]), i * N + h * 4 + q);
+                    best.offer(e.y, log2_uniform(w[q + 1]), i * N + h * 4 + q + 1);
                 }
             }
         }
