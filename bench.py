@@ -243,7 +243,7 @@ def run_ours(args, cfg):
         step()
     torch.cuda.synchronize()
 
-    # ---- timed region: K steps of the whole path (ppo_step: 5 launches per step), device-timed.
+    # ---- timed region: K steps of the whole path (ppo_step: 3 launches per step), device-timed.
     # Default: the step is recorded once into a CUDA graph and replayed K times; --eager launches it
     # call by call instead.
     K = args.steps

@@ -1,5 +1,5 @@
 // The whole path as one call (ppo_step) and its host-buffer variant (ppo_step_host): sequencing of the
-// steps (the token-level ones fused into two launches) plus the host<->device copies.
+// steps (the token-level ones fused into one launch that overlaps its neighbours) plus the host<->device copies.
 #include "ppo_common.cuh"
 
 using namespace ppo;
