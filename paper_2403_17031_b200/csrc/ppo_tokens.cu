@@ -256,11 +256,12 @@ loss_prepare_kernel(const uint8_t *__restrict__ mask, int64_t rows, WorkspaceHea
 }
 
 // ---------------------------------------------------------------- fused launch of ppo_step
-// Everything token-level in one launch, after the two log-prob calls (which do not need the mask):
-// one warp per sequence runs the EOS trick, the KL rewards and GAE; the last block to finish then
-// runs the loss prologue (token count, row order) and whitens the advantages of the whole batch,
-// each with exactly the code and thread assignment of the stand-alone kernels, so the results are
-// bit-identical to calling the steps one by one.
+// Everything token-level in one launch, after the log-prob launch (which does not need the mask):
+// one warp per sequence runs the EOS trick, the KL rewards and GAE; one extra block runs the loss
+// prologue (token count, row order) as soon as every sequence has had the EOS trick, and the last
+// sequence block to finish whitens the advantages of the whole batch - each with exactly the code and
+// thread assignment of the stand-alone kernels, so the results are bit-identical to calling the steps
+// one by one. The launch overlaps its neighbours (see grid_dependency_wait / flag_set below).
 //
 // PHASE 0: all of it. With reward whitening (detail "(Optional) Reward whitening": the rewards of the
 // batch are whitened without shifting the mean BEFORE GAE) the advantages need batch-wide statistics of
