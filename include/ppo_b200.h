@@ -238,6 +238,17 @@ int ppo_loss_from_logprob(const float *new_logprob, const float *entropy, int32_
                           float *dvalues, void *workspace, void *stream);
 
 /*
+ * Step 1 for the policy and the frozen reference in ONE launch (same tokens, same shape, row pitch V):
+ * logprob / entropy (nullable) from policy_logits, ref_logprob from ref_logits; otherwise exactly
+ * ppo_logprob_entropy called twice (which is what happens for layouts without 16-byte packs).  One
+ * launch boundary less, at which the SMs would drain and refill; with a mask, rows with mask 0 are
+ * skipped in both tensors (outputs 0).
+ */
+int ppo_logprob_entropy_pair(const void *policy_logits, const void *ref_logits, int dtype, int64_t rows, int64_t V,
+                             const int32_t *tokens, const uint8_t *mask, float temperature, float *logprob,
+                             float *entropy, float *ref_logprob, void *workspace, void *stream);
+
+/*
  * Temperature sampling fused with step 1 (Table "PPO hyperparameters": temperature): draws one token
  * per row from softmax(logits / temperature) and returns its log-prob, the row's entropy and
  * log-sum-exp from the same single pass over HBM.  The draw is reproducible and defined as follows:

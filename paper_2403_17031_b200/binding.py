@@ -91,6 +91,9 @@ _SIGS = {
                            C.c_void_p]),
     "ppo_step_host": (C.c_int, [C.POINTER(PPOStepIO), C.POINTER(PPOStepIO), C.c_int, C.c_int32, C.c_int32, C.c_int64,
                                 C.POINTER(PPOParams), C.c_void_p]),
+    "ppo_logprob_entropy_pair": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p,
+                                           C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                           C.c_void_p]),
     "ppo_sample_logprob_entropy": (C.c_int, [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_float,
                                              C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                              C.c_void_p, C.c_void_p]),
@@ -468,3 +471,24 @@ def sample_logprob_entropy(logits: torch.Tensor, temperature: float, seed: int, 
                                           _ptr(lse, torch.float32), _ptr(workspace), _stream())
     _check("ppo_sample_logprob_entropy", rc)
     return tok, lp, ent, lse
+
+
+def logprob_entropy_pair(policy_logits, ref_logits, tokens, temperature: float, mask=None, workspace=None,
+                         want_entropy: bool = True, out=None):
+    """Step 1 for policy and reference logits [..., V] (contiguous) in one launch. Returns (logprob, entropy, ref_logprob)."""
+    V = policy_logits.shape[-1]
+    rows = policy_logits.numel() // V
+    if ref_logits.shape != policy_logits.shape or ref_logits.dtype != policy_logits.dtype:
+        raise TypeError("policy and reference logits must have the same shape and dtype")
+    if out is None:
+        dev = policy_logits.device
+        out = (torch.empty(tokens.shape, dtype=torch.float32, device=dev),
+               torch.empty(tokens.shape, dtype=torch.float32, device=dev) if want_entropy else None,
+               torch.empty(tokens.shape, dtype=torch.float32, device=dev))
+    lp, ent, rlp = out
+    rc = lib().ppo_logprob_entropy_pair(_ptr(policy_logits), _ptr(ref_logits), _logits_dtype(policy_logits), rows, V,
+                                        _ptr(tokens, torch.int32), _ptr(mask, torch.uint8), float(temperature),
+                                        _ptr(lp, torch.float32), _ptr(ent, torch.float32), _ptr(rlp, torch.float32),
+                                        _ptr(workspace), _stream())
+    _check("ppo_logprob_entropy_pair", rc)
+    return lp, ent, rlp

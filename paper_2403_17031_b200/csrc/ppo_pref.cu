@@ -58,8 +58,9 @@ __device__ __forceinline__ double masked_sum(const float *__restrict__ x, const 
     return warp_sum(s);
 }
 
-// One block; warp w owns pairs w, w + 32, ...: four sequence sums, the implicit rewards, the pair's
-// loss and the per-token gradient of the MEAN loss w.r.t. the policy's token log-probs.
+// One block. Four warps share a pair (one masked sequence sum each: policy / reference x chosen / rejected), so
+// eight pairs are in flight per round; then each of the four computes the pair's terms from the four sums and two
+// of them write the per-token gradient of the MEAN loss w.r.t. the policy's token log-probs (chosen, rejected).
 __global__ void __launch_bounds__(kPrefThreads)
 dpo_loss_kernel(const float *__restrict__ lp_c, const float *__restrict__ lp_r, const float *__restrict__ ref_c,
                 const float *__restrict__ ref_r, const uint8_t *__restrict__ mask_c,
@@ -68,31 +69,48 @@ dpo_loss_kernel(const float *__restrict__ lp_c, const float *__restrict__ lp_r, 
                 float *__restrict__ dlp_r)
 {
     __shared__ double red[32];
+    __shared__ double sums[kPrefThreads / 128][4];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int slot = warp >> 2, part = warp & 3;
     const double inv_p = 1.0 / (double)P;
-    double s_loss = 0.0, s_acc = 0.0, s_c = 0.0, s_r = 0.0;   // per-warp partial sums (same value in every lane)
-    for (int64_t i = warp; i < P; i += kPrefThreads / 32) {
+    double s_loss = 0.0, s_acc = 0.0, s_c = 0.0, s_r = 0.0;   // partial sums, carried by the `part == 0` warps
+    for (int64_t i0 = 0; i0 < P; i0 += kPrefThreads / 128) {
+        const int64_t i = i0 + slot;
         const int64_t o = i * T;
-        const double rc = beta * (masked_sum(lp_c + o, mask_c + o, T, lane) - masked_sum(ref_c + o, mask_c + o, T, lane));
-        const double rr = beta * (masked_sum(lp_r + o, mask_r + o, T, lane) - masked_sum(ref_r + o, mask_r + o, T, lane));
-        double loss, sn;
-        logistic_terms(rc - rr, loss, sn);
-        s_loss += loss;
-        s_acc += rc > rr ? 1.0 : 0.0;
-        s_c += rc;
-        s_r += rr;
-        if (lane == 0) {
-            if (reward_c) reward_c[i] = (float)rc;
-            if (reward_r) reward_r[i] = (float)rr;
+        if (i < P) {
+            const float *x = part == 0 ? lp_c : (part == 1 ? ref_c : (part == 2 ? lp_r : ref_r));
+            const uint8_t *m = part < 2 ? mask_c : mask_r;
+            const double v = masked_sum(x + o, m + o, T, lane);
+            if (lane == 0) sums[slot][part] = v;
         }
-        const float gc = (float)(-beta * sn * inv_p), gr = (float)(beta * sn * inv_p);
-        for (int t = lane; t < T; t += 32) {
-            if (dlp_c) dlp_c[o + t] = mask_c[o + t] ? gc : 0.f;
-            if (dlp_r) dlp_r[o + t] = mask_r[o + t] ? gr : 0.f;
+        __syncthreads();
+        if (i < P) {
+            const double rc = beta * (sums[slot][0] - sums[slot][1]);
+            const double rr = beta * (sums[slot][2] - sums[slot][3]);
+            double loss, sn;
+            logistic_terms(rc - rr, loss, sn);
+            if (part == 0) {
+                s_loss += loss;
+                s_acc += rc > rr ? 1.0 : 0.0;
+                s_c += rc;
+                s_r += rr;
+                if (lane == 0) {
+                    if (reward_c) reward_c[i] = (float)rc;
+                    if (reward_r) reward_r[i] = (float)rr;
+                }
+                if (dlp_c) {
+                    const float gc = (float)(-beta * sn * inv_p);
+                    for (int t = lane; t < T; t += 32) dlp_c[o + t] = mask_c[o + t] ? gc : 0.f;
+                }
+            } else if (part == 2 && dlp_r) {
+                const float gr = (float)(beta * sn * inv_p);
+                for (int t = lane; t < T; t += 32) dlp_r[o + t] = mask_r[o + t] ? gr : 0.f;
+            }
         }
+        __syncthreads();   // sums[] is rewritten in the next round
     }
-    // one lane per warp carries the warp's sums into the block sums
-    const double keep = lane == 0 ? 1.0 : 0.0;
+    // one lane of every `part == 0` warp carries that warp's sums into the block sums
+    const double keep = (lane == 0 && part == 0) ? 1.0 : 0.0;
     s_loss = block_sum<kPrefThreads>(s_loss * keep, red);
     s_acc = block_sum<kPrefThreads>(s_acc * keep, red);
     s_c = block_sum<kPrefThreads>(s_c * keep, red);

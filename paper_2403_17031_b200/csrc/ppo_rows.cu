@@ -76,19 +76,20 @@ logprob_entropy_kernel(const T *__restrict__ logits, int V, int64_t row_stride, 
 template <typename T, int THREADS>
 __global__ void __launch_bounds__(THREADS)
 logprob_pair_kernel(const T *__restrict__ policy_logits, const T *__restrict__ ref_logits, int V,
-                    const int32_t *__restrict__ tokens, float c, float *__restrict__ logprob,
-                    float *__restrict__ entropy, float *__restrict__ ref_logprob, int *status, int *flags2)
+                    const int32_t *__restrict__ tokens, const uint8_t *__restrict__ mask, float c,
+                    float *__restrict__ logprob, float *__restrict__ entropy, float *__restrict__ ref_logprob,
+                    int *status, int *flags2)
 {
     __shared__ float red[96];
-    // the hand-over flags between the two kernels that follow in ppo_step start at 0 (nothing runs beside this
+    // ppo_step: the hand-over flags between the two kernels that follow start at 0 (nothing runs beside this
     // kernel on the stream, and the next kernel starts after it has ended)
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) { flags2[0] = 0; flags2[1] = 0; }
+    if (flags2 && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) { flags2[0] = 0; flags2[1] = 0; }
     grid_dependents_may_launch();   // the token-level kernel may be scheduled as this grid drains; it waits for its end
     if (blockIdx.y == 0)
-        logprob_entropy_row<T, true, true, THREADS>(policy_logits, V, V, tokens, nullptr, c, logprob, entropy, nullptr,
+        logprob_entropy_row<T, true, true, THREADS>(policy_logits, V, V, tokens, mask, c, logprob, entropy, nullptr,
                                                     status, red);
     else
-        logprob_entropy_row<T, true, false, THREADS>(ref_logits, V, V, tokens, nullptr, c, ref_logprob, nullptr,
+        logprob_entropy_row<T, true, false, THREADS>(ref_logits, V, V, tokens, mask, c, ref_logprob, nullptr,
                                                      nullptr, status, red);
 }
 
@@ -266,10 +267,10 @@ static int launch_logprob(const void *logits, int64_t rows, int V, int64_t row_s
 
 // PPO_ERR_UNSUPPORTED when the pointers or the shape do not allow 16-byte packs (the caller then makes two calls)
 int launch_logprob_pair(const void *policy_logits, const void *ref_logits, int dtype, int64_t rows, int V,
-                        const int32_t *tokens, float c, float *logprob, float *entropy, float *ref_logprob,
-                        WorkspaceHeader *hdr, cudaStream_t s)
+                        const int32_t *tokens, const uint8_t *mask, float c, float *logprob, float *entropy,
+                        float *ref_logprob, WorkspaceHeader *hdr, bool clear_flags, cudaStream_t s)
 {
-    int *status = &hdr->status, *flags2 = &hdr->order_ready;
+    int *status = hdr ? &hdr->status : nullptr, *flags2 = (hdr && clear_flags) ? &hdr->order_ready : nullptr;
     static_assert(offsetof(WorkspaceHeader, adv_ready) == offsetof(WorkspaceHeader, order_ready) + sizeof(int),
                   "the two flags are cleared as a pair");
     constexpr int THREADS = 256;
@@ -280,12 +281,12 @@ int launch_logprob_pair(const void *policy_logits, const void *ref_logits, int d
     const dim3 grid((unsigned)rows, 2);
     if (dtype == PPO_F32)
         logprob_pair_kernel<float, THREADS><<<grid, THREADS, 0, s>>>(
-            reinterpret_cast<const float *>(policy_logits), reinterpret_cast<const float *>(ref_logits), V, tokens, c,
-            logprob, entropy, ref_logprob, status, flags2);
+            reinterpret_cast<const float *>(policy_logits), reinterpret_cast<const float *>(ref_logits), V, tokens, mask,
+            c, logprob, entropy, ref_logprob, status, flags2);
     else
         logprob_pair_kernel<__nv_bfloat16, THREADS><<<grid, THREADS, 0, s>>>(
             reinterpret_cast<const __nv_bfloat16 *>(policy_logits), reinterpret_cast<const __nv_bfloat16 *>(ref_logits),
-            V, tokens, c, logprob, entropy, ref_logprob, status, flags2);
+            V, tokens, mask, c, logprob, entropy, ref_logprob, status, flags2);
     return launch_status();
 }
 
@@ -470,4 +471,29 @@ extern "C" int ppo_logprob_bwd(const void *logits, int dtype, int64_t rows, int6
     rc = dtype == PPO_F32 ? launch_loss<float>(a, s) : launch_loss<__nv_bfloat16>(a, s);
     if (rc) return rc;
     return launch_loss_finalize(rows, 0.f, sink, workspace, s);
+}
+
+extern "C" int ppo_logprob_entropy_pair(const void *policy_logits, const void *ref_logits, int dtype, int64_t rows,
+                                        int64_t V, const int32_t *tokens, const uint8_t *mask, float temperature,
+                                        float *logprob, float *entropy, float *ref_logprob, void *workspace,
+                                        void *stream)
+{
+    if (dtype != PPO_F32 && dtype != PPO_BF16) return PPO_ERR_DTYPE;
+    if (rows < 0 || rows >= ((int64_t)1 << 31) || V <= 0 || V >= ((int64_t)1 << 31)) return PPO_ERR_SHAPE;
+    if (!(temperature > 0.f) || !finite_f(temperature)) return PPO_ERR_PARAM;
+    if (rows == 0) return PPO_OK;
+    if (!policy_logits || !ref_logits || !tokens || !logprob || !ref_logprob) return PPO_ERR_NULL;
+    const size_t es = dtype == PPO_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(policy_logits) % es || reinterpret_cast<uintptr_t>(ref_logits) % es)
+        return PPO_ERR_ALIGN;
+    int rc = launch_logprob_pair(policy_logits, ref_logits, dtype, rows, (int)V, tokens, mask, kLog2e / temperature,
+                                 logprob, entropy, ref_logprob, workspace ? ws_header(workspace) : nullptr, false,
+                                 reinterpret_cast<cudaStream_t>(stream));
+    if (rc != PPO_ERR_UNSUPPORTED) return rc;
+    // no 16-byte packs in this layout: one launch per tensor
+    rc = ppo_logprob_entropy(policy_logits, dtype, rows, V, V, tokens, mask, temperature, logprob, entropy, nullptr,
+                             workspace, stream);
+    if (rc) return rc;
+    return ppo_logprob_entropy(ref_logits, dtype, rows, V, V, tokens, mask, temperature, ref_logprob, nullptr, nullptr,
+                               workspace, stream);
 }

@@ -28,9 +28,9 @@ extern "C" int ppo_step(const ppo_step_io *io, int dtype, int32_t B, int32_t T, 
     int rc = PPO_ERR_UNSUPPORTED;
     if ((dtype == PPO_F32 || dtype == PPO_BF16) && V < ((int64_t)1 << 31) && p->temperature > 0.f &&
         finite_f(p->temperature) && option_value(PPO_OPT_ROW_ENGINE) != 2)
-        rc = launch_logprob_pair(io->policy_logits, io->ref_logits, dtype, rows, (int)V, io->responses,
+        rc = launch_logprob_pair(io->policy_logits, io->ref_logits, dtype, rows, (int)V, io->responses, nullptr,
                                  kLog2e / p->temperature, io->logprob, io->entropy, io->ref_logprob,
-                                 ws_header(io->workspace), s);
+                                 ws_header(io->workspace), true, s);
     const bool flags_cleared = rc == PPO_OK;
     if (rc == PPO_ERR_UNSUPPORTED) {   // layout without 16-byte packs (or the row engine was asked for): two calls
         rc = ppo_logprob_entropy(io->policy_logits, dtype, rows, V, V, io->responses, nullptr, p->temperature,

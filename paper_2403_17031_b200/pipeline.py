@@ -131,10 +131,8 @@ class DPOStep:
 
     def step(self, policy_logits, ref_logits, tokens, mask):
         o = self.out
-        _b.logprob_entropy(policy_logits, tokens, 1.0, mask=mask, workspace=self.workspace, want_entropy=False,
-                           out=(o["logprob"], None, None))
-        _b.logprob_entropy(ref_logits, tokens, 1.0, mask=mask, workspace=self.workspace, want_entropy=False,
-                           out=(o["ref_logprob"], None, None))
+        _b.logprob_entropy_pair(policy_logits, ref_logits, tokens, 1.0, mask=mask, workspace=self.workspace,
+                                out=(o["logprob"], None, o["ref_logprob"]))
         _b.dpo_loss(o["logprob"][0], o["logprob"][1], o["ref_logprob"][0], o["ref_logprob"][1], mask[0], mask[1],
                     self.beta, out={"out4": o["out4"], "reward_c": o["reward_c"], "reward_r": o["reward_r"],
                                     "dlp_c": o["dlogprob"][0], "dlp_r": o["dlogprob"][1]})

@@ -148,3 +148,18 @@ def test_dpo_step_chained(P, oracle):
     assert not got[m.reshape(-1) == 0].any()
     assert_abs(n * got, n * want, 2e-3, "P * dlogits (chained)")
     assert st.device_status() == 0
+
+
+def test_logprob_entropy_pair_equals_two_calls(P):
+    """One launch for policy and reference logits (with and without a mask) gives the bits of two separate calls;
+    V = 1001 takes the layout without 16-byte packs (two launches inside)."""
+    g = torch.Generator(device="cuda").manual_seed(21)
+    for dtype, rows, V in ((torch.bfloat16, 300, 2048), (torch.float32, 77, 1000), (torch.float32, 9, 1001)):
+        x = (2.0 * torch.randn((rows, V), generator=g, device="cuda")).to(dtype)
+        y = (x.float() + 0.3 * torch.randn((rows, V), generator=g, device="cuda")).to(dtype)
+        tok = torch.randint(0, V, (rows,), generator=g, device="cuda", dtype=torch.int32)
+        for mask in (None, (torch.rand((rows,), generator=g, device="cuda") < 0.3).to(torch.uint8)):
+            lp, ent, _ = P.logprob_entropy(x, tok, 0.7, mask=mask)
+            rlp, _, _ = P.logprob_entropy(y, tok, 0.7, mask=mask, want_entropy=False)
+            lp2, ent2, rlp2 = P.logprob_entropy_pair(x, y, tok, 0.7, mask=mask)
+            assert torch.equal(lp, lp2) and torch.equal(ent, ent2) and torch.equal(rlp, rlp2)

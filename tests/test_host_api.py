@@ -154,6 +154,12 @@ def test_argument_errors_of_the_widened_entry_points(L):
     assert call(lb, ok, _8=P(FAKE)) == -3                 # in place is not supported
     assert call(lb, ok, _11=P(FAKE + 64)) == -4
 
+    lpp = L.ppo_logprob_entropy_pair
+    okq = [P(FAKE), P(FAKE), b.PPO_BF16, 64, 1000, P(FAKE), None, 0.7, P(FAKE), None, P(FAKE), None, None]
+    assert call(lpp, okq, _2=4) == -5 and call(lpp, okq, _4=0) == -2 and call(lpp, okq, _7=0.0) == -3
+    assert call(lpp, okq, _1=None) == -1 and call(lpp, okq, _10=None) == -1 and call(lpp, okq, _3=0) == 0
+    assert call(lpp, okq, _0=P(FAKE + 1)) == -4
+
     pw = L.ppo_pairwise_loss
     okp = [P(FAKE), P(FAKE), 8, P(FAKE), None, None, None]
     assert call(pw, okp, _2=0) == -2 and call(pw, okp, _0=None) == -1 and call(pw, okp, _3=None) == -1
