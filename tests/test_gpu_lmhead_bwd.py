@@ -127,3 +127,17 @@ def test_lmhead_bwd_config4_full_size_sampled(P):
     rhs = (H.double() @ u) @ Dc
     scale = (H.double().abs() @ u.abs()) @ Dc.abs()      # sum_k |u_k| (|H|^T |D|)[k, v]: the scale of dW's rounding
     assert float(((lhs - rhs).abs() / scale.clamp_min(1e-30)).max()) < 2.0 ** -8
+
+
+def test_lmhead_bwd_all_rows_masked(P):
+    M, K, V = 200, 128, 1000
+    H = torch.randn((M, K), device="cuda").to(torch.bfloat16)
+    W = torch.randn((K, V), device="cuda").to(torch.bfloat16)
+    tok = torch.randint(0, V, (M,), device="cuda", dtype=torch.int32)
+    ws = P.new_workspace(P.lmhead_workspace_bytes(M, K, V))
+    _, _, lse = P.lmhead_logprob_entropy(H, W, tok, 0.7, ws, want_lse=True)
+    o = P.lmhead_bwd(H, W, tok, lse, torch.ones(M, device="cuda"), 0.7, ws,
+                     mask=torch.zeros(M, dtype=torch.uint8, device="cuda"))
+    torch.cuda.synchronize()
+    assert not o["dlogits"].float().any() and not o["dH"].float().any() and not o["dW"].float().any()
+    assert P.last_device_status(ws) == 0

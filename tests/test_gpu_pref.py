@@ -163,3 +163,21 @@ def test_logprob_entropy_pair_equals_two_calls(P):
             rlp, _, _ = P.logprob_entropy(y, tok, 0.7, mask=mask, want_entropy=False)
             lp2, ent2, rlp2 = P.logprob_entropy_pair(x, y, tok, 0.7, mask=mask)
             assert torch.equal(lp, lp2) and torch.equal(ent, ent2) and torch.equal(rlp, rlp2)
+
+
+def test_degenerate_shapes(P, oracle):
+    """One pair of one token; a backward call whose mask selects no row (everything zero, status bit set)."""
+    o = P.dpo_loss(*(dev(np.array([[v]], np.float32)) for v in (-1.0, -2.0, -1.5, -1.0)),
+                   dev(np.ones((1, 1), np.uint8)), dev(np.ones((1, 1), np.uint8)), 0.5)
+    ref = R.dpo_loss([[-1.0]], [[-2.0]], [[-1.5]], [[-1.0]], np.ones((1, 1)), np.ones((1, 1)), 0.5)
+    assert abs(float(o["out4"][0]) - ref["loss"]) < 1e-6 and float(o["out4"][1]) == ref["accuracy"]
+    assert_abs(npy(o["dlp_c"]), ref["dlp_c"], 1e-6, "dlp_c")
+    rows, V = 40, 2048
+    x = torch.randn((rows, V), device="cuda").to(torch.bfloat16)
+    tok = torch.zeros(rows, dtype=torch.int32, device="cuda")
+    ws = P.new_workspace(P.workspace_bytes(rows, 1, V))
+    out = P.logprob_bwd(x, tok, torch.zeros(rows, dtype=torch.uint8, device="cuda"), torch.ones(rows, device="cuda"),
+                        1.0, ws, want_aux=True)
+    torch.cuda.synchronize()
+    assert not out["dlogits"].float().any() and not out["new_logprob"].any()
+    assert P.last_device_status(ws) == 2                                  # PPO_DEV_EMPTY_MASK

@@ -104,3 +104,18 @@ def test_rows_far_above_their_first_pack_take_the_exact_maximum(P, oracle):
     _compare(P, oracle, x, 0.7, seed=77)
     xb = x.to(torch.bfloat16)
     _compare(P, oracle, xb, 0.7, seed=78)
+
+
+def test_tiny_rows_and_odd_widths(P, oracle):
+    g = torch.Generator(device="cuda").manual_seed(4)
+    for dtype, rows, V in ((torch.float32, 1, 8), (torch.float32, 3, 5), (torch.bfloat16, 2, 16), (torch.bfloat16, 5, 37)):
+        x = torch.randn((rows, V), generator=g, device="cuda").to(dtype)
+        ws = P.new_workspace(P.workspace_bytes(rows, 1, V))
+        tok, lp, ent, lse = P.sample_logprob_entropy(x, 0.7, 99, workspace=ws, want_lse=True)
+        want, keys = S.sample(x.double().cpu().numpy(), 0.7, 99)
+        t = npy(tok).astype(np.int64)
+        assert (keys.max(axis=1) - keys[np.arange(rows), t] <= GAP).all()
+        o_lp, o_ent, o_lse = oracle.logprob_entropy(host_logits(x), t.astype(np.int32), 0.7)
+        assert_abs(npy(lp), o_lp, TOL_LOGPROB, "logprob")
+        assert_abs(npy(ent), o_ent, TOL_LOGPROB, "entropy")
+        assert P.last_device_status(ws) == 0
