@@ -2,7 +2,7 @@
 // by tile on the 5th-generation tensor cores and consumed straight out of tensor memory; they are
 // never written to global memory.
 //
-// One persistent block per SM, 192 threads in three roles:
+// One persistent block per SM, 192 threads (320 when a work unit covers two row tiles, see LmShape) in three roles:
 //   warp 0 (one lane)   TMA producer: 128x64 tiles of H (K-major) and 64x256 tiles of W (vocabulary-
 //                       major, as stored: W is [K,V] row-major) into a 4-stage shared-memory ring,
 //                       128-byte swizzle, completion counted on mbarriers
@@ -29,12 +29,21 @@
 namespace ppo {
 
 constexpr int kBlockM = 128, kBlockN = 256, kBlockK = 64;
-constexpr int kStages = 4;
+constexpr int kMaxStages = 4;
 constexpr int kABytes = kBlockM * kBlockK * 2;          // 16 KB
 constexpr int kBBoxBytes = 64 * kBlockK * 2;            // 8 KB: one 64(N) x 64(K) box of W
 constexpr int kBBytes = (kBlockN / 64) * kBBoxBytes;    // 32 KB
-constexpr int kStageBytes = kABytes + kBBytes;          // 48 KB
-constexpr int kLmThreads = 192;
+// MT = row tiles of 128 that one work unit multiplies with the same W tile. MT = 2 (the default for
+// M > 128): two accumulators of 256 columns fill the tensor memory, every W tile staged in shared memory
+// feeds two MMAs, and the ring moves 64 KB instead of 96 KB per 2 x (128 x 256 x 64) multiply-adds - the
+// ring, not the tensor pipe, is what limits this kernel. The price: no second accumulator set, so the
+// epilogue (eight warps, four per accumulator) is not hidden behind the next tile's MMAs.
+template <int MT> struct LmShape {
+    static constexpr int kStages = MT == 1 ? 4 : 3;
+    static constexpr int kStageBytes = MT * kABytes + kBBytes;      // 48 KB / 64 KB
+    static constexpr int kThreads = 64 + MT * 128;                  // TMA warp, MMA warp, 4 * MT epilogue warps
+    static constexpr int kSets = MT == 1 ? 2 : 1;                   // accumulator sets in the 512 columns
+};
 constexpr int kTilesPerChunk = 6;                       // vocabulary tiles per work unit
 constexpr int kRowGroup = 37;                           // row tiles that sweep the vocabulary together
 constexpr int kTmemCols = 512;
@@ -42,7 +51,7 @@ constexpr uint32_t kLmWaitTries = 1u << 19;         // x up to ~2 us per try
 constexpr uint32_t kAbsentBits = 0xffffffffu;           // "this chunk does not hold the sampled token"
 
 struct LmSmem {
-    unsigned long long full[kStages], empty[kStages], tmem_full[2], tmem_empty[2];
+    unsigned long long full[kMaxStages], empty[kMaxStages], tmem_full[2], tmem_empty[2];
     uint32_t tmem_base;
 };
 
@@ -151,9 +160,11 @@ struct LmArgs {
     int *status;
 };
 
-__global__ void __launch_bounds__(kLmThreads, 1)
+template <int MT>
+__global__ void __launch_bounds__(LmShape<MT>::kThreads, 1)
 lmhead_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w, const LmArgs a)
 {
+    constexpr int kStages = LmShape<MT>::kStages, kStageBytes = LmShape<MT>::kStageBytes, kSets = LmShape<MT>::kSets;
     extern __shared__ __align__(1024) unsigned char lm_smem_raw[];
     __shared__ LmSmem sm;
     // the ring must start on a 1024-byte boundary (swizzle atoms)
@@ -168,7 +179,8 @@ lmhead_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__
         }
         for (int b = 0; b < 2; ++b) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(lm_smem_addr(&sm.tmem_full[b])) : "memory");
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 4;" ::"r"(lm_smem_addr(&sm.tmem_empty[b])) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(lm_smem_addr(&sm.tmem_empty[b])), "r"(4 * MT)
+                         : "memory");
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -198,11 +210,14 @@ lmhead_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__
                         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(lm_smem_addr(&sm.full[s])),
                                      "r"((uint32_t)kStageBytes)
                                      : "memory");
-                        tma_load_2d(stage, &map_h, kb * kBlockK, un.m_tile * kBlockM, &sm.full[s]);
+#pragma unroll
+                        for (int j = 0; j < MT; ++j)   // (a tile past the last row is filled with zeros)
+                            tma_load_2d(stage + j * kABytes, &map_h, kb * kBlockK, (un.m_tile * MT + j) * kBlockM,
+                                        &sm.full[s]);
 #pragma unroll
                         for (int j = 0; j < kBlockN / 64; ++j)
-                            tma_load_2d(stage + kABytes + j * kBBoxBytes, &map_w, t * kBlockN + j * 64, kb * kBlockK,
-                                        &sm.full[s]);
+                            tma_load_2d(stage + MT * kABytes + j * kBBoxBytes, &map_w, t * kBlockN + j * 64,
+                                        kb * kBlockK, &sm.full[s]);
                     }
                 }
             }
@@ -216,24 +231,27 @@ lmhead_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__
                 const LmUnit un = lm_unit(u, a.m_tiles, a.n_chunks);
                 const int t0 = un.chunk * kTilesPerChunk, t1 = min(t0 + kTilesPerChunk, a.n_tiles);
                 for (int t = t0; t < t1; ++t, ++tc) {
-                    const uint32_t buf = tc & 1;
-                    if (tc >= 2) lm_wait(&sm.tmem_empty[buf], ((tc >> 1) - 1) & 1, a.status);
+                    const uint32_t buf = tc % kSets;
+                    if (tc >= (uint32_t)kSets) lm_wait(&sm.tmem_empty[buf], ((tc / kSets) - 1) & 1, a.status);
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t tmem_d = tmem_base + buf * kBlockN;
+                    const uint32_t tmem_d = tmem_base + buf * (MT * kBlockN);
                     for (int kb = 0; kb < k_blocks; ++kb, ++it) {
                         const int s = it % kStages;
                         lm_wait(&sm.full[s], (it / kStages) & 1, a.status);
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                         const uint32_t a_addr = lm_smem_addr(ring + (size_t)s * kStageBytes);
-                        const uint32_t b_addr = a_addr + kABytes;
+                        const uint32_t b_addr = a_addr + MT * kABytes;
 #pragma unroll
                         for (int kk = 0; kk < kBlockK / 16; ++kk) {
-                            // A: K-major, 8-row groups 1024 B apart; 16 K-elements = 32 bytes further
-                            const uint64_t ad = smem_desc(a_addr + kk * 32, 16, 1024);
                             // B: vocabulary-major; 64-column boxes 8192 B apart, 8 K-rows 1024 B apart;
                             //    16 K-rows = 2048 bytes further
                             const uint64_t bd = smem_desc(b_addr + kk * 2048, kBBoxBytes, 1024);
-                            umma(tmem_d, ad, bd, (kb | kk) ? 1u : 0u);
+#pragma unroll
+                            for (int j = 0; j < MT; ++j) {
+                                // A: K-major, 8-row groups 1024 B apart; 16 K-elements = 32 bytes further
+                                const uint64_t ad = smem_desc(a_addr + j * kABytes + kk * 32, 16, 1024);
+                                umma(tmem_d + j * kBlockN, ad, bd, (kb | kk) ? 1u : 0u);
+                            }
                         }
                         umma_commit(&sm.empty[s]);            // ring slot is free once these MMAs have read it
                     }
@@ -245,22 +263,23 @@ lmhead_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..5)
         const int q = warp & 3;                      // tensor-memory lane quarter this warp may read
+        const int acc = (warp - 2) >> 2;             // which of the unit's MT accumulators / row tiles
         const int row_in_tile = q * 32 + lane;
         uint32_t tc = 0;
         for (int u = blockIdx.x; u < a.n_units; u += gridDim.x) {
             const LmUnit un = lm_unit(u, a.m_tiles, a.n_chunks);
             const int t0 = un.chunk * kTilesPerChunk, t1 = min(t0 + kTilesPerChunk, a.n_tiles);
-            const int row = un.m_tile * kBlockM + row_in_tile;
+            const int row = (un.m_tile * MT + acc) * kBlockM + row_in_tile;
             const bool row_ok = row < a.M;
             const int tok = row_ok ? a.tokens[row] : -1;
             float m = 0.f, s0 = 0.f, s1 = 0.f, u0 = 0.f, u1 = 0.f;
             bool have_ref = false;
             uint32_t xtok_bits = kAbsentBits;
             for (int t = t0; t < t1; ++t, ++tc) {
-                const uint32_t buf = tc & 1;
-                lm_wait(&sm.tmem_full[buf], (tc >> 1) & 1, a.status);
+                const uint32_t buf = tc % kSets;
+                lm_wait(&sm.tmem_full[buf], (tc / kSets) & 1, a.status);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t taddr = tmem_base + buf * kBlockN + ((uint32_t)(q * 32) << 16);
+                const uint32_t taddr = tmem_base + buf * (MT * kBlockN) + acc * kBlockN + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
                 for (int cc = 0; cc < kBlockN / 32; ++cc) {
                     uint32_t r[32];
@@ -469,10 +488,20 @@ extern "C" int ppo_lmhead_logprob_entropy(const void *H, const void *W, int64_t 
     int dev = 0, sms = 148;
     PPO_RETURN_IF_CUDA(cudaGetDevice(&dev));
     PPO_RETURN_IF_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    const size_t smem = (size_t)kStages * kStageBytes + 1024;   // + slack to align the ring to 1024 bytes
-    PPO_RETURN_IF_CUDA(cudaFuncSetAttribute(lmhead_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    const int grid = a.n_units < sms ? a.n_units : sms;
-    lmhead_kernel<<<grid, kLmThreads, smem, s>>>(map_h, map_w, a);
+    if (a.m_tiles >= 2) {
+        // two row tiles per unit: the unit grid is over pairs of row tiles
+        a.m_tiles = (a.m_tiles + 1) / 2;
+        a.n_units = a.m_tiles * a.n_chunks;
+        const size_t smem = (size_t)LmShape<2>::kStages * LmShape<2>::kStageBytes + 1024;   // + slack to align the ring
+        PPO_RETURN_IF_CUDA(cudaFuncSetAttribute(lmhead_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        const int grid = a.n_units < sms ? a.n_units : sms;
+        lmhead_kernel<2><<<grid, LmShape<2>::kThreads, smem, s>>>(map_h, map_w, a);
+    } else {
+        const size_t smem = (size_t)LmShape<1>::kStages * LmShape<1>::kStageBytes + 1024;
+        PPO_RETURN_IF_CUDA(cudaFuncSetAttribute(lmhead_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        const int grid = a.n_units < sms ? a.n_units : sms;
+        lmhead_kernel<1><<<grid, LmShape<1>::kThreads, smem, s>>>(map_h, map_w, a);
+    }
     rc = launch_status();
     if (rc) return rc;
     lmhead_finalize_kernel<<<(unsigned)((M + 255) / 256), 256, 0, s>>>(a.partials, a.M, a.V, a.n_chunks, tokens, mask, a.c,
