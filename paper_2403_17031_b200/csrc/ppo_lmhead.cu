@@ -488,8 +488,9 @@ extern "C" int ppo_lmhead_logprob_entropy(const void *H, const void *W, int64_t 
     int dev = 0, sms = 148;
     PPO_RETURN_IF_CUDA(cudaGetDevice(&dev));
     PPO_RETURN_IF_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    if (a.m_tiles >= 2) {
-        // two row tiles per unit: the unit grid is over pairs of row tiles
+    // two row tiles per unit pay off when the units still spread evenly over the SMs (a unit is twice as long)
+    if (a.m_tiles >= 2 && (int64_t)((a.m_tiles + 1) / 2) * a.n_chunks >= 12 * (int64_t)sms) {
+        // the unit grid is over pairs of row tiles
         a.m_tiles = (a.m_tiles + 1) / 2;
         a.n_units = a.m_tiles * a.n_chunks;
         const size_t smem = (size_t)LmShape<2>::kStages * LmShape<2>::kStageBytes + 1024;   // + slack to align the ring
