@@ -422,7 +422,7 @@ int ppo::loss_fwd_bwd_prepared(const void *logits, int dtype, int32_t B, int32_t
     a.c1 = p->vf_coef;
     rc = PPO_ERR_UNSUPPORTED;
     if (option_value(PPO_OPT_ROW_ENGINE) != 1) {
-        rc = launch_loss_bulk(a, dtype, workspace, losses, p->vf_coef, prepared, s);
+        rc = launch_loss_bulk(a, dtype, workspace, losses, p->vf_coef, true, s);
         if (rc != PPO_ERR_UNSUPPORTED) return rc;      // the engine reduces the partials itself
     }
     rc = dtype == PPO_F32 ? launch_loss<float>(a, s) : launch_loss<__nv_bfloat16>(a, s);
@@ -465,7 +465,7 @@ extern "C" int ppo_logprob_bwd(const void *logits, int dtype, int64_t rows, int6
     float *sink = reinterpret_cast<float *>(ws_header(workspace)->reserved);
     rc = PPO_ERR_UNSUPPORTED;
     if (option_value(PPO_OPT_ROW_ENGINE) != 1) {
-        rc = launch_loss_bulk(a, dtype, workspace, sink, 0.f, false, s);
+        rc = launch_loss_bulk(a, dtype, workspace, sink, 0.f, true, s);
         if (rc != PPO_ERR_UNSUPPORTED) return rc;
     }
     rc = dtype == PPO_F32 ? launch_loss<float>(a, s) : launch_loss<__nv_bfloat16>(a, s);

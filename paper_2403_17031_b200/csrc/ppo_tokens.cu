@@ -252,7 +252,17 @@ __global__ void __launch_bounds__(kReduceThreads)
 loss_prepare_kernel(const uint8_t *__restrict__ mask, int64_t rows, WorkspaceHeader *hdr, int32_t *__restrict__ order)
 {
     __shared__ int warp_tot[32];
-    loss_prepare_block(mask, rows, hdr, order, warp_tot, false);
+    // the loss kernel that follows is launched as a programmatic dependent: it may start now and waits on the
+    // two flags, which are cleared before this (only) block lets it launch
+    if (threadIdx.x == 0) {
+        hdr->order_ready = 0;
+        hdr->adv_ready = 0;
+        __threadfence();
+    }
+    __syncthreads();
+    grid_dependents_may_launch();
+    loss_prepare_block(mask, rows, hdr, order, warp_tot, true);
+    if (threadIdx.x == 0) flag_set(&hdr->adv_ready);   // stand-alone loss call: its other inputs exist already
 }
 
 // ---------------------------------------------------------------- fused launch of ppo_step
