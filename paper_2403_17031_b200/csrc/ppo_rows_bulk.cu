@@ -8,12 +8,17 @@
 //     next row's bytes stream in behind the pass that is still consuming the current row: the
 //     block never drains its loads at a row boundary;
 //   * step 1 (log-prob/entropy) makes one pass and releases chunks as it goes; step 6 (loss)
-//     keeps the row for a second pass that writes the gradient with 16-byte streaming stores and
-//     releases the chunks there. Rows whose mask is 0 are only zero-filled: a filler thread per
-//     block takes them from a shared work counter and writes them with bulk shared->global
-//     copies of a small block of zeros while the consumers work on real rows (the real-row
-//     phase alone leaves HBM bandwidth idle); consumers that run out of real rows join in;
-//   * two blocks per SM while a row is <= 112 KB (bf16, V = 50304), one otherwise.
+//     keeps the row for a second pass that writes the gradient IN PLACE over the logits in shared
+//     memory; the producer ships each finished chunk with one bulk shared->global copy and refills
+//     the space, one chunk behind, with the next row. Rows whose mask is 0 are only zero-filled: a
+//     filler thread per block takes them from a shared work counter and writes them with bulk
+//     shared->global copies of a small block of zeros while the consumers work on real rows (the
+//     real-row phase alone leaves HBM bandwidth idle); consumers that run out of real rows join in;
+//   * step 6 hands its rows out dynamically (a counter in the workspace header; the row index reaches
+//     the consumers through a small ring in shared memory), since SMs do not stream at equal speed;
+//   * two blocks per SM while a row is <= 110 KB (bf16, V = 50304), one otherwise;
+//   * step 6 may be launched while the kernel that produces its row order and advantages is still
+//     running (programmatic dependent launch): it then polls two flags of the workspace header.
 //
 // Every wait is bounded: when it runs out the block records PPO_DEV_TIMEOUT in the status word
 // and carries on with the same control flow (so no barrier is left short), which makes the
@@ -35,7 +40,6 @@ struct EngineSmem {
     unsigned long long full[kMaxChunks];
     unsigned long long empty[kMaxChunks];
     float red[2][96];      // by row parity: a row's sums are read while the next row's are written
-    float bc[4];
     int next_item;
     int is_last;
     int ring[4];           // row of the block's k-th item at [k % 4], -1 = no further item
