@@ -151,8 +151,8 @@ def _oracle_chain_time(cfg, inp):
     f32 = lambda a: np.asarray(a, np.float64).astype(np.float32)
     t0 = time.perf_counter()
     _, _, L, m, so = O.truncate_and_score(resp, h.eos_id, h.pad_id, inp["scores"], np.float32(h.no_eos_score))
-    lp, _, _ = O.logprob_entropy(pl.reshape(-1, V), resp, tau)
-    rlp, _, _ = O.logprob_entropy(rl.reshape(-1, V), resp, tau)
+    lp, _, _ = O.logprob_entropy(pl.reshape(-1, V), resp, tau, mask=m.reshape(-1))    # padding rows: not read, 0
+    rlp, _, _ = O.logprob_entropy(rl.reshape(-1, V), resp, tau, mask=m.reshape(-1))
     lp, rlp = lp.reshape(resp.shape), rlp.reshape(resp.shape)
     _, rew = O.kl_rewards(f32(lp), f32(rlp), m, L, f32(so), np.float32(h.kl_coef))
     adv, ret = O.gae(f32(rew), inp["values"], L, np.float32(h.gamma), np.float32(h.lam))
@@ -308,7 +308,8 @@ def run_ours(args, cfg):
     loss_bytes = n_real * V * esize + B * T * V * esize
     loss_gbs = loss_bytes / (loss_ms * 1e-3) / 1e9
     lp_gbs = R / (lp_ms * 1e-3) / 1e9
-    path_bytes = 2 * R + loss_bytes
+    # the step reads the logits of the real rows only (policy, reference, loss) and writes every gradient row
+    path_bytes = 2 * n_real * V * esize + loss_bytes
 
     # ---- end to end: inputs start in pinned host memory, results are read back to the host
     e2e = None
@@ -374,8 +375,9 @@ def run_ours(args, cfg):
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": "config%d %s" % (cfg.index, cfg.name), "B_per_gpu": B, "T": T, "V": V,
                        "logits_dtype": cfg.dtype, "real_tokens": n_real,
-                       "l2": "inputs larger than L2 (%.0f MB of logits read + %.0f MB written per step)" %
-                             (2 * R / 1e6, R / 1e6),
+                       "l2": "inputs larger than L2 (%.0f MB of logits read on the %d real rows, 3 tensors, + %.0f MB "
+                             "of gradient written per step; padding rows are not read)" %
+                             (3 * n_real * V * esize / 1e6, n_real, R / 1e6),
                        "path_hbm_gbs": path_bytes / (ms_per_step * 1e-3) / 1e9,
                        "path_hbm_frac_of_8tbs": path_bytes / (ms_per_step * 1e-3) / 8e12,
                        "logprob_entropy_ms": lp_ms, "logprob_entropy_gbs": lp_gbs,

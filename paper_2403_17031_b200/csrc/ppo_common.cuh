@@ -400,10 +400,11 @@ int loss_fwd_bwd_prepared(const void *logits, int dtype, int32_t B, int32_t T, i
                           float *dlogprob, void *workspace, void *stream, bool prepared);
 int launch_loss_prepare(const uint8_t *mask, int64_t rows, void *workspace, cudaStream_t s);
 // step 1 for policy and reference logits in one launch; PPO_ERR_UNSUPPORTED if the layout rules it out
-// (also clears the two hand-over flags of the header for the kernels that follow in ppo_step)
+// (also clears the two hand-over flags of the header for the kernels that follow in ppo_step).
+// seq_T > 0: rows = B * seq_T responses, and rows after a sequence's first eos_id are padding (skipped, outputs 0)
 int launch_logprob_pair(const void *policy_logits, const void *ref_logits, int dtype, int64_t rows, int V,
-                        const int32_t *tokens, const uint8_t *mask, float c, float *logprob, float *entropy,
-                        float *ref_logprob, WorkspaceHeader *hdr, bool clear_flags, cudaStream_t s);
+                        const int32_t *tokens, const uint8_t *mask, int seq_T, int eos_id, float c, float *logprob,
+                        float *entropy, float *ref_logprob, WorkspaceHeader *hdr, bool clear_flags, cudaStream_t s);
 // flags_cleared: the launch before this one has cleared the header's hand-over flags already
 int launch_rollout(const ppo_step_io *io, int B, int T, const ppo_params *p, bool flags_cleared, cudaStream_t s);
 int launch_loss_finalize(int64_t rows, float vf_coef, float *losses, void *workspace, cudaStream_t s);

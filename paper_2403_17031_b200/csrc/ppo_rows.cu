@@ -73,18 +73,39 @@ logprob_entropy_kernel(const T *__restrict__ logits, int V, int64_t row_stride, 
 // Step 1 for the policy and the frozen reference in one launch (grid.y = 2): same tokens, same shape.
 // y = 0: policy logits -> log-prob and entropy; y = 1: reference logits -> log-prob only. One launch
 // instead of two saves a launch boundary, at which the SMs drain and refill.
+// seq_T > 0: the rows are [B, seq_T] responses and everything after a sequence's first EOS is padding (the EOS
+// trick of the paper's detail "EOS trick"; the token-level kernel that follows writes the same mask): such a
+// row's logits are not read and its outputs are 0, as with mask[row] == 0.
 template <typename T, int THREADS>
 __global__ void __launch_bounds__(THREADS)
 logprob_pair_kernel(const T *__restrict__ policy_logits, const T *__restrict__ ref_logits, int V,
-                    const int32_t *__restrict__ tokens, const uint8_t *__restrict__ mask, float c,
-                    float *__restrict__ logprob, float *__restrict__ entropy, float *__restrict__ ref_logprob,
-                    int *status, int *flags2)
+                    const int32_t *__restrict__ tokens, const uint8_t *__restrict__ mask, int seq_T, int eos_id,
+                    float c, float *__restrict__ logprob, float *__restrict__ entropy,
+                    float *__restrict__ ref_logprob, int *status, int *flags2)
 {
     __shared__ float red[96];
     // ppo_step: the hand-over flags between the two kernels that follow start at 0 (nothing runs beside this
     // kernel on the stream, and the next kernel starts after it has ended)
     if (flags2 && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) { flags2[0] = 0; flags2[1] = 0; }
     grid_dependents_may_launch();   // the token-level kernel may be scheduled as this grid drains; it waits for its end
+    if (seq_T > 0) {
+        const int64_t row = blockIdx.x;
+        const int t = (int)(row % seq_T);
+        const int32_t *r = tokens + (row - t);
+        int hit = 0;
+        for (int i = threadIdx.x; i < t; i += THREADS) hit |= r[i] == eos_id;
+        if (__syncthreads_or(hit)) {
+            if (threadIdx.x == 0) {
+                if (blockIdx.y == 0) {
+                    logprob[row] = 0.f;
+                    entropy[row] = 0.f;
+                } else {
+                    ref_logprob[row] = 0.f;
+                }
+            }
+            return;
+        }
+    }
     if (blockIdx.y == 0)
         logprob_entropy_row<T, true, true, THREADS>(policy_logits, V, V, tokens, mask, c, logprob, entropy, nullptr,
                                                     status, red);
@@ -267,8 +288,8 @@ static int launch_logprob(const void *logits, int64_t rows, int V, int64_t row_s
 
 // PPO_ERR_UNSUPPORTED when the pointers or the shape do not allow 16-byte packs (the caller then makes two calls)
 int launch_logprob_pair(const void *policy_logits, const void *ref_logits, int dtype, int64_t rows, int V,
-                        const int32_t *tokens, const uint8_t *mask, float c, float *logprob, float *entropy,
-                        float *ref_logprob, WorkspaceHeader *hdr, bool clear_flags, cudaStream_t s)
+                        const int32_t *tokens, const uint8_t *mask, int seq_T, int eos_id, float c, float *logprob,
+                        float *entropy, float *ref_logprob, WorkspaceHeader *hdr, bool clear_flags, cudaStream_t s)
 {
     int *status = hdr ? &hdr->status : nullptr, *flags2 = (hdr && clear_flags) ? &hdr->order_ready : nullptr;
     static_assert(offsetof(WorkspaceHeader, adv_ready) == offsetof(WorkspaceHeader, order_ready) + sizeof(int),
@@ -282,11 +303,11 @@ int launch_logprob_pair(const void *policy_logits, const void *ref_logits, int d
     if (dtype == PPO_F32)
         logprob_pair_kernel<float, THREADS><<<grid, THREADS, 0, s>>>(
             reinterpret_cast<const float *>(policy_logits), reinterpret_cast<const float *>(ref_logits), V, tokens, mask,
-            c, logprob, entropy, ref_logprob, status, flags2);
+            seq_T, eos_id, c, logprob, entropy, ref_logprob, status, flags2);
     else
         logprob_pair_kernel<__nv_bfloat16, THREADS><<<grid, THREADS, 0, s>>>(
             reinterpret_cast<const __nv_bfloat16 *>(policy_logits), reinterpret_cast<const __nv_bfloat16 *>(ref_logits),
-            V, tokens, mask, c, logprob, entropy, ref_logprob, status, flags2);
+            V, tokens, mask, seq_T, eos_id, c, logprob, entropy, ref_logprob, status, flags2);
     return launch_status();
 }
 
@@ -486,7 +507,7 @@ extern "C" int ppo_logprob_entropy_pair(const void *policy_logits, const void *r
     const size_t es = dtype == PPO_F32 ? 4 : 2;
     if (reinterpret_cast<uintptr_t>(policy_logits) % es || reinterpret_cast<uintptr_t>(ref_logits) % es)
         return PPO_ERR_ALIGN;
-    int rc = launch_logprob_pair(policy_logits, ref_logits, dtype, rows, (int)V, tokens, mask, kLog2e / temperature,
+    int rc = launch_logprob_pair(policy_logits, ref_logits, dtype, rows, (int)V, tokens, mask, 0, 0, kLog2e / temperature,
                                  logprob, entropy, ref_logprob, workspace ? ws_header(workspace) : nullptr, false,
                                  reinterpret_cast<cudaStream_t>(stream));
     if (rc != PPO_ERR_UNSUPPORTED) return rc;

@@ -24,19 +24,25 @@ extern "C" int ppo_step(const ppo_step_io *io, int dtype, int32_t B, int32_t T, 
     if (rows >= ((int64_t)1 << 31)) return PPO_ERR_SHAPE;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     // three launches: log-probs (policy and reference) -> [EOS trick + KL rewards + GAE, then loss
-    // prologue + whitening in the last block] -> loss forward/backward
+    // prologue + whitening in the last block] -> loss forward/backward.
+    // Padding rows (after a sequence's first EOS) are masked out of every later step, so step 1 does not read
+    // their logits: the log-prob kernel finds them from the sampled tokens alone and writes 0 there.
     int rc = PPO_ERR_UNSUPPORTED;
     if ((dtype == PPO_F32 || dtype == PPO_BF16) && V < ((int64_t)1 << 31) && p->temperature > 0.f &&
         finite_f(p->temperature) && option_value(PPO_OPT_ROW_ENGINE) != 2)
-        rc = launch_logprob_pair(io->policy_logits, io->ref_logits, dtype, rows, (int)V, io->responses, nullptr,
-                                 kLog2e / p->temperature, io->logprob, io->entropy, io->ref_logprob,
+        rc = launch_logprob_pair(io->policy_logits, io->ref_logits, dtype, rows, (int)V, io->responses, nullptr, T,
+                                 p->eos_id, kLog2e / p->temperature, io->logprob, io->entropy, io->ref_logprob,
                                  ws_header(io->workspace), true, s);
     const bool flags_cleared = rc == PPO_OK;
-    if (rc == PPO_ERR_UNSUPPORTED) {   // layout without 16-byte packs (or the row engine was asked for): two calls
-        rc = ppo_logprob_entropy(io->policy_logits, dtype, rows, V, V, io->responses, nullptr, p->temperature,
+    if (rc == PPO_ERR_UNSUPPORTED) {   // layout without 16-byte packs (or the row engine was asked for): the EOS
+                                       // trick first (for the mask), then one call per tensor
+        rc = ppo_truncate_and_score(io->responses, B, T, p->eos_id, p->pad_id, io->scores, p->no_eos_score,
+                                    io->responses_out, io->eos_index, io->seq_len, io->mask, io->scores_out, stream);
+        if (rc) return rc;
+        rc = ppo_logprob_entropy(io->policy_logits, dtype, rows, V, V, io->responses, io->mask, p->temperature,
                                  io->logprob, io->entropy, nullptr, io->workspace, stream);
         if (rc) return rc;
-        rc = ppo_logprob_entropy(io->ref_logits, dtype, rows, V, V, io->responses, nullptr, p->temperature,
+        rc = ppo_logprob_entropy(io->ref_logits, dtype, rows, V, V, io->responses, io->mask, p->temperature,
                                  io->ref_logprob, nullptr, nullptr, io->workspace, stream);
     }
     if (rc) return rc;

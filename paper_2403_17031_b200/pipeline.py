@@ -15,6 +15,8 @@ class PPOHotPath:
     step(...) runs: EOS trick -> log-prob/entropy of policy and reference -> KL rewards -> GAE ->
     advantage whitening -> clipped losses + gradients, all on the current CUDA stream, and
     returns the dict of output tensors (owned by this object, overwritten by the next step).
+    Padding rows (after a response's first EOS) are masked out of every later step, so their logits
+    are not read: log-prob and entropy are 0 there.
     """
 
     def __init__(self, B: int, T: int, V: int, logits_dtype: torch.dtype, params: _b.PPOParams,
@@ -41,12 +43,12 @@ class PPOHotPath:
                           "dvalues": self.out["dvalues"], "new_logprob": self.out["new_logprob"],
                           "entropy": self.out["new_entropy"], "dlogprob": self.out["dlogprob"]}
 
-    def rollout_stats(self, policy_logits, ref_logits, responses, scores, values, skip_masked_rows=False):
-        """Steps 1-5: everything between sampling and the first PPO epoch."""
+    def rollout_stats(self, policy_logits, ref_logits, responses, scores, values):
+        """Steps 1-5, one C call per step: everything between sampling and the first PPO epoch."""
         o, p = self.out, self.params
         _b.truncate_and_score(responses, scores, p.eos_id, p.pad_id, p.no_eos_score,
                               out=(o["responses_out"], o["eos_index"], o["seq_len"], o["mask"], o["scores_out"]))
-        m = o["mask"] if skip_masked_rows else None
+        m = o["mask"]
         _b.logprob_entropy(policy_logits, responses, p.temperature, mask=m, workspace=self.workspace,
                            out=(o["logprob"], o["entropy"], None))
         _b.logprob_entropy(ref_logits, responses, p.temperature, mask=m, workspace=self.workspace,
@@ -68,14 +70,9 @@ class PPOHotPath:
         return o
 
     def step(self, policy_logits, ref_logits, responses, scores, values, values_new, old_logprob=None,
-             loss_logits=None, skip_masked_rows=False):
-        """One pass of the whole path. old_logprob defaults to the rollout log-probs just computed
-        (first PPO epoch: ratio = 1); loss_logits defaults to policy_logits. One C call (ppo_step)
-        unless masked rows are to be skipped in step 1."""
-        if skip_masked_rows:
-            o = self.rollout_stats(policy_logits, ref_logits, responses, scores, values, True)
-            return self.loss(policy_logits if loss_logits is None else loss_logits, responses,
-                             o["logprob"] if old_logprob is None else old_logprob, values_new, values)
+             loss_logits=None):
+        """One pass of the whole path in one C call (ppo_step). old_logprob defaults to the rollout
+        log-probs just computed (first PPO epoch: ratio = 1); loss_logits defaults to policy_logits."""
         io = self.step_io({"policy_logits": policy_logits, "ref_logits": ref_logits, "loss_logits": loss_logits,
                            "responses": responses, "scores": scores, "values": values, "values_new": values_new,
                            "old_logprob": old_logprob})

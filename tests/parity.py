@@ -64,9 +64,12 @@ def assert_grad(got_scaled, want_scaled, bf16: bool, what):
                                                                    np.abs(got - want)[bad].max())
 
 
-def oracle_chain(O, batch, h, old_logprob=None, loss_logits=None, sel_rows=None, want_dlogits=True):
+def oracle_chain(O, batch, h, old_logprob=None, loss_logits=None, sel_rows=None, want_dlogits=True,
+                 step1_mask=True):
     """The whole path on the oracle, each stage fed the previous stage's float64 results rounded
-    to fp32 (the precision in which the GPU stages exchange data)."""
+    to fp32 (the precision in which the GPU stages exchange data). step1_mask: step 1 is given the
+    mask of the EOS trick (padding rows output 0, as in the chained GPU path); False computes every row
+    (what the stand-alone log-prob call without a mask returns)."""
     pl = host_logits(batch["policy_logits"])
     rl = host_logits(batch["ref_logits"])
     B, T, V = pl.shape
@@ -75,8 +78,9 @@ def oracle_chain(O, batch, h, old_logprob=None, loss_logits=None, sel_rows=None,
     r = {}
     r["responses_out"], r["eos_index"], r["seq_len"], r["mask"], r["scores_out"] = O.truncate_and_score(
         resp, h.eos_id, h.pad_id, npy(batch["scores"]), np.float32(h.no_eos_score))
-    lp, ent, _ = O.logprob_entropy(pl.reshape(-1, V), resp, tau)
-    rlp, _, _ = O.logprob_entropy(rl.reshape(-1, V), resp, tau)
+    m1 = r["mask"].reshape(-1) if step1_mask else None
+    lp, ent, _ = O.logprob_entropy(pl.reshape(-1, V), resp, tau, mask=m1)
+    rlp, _, _ = O.logprob_entropy(rl.reshape(-1, V), resp, tau, mask=m1)
     r["logprob"], r["entropy"], r["ref_logprob"] = lp.reshape(B, T), ent.reshape(B, T), rlp.reshape(B, T)
     r["kl"], r["rewards"] = O.kl_rewards(f32(r["logprob"]), f32(r["ref_logprob"]), r["mask"], r["seq_len"],
                                          f32(r["scores_out"]), np.float32(h.kl_coef))

@@ -31,7 +31,7 @@ def _check_stagewise(P, O, cfg, batch, n_grad_rows=None, seed=0):
     B, T, V = batch["policy_logits"].shape
     bf16 = batch["policy_logits"].dtype == torch.bfloat16
     rng = np.random.default_rng(seed)
-    ref = oracle_chain(O, batch, h, want_dlogits=False)
+    ref = oracle_chain(O, batch, h, want_dlogits=False, step1_mask=False)
     mask_np = ref["mask"].astype(bool)
     real_rows = np.flatnonzero(mask_np.reshape(-1))
     masked_rows = np.flatnonzero(~mask_np.reshape(-1))
