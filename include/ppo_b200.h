@@ -377,7 +377,8 @@ int ppo_lmhead_bwd(const void *H, const void *W, int64_t M, int64_t K, int64_t V
  *            responses [B,T] i32; scores [B]; values, values_new [B,T];
  *            old_logprob [B,T] or NULL (= the log-probs this call computes: first PPO epoch, ratio 1)
  *   outputs  responses_out, eos_index, seq_len, mask, scores_out (step 2); logprob, entropy,
- *            ref_logprob (step 1); kl, rewards (step 3; with params.whiten_rewards the rewards
+ *            ref_logprob (step 1, as with the mask of step 2: 0 at the padding positions after a
+ *            response's first EOS, whose logits are not read); kl, rewards (step 3; with params.whiten_rewards the rewards
  *            array holds the whitened rewards that GAE consumed); advantages, returns (step 4);
  *            advantages_whitened, whiten_stats[3] (step 5); losses[8], dlogits, dvalues and the
  *            nullable new_logprob, new_entropy, dlogprob (step 6); workspace (device only)
