@@ -385,3 +385,38 @@ def test_step_overlapped_launches_repeatable(P, B, T, V, dtype):
         for k in names:
             assert torch.equal(b.out[k], want[k]), (k, "graph", it)
     assert b.device_status() == 0
+
+
+@pytest.mark.parametrize("B,T,V,dtype", [(70, 53, 2048, "bf16"), (6, 16, 1001, "f32")])
+def test_step_never_reads_padding_rows(P, B, T, V, dtype):
+    """Everything after a response's first EOS is padding (EOS trick): the whole-path call must not read those rows
+    of any logits tensor. NaN planted there changes no output bit and raises no status; V = 1001 takes the path
+    without 16-byte packs."""
+    import dataclasses
+    from paper_2403_17031_b200.pipeline import PPOHotPath
+    from paper_2403_17031_b200.synthetic import CONFIGS, make_batch
+    cfg = dataclasses.replace(CONFIGS[0], B=B, T=T, V=V, dtype=dtype, n_no_eos_exact=None)
+    batch = make_batch(cfg, "cuda")
+    pp = _params(P, cfg.hyper)
+    names = ("mask", "seq_len", "logprob", "entropy", "ref_logprob", "kl", "rewards", "advantages", "returns",
+             "advantages_whitened", "losses", "dlogits", "dvalues", "new_logprob", "dlogprob")
+    args = lambda pl, rl: (pl, rl, batch["responses"], batch["scores"], batch["values"], batch["values_new"])
+    a = PPOHotPath(B, T, V, cfg.torch_dtype, pp)
+    a.step(*args(batch["policy_logits"], batch["ref_logits"]))
+    torch.cuda.synchronize()
+    pad = a.out["mask"] == 0
+    assert pad.any() and not pad.all()
+    for k in ("logprob", "entropy", "ref_logprob", "kl", "rewards", "advantages", "advantages_whitened"):
+        assert not a.out[k][pad].any(), k
+    assert not a.out["dlogits"][pad].any()
+    poisoned = []
+    for k in ("policy_logits", "ref_logits"):
+        t = batch[k].clone()
+        t[pad] = float("nan")
+        poisoned.append(t)
+    b = PPOHotPath(B, T, V, cfg.torch_dtype, pp)
+    b.step(*args(*poisoned))
+    torch.cuda.synchronize()
+    for k in names:
+        assert torch.equal(a.out[k], b.out[k]), k
+    assert b.device_status() == 0
