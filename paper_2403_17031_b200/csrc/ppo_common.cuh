@@ -399,6 +399,9 @@ int loss_fwd_bwd_prepared(const void *logits, int dtype, int32_t B, int32_t T, i
                           float *losses, void *dlogits, float *dvalues, float *new_logprob, float *entropy,
                           float *dlogprob, void *workspace, void *stream, bool prepared);
 int launch_loss_prepare(const uint8_t *mask, int64_t rows, void *workspace, cudaStream_t s);
+// the same prologue with the order array at a place of the caller's choice: hdr->n_tokens = number of rows with
+// mask 1, order[0 .. n_tokens) = those rows (ascending), order[n_tokens .. rows) = the other rows
+int launch_row_order(const uint8_t *mask, int64_t rows, WorkspaceHeader *hdr, int32_t *order, cudaStream_t s);
 // step 1 for policy and reference logits in one launch; PPO_ERR_UNSUPPORTED if the layout rules it out
 // (also clears the two hand-over flags of the header for the kernels that follow in ppo_step).
 // seq_T > 0: rows = B * seq_T responses, and rows after a sequence's first eos_id are padding (skipped, outputs 0)

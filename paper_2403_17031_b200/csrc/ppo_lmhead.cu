@@ -154,6 +154,11 @@ __device__ __forceinline__ LmUnit lm_unit(int u, int m_tiles, int n_chunks)
 struct LmArgs {
     int M, K, V;
     int m_tiles, n_tiles, n_chunks, n_units;
+    // Row compaction (the call was given a mask): H holds the rows with mask 1 only, packed by an earlier kernel of
+    // the stream; *m_eff = how many (known on the device only: M, m_tiles and n_units above are upper bounds),
+    // order[j] = the original index of packed row j (tokens is indexed by the original row)
+    const int *m_eff;
+    const int32_t *order;
     const int32_t *tokens;
     float c;
     float4 *partials;     // [m_tiles*128][n_chunks]
@@ -171,6 +176,13 @@ lmhead_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__
     unsigned char *ring = lm_smem_raw + ((1024u - (lm_smem_addr(lm_smem_raw) & 1023u)) & 1023u);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int k_blocks = a.K / kBlockK;
+    // every role walks the same unit list, derived from the same row count
+    int n_rows = a.M, m_tiles = a.m_tiles, n_units = a.n_units;
+    if (a.m_eff) {
+        n_rows = max(0, min(*a.m_eff, a.M));
+        m_tiles = ((n_rows + kBlockM - 1) / kBlockM + MT - 1) / MT;
+        n_units = m_tiles * a.n_chunks;
+    }
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -199,8 +211,8 @@ lmhead_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t it = 0;
-            for (int u = blockIdx.x; u < a.n_units; u += gridDim.x) {
-                const LmUnit un = lm_unit(u, a.m_tiles, a.n_chunks);
+            for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+                const LmUnit un = lm_unit(u, m_tiles, a.n_chunks);
                 const int t0 = un.chunk * kTilesPerChunk, t1 = min(t0 + kTilesPerChunk, a.n_tiles);
                 for (int t = t0; t < t1; ++t) {
                     for (int kb = 0; kb < k_blocks; ++kb, ++it) {
@@ -227,8 +239,8 @@ lmhead_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             uint32_t it = 0, tc = 0;
-            for (int u = blockIdx.x; u < a.n_units; u += gridDim.x) {
-                const LmUnit un = lm_unit(u, a.m_tiles, a.n_chunks);
+            for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+                const LmUnit un = lm_unit(u, m_tiles, a.n_chunks);
                 const int t0 = un.chunk * kTilesPerChunk, t1 = min(t0 + kTilesPerChunk, a.n_tiles);
                 for (int t = t0; t < t1; ++t, ++tc) {
                     const uint32_t buf = tc % kSets;
@@ -266,12 +278,12 @@ lmhead_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__
         const int acc = (warp - 2) >> 2;             // which of the unit's MT accumulators / row tiles
         const int row_in_tile = q * 32 + lane;
         uint32_t tc = 0;
-        for (int u = blockIdx.x; u < a.n_units; u += gridDim.x) {
-            const LmUnit un = lm_unit(u, a.m_tiles, a.n_chunks);
+        for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+            const LmUnit un = lm_unit(u, m_tiles, a.n_chunks);
             const int t0 = un.chunk * kTilesPerChunk, t1 = min(t0 + kTilesPerChunk, a.n_tiles);
             const int row = (un.m_tile * MT + acc) * kBlockM + row_in_tile;
-            const bool row_ok = row < a.M;
-            const int tok = row_ok ? a.tokens[row] : -1;
+            const bool row_ok = row < n_rows;
+            const int tok = row_ok ? a.tokens[a.order ? a.order[row] : row] : -1;
             float m = 0.f, s0 = 0.f, s1 = 0.f, u0 = 0.f, u1 = 0.f;
             bool have_ref = false;
             uint32_t xtok_bits = kAbsentBits;
@@ -358,21 +370,37 @@ lmhead_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__
     }
 }
 
-// merge the chunk partials of each row in chunk order; one thread per row
+// pack the rows with mask 1 (order[0 .. *n)) of H [M, K] into Hc; k16 = 16-byte pieces per row
+__global__ void __launch_bounds__(256)
+lmhead_pack_rows_kernel(const uint4 *__restrict__ H, int k16, const int32_t *__restrict__ order, const int *__restrict__ n,
+                        uint4 *__restrict__ Hc)
+{
+    const int j = blockIdx.x;
+    if (j >= *n) return;
+    const uint4 *src = H + (size_t)order[j] * k16;
+    uint4 *dst = Hc + (size_t)j * k16;
+    for (int i = threadIdx.x; i < k16; i += blockDim.x) dst[i] = src[i];
+}
+
+// merge the chunk partials of each row in chunk order; one thread per row. With row compaction thread i holds
+// packed row i < *m_eff (original row order[i]); the threads beyond write the zeros of the rows with mask 0.
 __global__ void __launch_bounds__(256)
 lmhead_finalize_kernel(const float4 *__restrict__ partials, int M, int V, int n_chunks, const int32_t *__restrict__ tokens,
-                       const uint8_t *__restrict__ mask, float c, float *__restrict__ logprob,
+                       const uint8_t *__restrict__ mask, const int32_t *__restrict__ order,
+                       const int *__restrict__ m_eff, float c, float *__restrict__ logprob,
                        float *__restrict__ entropy, float *__restrict__ lse, int *status)
 {
-    const int row = blockIdx.x * blockDim.x + threadIdx.x;
-    if (row >= M) return;
+    const int packed = blockIdx.x * blockDim.x + threadIdx.x;
+    if (packed >= M) return;
+    const int row = order ? order[packed] : packed;
+    const bool real = order ? packed < *m_eff : (!mask || mask[row]);
     float lp = 0.f, H = 0.f, L = 0.f;
-    if (!mask || mask[row]) {
+    if (real) {
         SoftmaxState st;
         st.init();
         uint32_t xbits = kAbsentBits;
         for (int k = 0; k < n_chunks; ++k) {
-            const float4 p = partials[(size_t)row * n_chunks + k];
+            const float4 p = partials[(size_t)packed * n_chunks + k];
             SoftmaxState o;
             o.m = p.x;
             o.s = p.y;
@@ -429,6 +457,11 @@ static int make_map(CUtensorMap *map, const void *base, uint64_t inner, uint64_t
     return r == CUDA_SUCCESS ? PPO_OK : (int)cudaErrorInvalidValue;
 }
 
+static size_t lm_partials_bytes(int m_tiles, int n_chunks)
+{
+    return align256((size_t)m_tiles * kBlockM * (size_t)n_chunks * sizeof(float4));
+}
+
 static void lm_shape(int64_t M, int64_t V, int *m_tiles, int *n_tiles, int *n_chunks)
 {
     *m_tiles = (int)((M + kBlockM - 1) / kBlockM);
@@ -442,11 +475,12 @@ using namespace ppo;
 
 extern "C" size_t ppo_lmhead_workspace_bytes(int64_t M, int64_t K, int64_t V)
 {
-    (void)K;
     if (M <= 0 || V <= 0) return kHeaderBytes;
     int m_tiles, n_tiles, n_chunks;
     lm_shape(M, V, &m_tiles, &n_tiles, &n_chunks);
-    return kHeaderBytes + align256((size_t)m_tiles * kBlockM * (size_t)n_chunks * sizeof(float4));
+    // header | per-row chunk partials | row order | packed copy of H (calls with a mask)
+    return kHeaderBytes + lm_partials_bytes(m_tiles, n_chunks) + align256((size_t)M * sizeof(int32_t)) +
+           align256((size_t)M * (size_t)(K > 0 ? K : 0) * 2);
 }
 
 extern "C" int ppo_lmhead_logprob_entropy(const void *H, const void *W, int64_t M, int64_t K, int64_t V,
@@ -476,11 +510,32 @@ extern "C" int ppo_lmhead_logprob_entropy(const void *H, const void *W, int64_t 
     a.n_units = (int)units;
     a.tokens = tokens;
     a.c = kLog2e / temperature;
-    a.partials = reinterpret_cast<float4 *>(reinterpret_cast<unsigned char *>(workspace) + kHeaderBytes);
+    unsigned char *ws = reinterpret_cast<unsigned char *>(workspace);
+    a.partials = reinterpret_cast<float4 *>(ws + kHeaderBytes);
     a.status = &ws_header(workspace)->status;
+    a.m_eff = nullptr;
+    a.order = nullptr;
+    int rc;
+    // With a mask, and more than one row tile, the rows with mask 0 are taken out of the GEMM: their order is
+    // found on the device, the other rows of H are packed into the workspace (M*K*2 bytes moved against
+    // 2*K*V flops saved per row with mask 0) and the kernels below work on the packed rows; the finalize kernel
+    // writes every result at its original row.
+    if (mask && a.m_tiles >= 2) {
+        int32_t *order = reinterpret_cast<int32_t *>(ws + kHeaderBytes + lm_partials_bytes(a.m_tiles, a.n_chunks));
+        uint4 *Hc = reinterpret_cast<uint4 *>(reinterpret_cast<unsigned char *>(order) + align256((size_t)M * sizeof(int32_t)));
+        rc = launch_row_order(mask, M, ws_header(workspace), order, s);
+        if (rc) return rc;
+        a.m_eff = &ws_header(workspace)->n_tokens;
+        a.order = order;
+        lmhead_pack_rows_kernel<<<(unsigned)M, 256, 0, s>>>(reinterpret_cast<const uint4 *>(H), (int)(K / 8), order, a.m_eff,
+                                                          Hc);
+        rc = launch_status();
+        if (rc) return rc;
+        H = Hc;
+    }
 
     CUtensorMap map_h, map_w;
-    int rc = make_map(&map_h, H, (uint64_t)K, (uint64_t)M, kBlockM);
+    rc = make_map(&map_h, H, (uint64_t)K, (uint64_t)M, kBlockM);
     if (rc) return rc;
     rc = make_map(&map_w, W, (uint64_t)V, (uint64_t)K, kBlockK);
     if (rc) return rc;
@@ -505,7 +560,7 @@ extern "C" int ppo_lmhead_logprob_entropy(const void *H, const void *W, int64_t 
     }
     rc = launch_status();
     if (rc) return rc;
-    lmhead_finalize_kernel<<<(unsigned)((M + 255) / 256), 256, 0, s>>>(a.partials, a.M, a.V, a.n_chunks, tokens, mask, a.c,
-                                                                       logprob, entropy, lse, a.status);
+    lmhead_finalize_kernel<<<(unsigned)((M + 255) / 256), 256, 0, s>>>(a.partials, a.M, a.V, a.n_chunks, tokens, mask, a.order,
+                                                                       a.m_eff, a.c, logprob, entropy, lse, a.status);
     return launch_status();
 }

@@ -183,7 +183,8 @@ constexpr int kReduceThreads = 1024;
 // thread owns one contiguous segment of rows, so the order is deterministic.
 __device__ __forceinline__ void loss_prepare_block(const uint8_t *mask, int64_t rows, WorkspaceHeader *hdr,
                                                    int32_t *__restrict__ order, int *warp_tot /* 32 ints */,
-                                                   bool publish /* a loss kernel may be waiting for the result */)
+                                                   bool publish /* a loss kernel may be waiting for the result */,
+                                                   bool flag_empty = true /* no row with mask 1: status bit */)
 {
     // segments are multiples of 16 rows so that a 16-byte aligned mask is read 16 rows per load (the result does
     // not depend on the segment length: segments are contiguous and ascending)
@@ -223,7 +224,7 @@ __device__ __forceinline__ void loss_prepare_block(const uint8_t *mask, int64_t 
             hdr->masked_next = 0;
             hdr->real_next = 0;
             hdr->done_blocks = 0;
-            if (wi == 0) atomicOr(&hdr->status, PPO_DEV_EMPTY_MASK);
+            if (wi == 0 && flag_empty) atomicOr(&hdr->status, PPO_DEV_EMPTY_MASK);
         }
     }
     __syncthreads();
@@ -249,7 +250,8 @@ __device__ __forceinline__ void loss_prepare_block(const uint8_t *mask, int64_t 
 }
 
 __global__ void __launch_bounds__(kReduceThreads)
-loss_prepare_kernel(const uint8_t *__restrict__ mask, int64_t rows, WorkspaceHeader *hdr, int32_t *__restrict__ order)
+loss_prepare_kernel(const uint8_t *__restrict__ mask, int64_t rows, WorkspaceHeader *hdr, int32_t *__restrict__ order,
+                    int flag_empty)
 {
     __shared__ int warp_tot[32];
     // the loss kernel that follows is launched as a programmatic dependent: it may start now and waits on the
@@ -261,7 +263,7 @@ loss_prepare_kernel(const uint8_t *__restrict__ mask, int64_t rows, WorkspaceHea
     }
     __syncthreads();
     grid_dependents_may_launch();
-    loss_prepare_block(mask, rows, hdr, order, warp_tot, true);
+    loss_prepare_block(mask, rows, hdr, order, warp_tot, true, flag_empty != 0);
     if (threadIdx.x == 0) flag_set(&hdr->adv_ready);   // stand-alone loss call: its other inputs exist already
 }
 
@@ -442,7 +444,14 @@ loss_from_logprob_kernel(const float *__restrict__ new_logprob, const float *__r
 
 int launch_loss_prepare(const uint8_t *mask, int64_t rows, void *workspace, cudaStream_t s)
 {
-    loss_prepare_kernel<<<1, kReduceThreads, 0, s>>>(mask, rows, ws_header(workspace), ws_order(workspace, rows));
+    loss_prepare_kernel<<<1, kReduceThreads, 0, s>>>(mask, rows, ws_header(workspace), ws_order(workspace, rows), 1);
+    return launch_status();
+}
+
+int launch_row_order(const uint8_t *mask, int64_t rows, WorkspaceHeader *hdr, int32_t *order, cudaStream_t s)
+{
+    // (an empty selection is not an error for the caller of this one: no status bit)
+    loss_prepare_kernel<<<1, kReduceThreads, 0, s>>>(mask, rows, hdr, order, 0);
     return launch_status();
 }
 

@@ -92,3 +92,45 @@ def test_lmhead_config4_full_size_sampled_rows(P, oracle):
     assert torch.isfinite(lp).all() and torch.isfinite(ent).all()
     # properties that hold for every row: entropy within [0, ln V], log-prob <= 0
     assert float(ent.min()) >= 0.0 and float(ent.max()) <= np.log(V) + 1e-4 and float(lp.max()) <= 1e-5
+
+
+@pytest.mark.parametrize("M,K,V,pattern", [(700, 128, 1000, "tails"), (700, 128, 1000, "random"), (300, 64, 520, "none"),
+                                           (300, 64, 520, "all"), (5000, 64, 264, "one")])
+def test_lmhead_mask_takes_rows_out_of_the_gemm(P, oracle, M, K, V, pattern):
+    """With a mask (and more than one row tile) the call packs the rows with mask 1 and multiplies only those. Rows with
+    mask 1 must carry the bits of the call without a mask (each logits row depends on its own row of H only), the
+    others 0; repeated on one workspace, with a stale packed copy from a call with another mask in it."""
+    H, W, tok = _inputs(M, K, V, seed=M + V)
+    g = torch.Generator(device="cuda").manual_seed(7)
+    if pattern == "tails":      # responses of 53 tokens, each real up to its own length: the shape of the PPO batch
+        t = torch.arange(M, device="cuda") % 53
+        L = torch.randint(1, 54, ((M + 52) // 53,), generator=g, device="cuda").repeat_interleave(53)[:M]
+        mask = (t < L).to(torch.uint8)
+    elif pattern == "random":
+        mask = (torch.rand(M, generator=g, device="cuda") < 0.5).to(torch.uint8)
+    elif pattern == "none":
+        mask = torch.zeros(M, dtype=torch.uint8, device="cuda")
+    elif pattern == "all":
+        mask = torch.ones(M, dtype=torch.uint8, device="cuda")
+    else:
+        mask = torch.zeros(M, dtype=torch.uint8, device="cuda")
+        mask[M - 3] = 1
+    ws = P.new_workspace(P.lmhead_workspace_bytes(M, K, V))
+    dense = [t.clone() for t in P.lmhead_logprob_entropy(H, W, tok, 0.7, ws)]
+    other = (torch.rand(M, generator=g, device="cuda") < 0.8).to(torch.uint8)
+    P.lmhead_logprob_entropy(H, W, tok, 0.7, ws, mask=other)      # leaves its packed rows behind
+    m = mask.bool()
+    for _ in range(2):
+        got = P.lmhead_logprob_entropy(H, W, tok, 0.7, ws, mask=mask)
+        torch.cuda.synchronize()
+        for a, b, name in zip(got, dense, ("logprob", "entropy", "lse")):
+            assert torch.equal(a[m], b[m]), name
+            assert not a[~m].any(), name
+    assert P.last_device_status(ws) == 0
+    if m.any():
+        sel = np.flatnonzero(npy(mask))[:64].astype(np.int64)
+        rlp, rent, rlse = oracle.lmhead_logprob_entropy(host_logits(H), host_logits(W), npy(tok), np.float32(0.7),
+                                                        sel_rows=sel)
+        assert_abs(npy(got[0])[sel], rlp, TOL_LOGPROB, "logprob")
+        assert_abs(npy(got[1])[sel], rent, TOL_LOGPROB, "entropy")
+        assert_abs(npy(got[2])[sel], rlse, TOL_LOGPROB, "lse")
