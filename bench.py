@@ -446,9 +446,10 @@ def run_lmhead(args, cfg):
     def step(old):
         binding.truncate_and_score(b["responses"], b["scores"], p.eos_id, p.pad_id, p.no_eos_score,
                                    out=(o["ro"], o["ei"], o["sl"], o["mask"], o["so"]))
-        binding.lmhead_logprob_entropy(b["H"], b["W"], tok, p.temperature, ws,
+        # (with the mask of the EOS trick: padding rows are taken out of the GEMM and get 0)
+        binding.lmhead_logprob_entropy(b["H"], b["W"], tok, p.temperature, ws, mask=o["mask"].view(-1),
                                        out=(o["lp"].view(-1), o["ent"].view(-1), o["lse"].view(-1)))
-        binding.lmhead_logprob_entropy(b["H"], b["W_ref"], tok, p.temperature, ws,
+        binding.lmhead_logprob_entropy(b["H"], b["W_ref"], tok, p.temperature, ws, mask=o["mask"].view(-1),
                                        out=(o["rlp"].view(-1), o["rent"].view(-1), None))
         binding.kl_rewards(o["lp"], o["rlp"], o["mask"], o["sl"], o["so"], p.kl_coef, out=(o["kl"], o["rew"]))
         binding.gae(o["rew"], b["values"], o["sl"], p.gamma, p.lam, out=(o["adv"], o["ret"]))
@@ -475,10 +476,10 @@ def run_lmhead(args, cfg):
             binding.truncate_and_score(b["responses"], b["scores"], p.eos_id, p.pad_id, p.no_eos_score,
                                        out=(o["ro"], o["ei"], o["sl"], o["mask"], o["so"]))
             lm_ev[i][0].record()
-            binding.lmhead_logprob_entropy(b["H"], b["W"], tok, p.temperature, ws,
+            binding.lmhead_logprob_entropy(b["H"], b["W"], tok, p.temperature, ws, mask=o["mask"].view(-1),
                                            out=(o["lp"].view(-1), o["ent"].view(-1), o["lse"].view(-1)))
             lm_ev[i][1].record()
-            binding.lmhead_logprob_entropy(b["H"], b["W_ref"], tok, p.temperature, ws,
+            binding.lmhead_logprob_entropy(b["H"], b["W_ref"], tok, p.temperature, ws, mask=o["mask"].view(-1),
                                            out=(o["rlp"].view(-1), o["rent"].view(-1), None))
             binding.kl_rewards(o["lp"], o["rlp"], o["mask"], o["sl"], o["so"], p.kl_coef, out=(o["kl"], o["rew"]))
             binding.gae(o["rew"], b["values"], o["sl"], p.gamma, p.lam, out=(o["adv"], o["ret"]))
@@ -500,7 +501,8 @@ def run_lmhead(args, cfg):
     lm_ms = statistics.mean(a.elapsed_time(c) for a, c in lm_ev)
     status = binding.last_device_status(ws)
     bwd_ms = statistics.mean(a.elapsed_time(c) for a, c in bw_ev) if bwd_out is not None else None
-    flops = 2.0 * M * K * V
+    n_real = int(o["mask"].sum().item())
+    flops = 2.0 * n_real * K * V      # the forward call multiplies the real rows only
     tf = flops / (lm_ms * 1e-3) / 1e12
     # the kernel runs back to back for the whole timed region: compare with the sustained figure
     peak, kind = _peaks("bf16_tflops_sustained", 1400.0)
@@ -514,14 +516,16 @@ def run_lmhead(args, cfg):
                        "l2": "inputs larger than L2 (H %.0f MB + 2 x W %.0f MB per step)" %
                              (M * K * 2 / 1e6, K * V * 2 / 1e6),
                        "lmhead_ms": lm_ms, "lmhead_bwd_ms": bwd_ms,
-                       "lmhead_bwd_tflops": None if bwd_ms is None else 3.0 * flops / (bwd_ms * 1e-3) / 1e12,
+                       "real_tokens": n_real,
+                       "lmhead_bwd_tflops": None if bwd_ms is None else 3.0 * 2.0 * M * K * V / (bwd_ms * 1e-3) / 1e12,
                        "device_status": status},
             "roofline": {"bound": "tensor", "kernel": "lmhead_kernel (ppo_lmhead_logprob_entropy)", "achieved": tf,
                          "peak": peak, "peak_kind": kind + " (sustained)", "unit": "TFLOP/s", "frac": tf / peak,
                          "frac_of_burst": tf / burst, "traffic": None,
-                         "timing": "CUDA events around the C-ABI call (GEMM kernel + finalize kernel)"},
+                         "timing": "CUDA events around the C-ABI call (row order, packing of the real rows, GEMM kernel, "
+                                   "finalize kernel); flops = 2 x real rows x K x V"},
             "clocks": clk.summary(), "e2e": None, "cpu_baseline": None,
-            "gpu_launches": (9 + (3 if bwd_out is not None else 0)) * K_steps,
+            "gpu_launches": (13 + (3 if bwd_out is not None else 0)) * K_steps,
         }
         print(json.dumps(line), flush=True)
     if distributed:

@@ -342,8 +342,12 @@ int ppo_loss_from_logprob_static(const float *new_logprob, const float *entropy,
  * in the epilogue; they are never written to memory.
  *   H [M,K] bf16 row-major;  W [K,V] bf16 row-major;  tokens [M];  mask nullable [M]
  *   logprob [M] f32;  entropy, lse nullable [M] f32
+ * Rows with mask 0 output 0 and are taken out of the multiplication: the rows with mask 1 are packed
+ * into the workspace first (their number is found on the device) and only those are multiplied;
+ * the results are those of the call without a mask on these rows, bit for bit.
  * Requirements: K % 64 == 0, V % 8 == 0, H and W 16-byte aligned; otherwise
- * PPO_ERR_UNSUPPORTED.  workspace required (ppo_lmhead_workspace_bytes).
+ * PPO_ERR_UNSUPPORTED.  workspace required (ppo_lmhead_workspace_bytes: per-row partial results,
+ * the row order and room for the packed copy of H, M*K*2 bytes).
  */
 int ppo_lmhead_logprob_entropy(const void *H, const void *W, int64_t M, int64_t K, int64_t V,
                                const int32_t *tokens, const uint8_t *mask, float temperature,
