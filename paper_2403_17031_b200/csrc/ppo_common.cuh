@@ -412,6 +412,19 @@ int launch_logprob_pair(const void *policy_logits, const void *ref_logits, int d
 int launch_rollout(const ppo_step_io *io, int B, int T, const ppo_params *p, bool flags_cleared, cudaStream_t s);
 int launch_loss_finalize(int64_t rows, float vf_coef, float *losses, void *workspace, cudaStream_t s);
 
+// Workspace of the LM-head calls: header | per-row chunk partials of the forward call | row order [M] i32 |
+// packed copy of H [M, K] bf16 (offsets in bytes from the workspace base; ppo_lmhead_workspace_bytes = bytes)
+struct LmWorkspace {
+    size_t order_off, packed_off, bytes;
+};
+LmWorkspace lm_workspace(int64_t M, int64_t K, int64_t V);
+// Rows with mask 1 of H [M, K] packed, in row order, into the workspace's copy; their number goes to the header's
+// n_tokens, their original indices to the order array (the other rows' indices follow). The copy's rows from that
+// number up to the next multiple of 128 (or M) are zero-filled, so that a contraction over the packed rows may run
+// over whole blocks.
+int launch_lm_pack_rows(const void *H, int64_t M, int64_t K, const uint8_t *mask, void *workspace,
+                        const LmWorkspace &lay, cudaStream_t s);
+
 // tuning options (ppo_set_option)
 int option_value(int key);
 

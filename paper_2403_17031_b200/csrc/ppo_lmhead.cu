@@ -370,16 +370,21 @@ lmhead_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__
     }
 }
 
-// pack the rows with mask 1 (order[0 .. *n)) of H [M, K] into Hc; k16 = 16-byte pieces per row
+// pack the rows with mask 1 (order[0 .. *n)) of H [M, K] into Hc, zeros up to the next multiple of 128 rows;
+// k16 = 16-byte pieces per row
 __global__ void __launch_bounds__(256)
 lmhead_pack_rows_kernel(const uint4 *__restrict__ H, int k16, const int32_t *__restrict__ order, const int *__restrict__ n,
                         uint4 *__restrict__ Hc)
 {
-    const int j = blockIdx.x;
-    if (j >= *n) return;
-    const uint4 *src = H + (size_t)order[j] * k16;
+    const int j = blockIdx.x, rows = *n;
     uint4 *dst = Hc + (size_t)j * k16;
-    for (int i = threadIdx.x; i < k16; i += blockDim.x) dst[i] = src[i];
+    if (j < rows) {
+        const uint4 *src = H + (size_t)order[j] * k16;
+        for (int i = threadIdx.x; i < k16; i += blockDim.x) dst[i] = src[i];
+    } else if (j < ((rows + kBlockM - 1) / kBlockM) * kBlockM) {
+        const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+        for (int i = threadIdx.x; i < k16; i += blockDim.x) dst[i] = z;
+    }
 }
 
 // merge the chunk partials of each row in chunk order; one thread per row. With row compaction thread i holds
@@ -469,6 +474,30 @@ static void lm_shape(int64_t M, int64_t V, int *m_tiles, int *n_tiles, int *n_ch
     *n_chunks = (*n_tiles + kTilesPerChunk - 1) / kTilesPerChunk;
 }
 
+LmWorkspace lm_workspace(int64_t M, int64_t K, int64_t V)
+{
+    int m_tiles, n_tiles, n_chunks;
+    lm_shape(M, V, &m_tiles, &n_tiles, &n_chunks);
+    LmWorkspace w;
+    w.order_off = kHeaderBytes + lm_partials_bytes(m_tiles, n_chunks);
+    w.packed_off = w.order_off + align256((size_t)M * sizeof(int32_t));
+    w.bytes = w.packed_off + align256((size_t)M * (size_t)(K > 0 ? K : 0) * 2);
+    return w;
+}
+
+int launch_lm_pack_rows(const void *H, int64_t M, int64_t K, const uint8_t *mask, void *workspace,
+                        const LmWorkspace &lay, cudaStream_t s)
+{
+    unsigned char *ws = reinterpret_cast<unsigned char *>(workspace);
+    int32_t *order = reinterpret_cast<int32_t *>(ws + lay.order_off);
+    int rc = launch_row_order(mask, M, ws_header(workspace), order, s);
+    if (rc) return rc;
+    lmhead_pack_rows_kernel<<<(unsigned)M, 256, 0, s>>>(reinterpret_cast<const uint4 *>(H), (int)(K / 8), order,
+                                                      &ws_header(workspace)->n_tokens,
+                                                      reinterpret_cast<uint4 *>(ws + lay.packed_off));
+    return launch_status();
+}
+
 }   // namespace ppo
 
 using namespace ppo;
@@ -476,11 +505,7 @@ using namespace ppo;
 extern "C" size_t ppo_lmhead_workspace_bytes(int64_t M, int64_t K, int64_t V)
 {
     if (M <= 0 || V <= 0) return kHeaderBytes;
-    int m_tiles, n_tiles, n_chunks;
-    lm_shape(M, V, &m_tiles, &n_tiles, &n_chunks);
-    // header | per-row chunk partials | row order | packed copy of H (calls with a mask)
-    return kHeaderBytes + lm_partials_bytes(m_tiles, n_chunks) + align256((size_t)M * sizeof(int32_t)) +
-           align256((size_t)M * (size_t)(K > 0 ? K : 0) * 2);
+    return lm_workspace(M, K, V).bytes;
 }
 
 extern "C" int ppo_lmhead_logprob_entropy(const void *H, const void *W, int64_t M, int64_t K, int64_t V,
@@ -521,17 +546,12 @@ extern "C" int ppo_lmhead_logprob_entropy(const void *H, const void *W, int64_t 
     // 2*K*V flops saved per row with mask 0) and the kernels below work on the packed rows; the finalize kernel
     // writes every result at its original row.
     if (mask && a.m_tiles >= 2) {
-        int32_t *order = reinterpret_cast<int32_t *>(ws + kHeaderBytes + lm_partials_bytes(a.m_tiles, a.n_chunks));
-        uint4 *Hc = reinterpret_cast<uint4 *>(reinterpret_cast<unsigned char *>(order) + align256((size_t)M * sizeof(int32_t)));
-        rc = launch_row_order(mask, M, ws_header(workspace), order, s);
+        const LmWorkspace lay = lm_workspace(M, K, V);
+        rc = launch_lm_pack_rows(H, M, K, mask, workspace, lay, s);
         if (rc) return rc;
         a.m_eff = &ws_header(workspace)->n_tokens;
-        a.order = order;
-        lmhead_pack_rows_kernel<<<(unsigned)M, 256, 0, s>>>(reinterpret_cast<const uint4 *>(H), (int)(K / 8), order, a.m_eff,
-                                                          Hc);
-        rc = launch_status();
-        if (rc) return rc;
-        H = Hc;
+        a.order = reinterpret_cast<const int32_t *>(ws + lay.order_off);
+        H = ws + lay.packed_off;
     }
 
     CUtensorMap map_h, map_w;

@@ -164,6 +164,13 @@ struct Args {
     const float *g;              // gradient on the token log-probs
     float c, inv_tau;
     int *status;
+    // Row packing (the call was given a mask): the rows dimension holds the rows with mask 1 only and their
+    // number is known on the device: *dev_rows replaces Mdim (rows_role 1) or Kc (rows_role 2); the sizes above
+    // are upper bounds. in_map: pass 1 reads its per-row inputs at in_map[row]; out_map: the output row of
+    // packed row r is out_map[r].
+    const int *dev_rows;
+    int rows_role;
+    const int32_t *in_map, *out_map;
 };
 
 // EPI 0: out = accumulator (bf16). EPI 1: out = g * (onehot - 2^(acc*c - Y)) / tau, Y = lse * log2(e).
@@ -175,7 +182,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     __shared__ Smem sm;
     unsigned char *ring = smem_raw + ((1024u - (saddr(smem_raw) & 1023u)) & 1023u);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int k_blocks = (a.Kc + kBlockK - 1) / kBlockK;     // a ragged last block is zero-filled by the copies
+    // every role walks the same unit list with the same contraction length
+    int Mdim = a.Mdim, Kc = a.Kc, m_tiles = a.m_tiles, n_units = a.n_units;
+    if (a.dev_rows) {
+        const int n = max(0, min(*a.dev_rows, a.rows_role == 1 ? a.Mdim : a.Kc));
+        if (a.rows_role == 1) {
+            Mdim = n;
+            m_tiles = (n + kBlockM - 1) / kBlockM;
+            n_units = m_tiles * a.n_tiles;
+        } else {
+            Kc = n;
+        }
+    }
+    const int k_blocks = (Kc + kBlockK - 1) / kBlockK;     // a ragged last block is zero-filled by the copies
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -203,8 +222,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t it = 0;
-            for (int u = blockIdx.x; u < a.n_units; u += gridDim.x) {
-                const Unit un = unit_of(u, a.m_tiles, a.n_tiles, a.gm, a.gn);
+            for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+                const Unit un = unit_of(u, m_tiles, a.n_tiles, a.gm, a.gn);
                 const int m0 = un.m_tile * kBlockM, n0 = un.n_tile * kBlockN;
                 for (int kb = 0; kb < k_blocks; ++kb, ++it) {
                     const int s = it % kStages;
@@ -236,7 +255,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         if (lane == 0) {
             constexpr uint32_t idesc = instr_desc<A_MN, B_MN>();
             uint32_t it = 0, tc = 0;
-            for (int u = blockIdx.x; u < a.n_units; u += gridDim.x, ++tc) {
+            for (int u = blockIdx.x; u < n_units; u += gridDim.x, ++tc) {
                 const uint32_t buf = tc & 1;
                 if (tc >= 2) wait(&sm.tmem_empty[buf], ((tc >> 1) - 1) & 1, a.status);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -267,25 +286,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const int q = warp & 3;
         const int row_in_tile = q * 32 + lane;
         uint32_t tc = 0;
-        for (int u = blockIdx.x; u < a.n_units; u += gridDim.x, ++tc) {
-            const Unit un = unit_of(u, a.m_tiles, a.n_tiles, a.gm, a.gn);
+        for (int u = blockIdx.x; u < n_units; u += gridDim.x, ++tc) {
+            const Unit un = unit_of(u, m_tiles, a.n_tiles, a.gm, a.gn);
             const int row = un.m_tile * kBlockM + row_in_tile;
-            const bool row_ok = row < a.Mdim;
+            const bool row_ok = row < Mdim;
             // per-row scalars of the gradient epilogue
             int tok = -1;
             float gs = 0.f, off = 0.f;
             bool neg = false;
-            if (EPI == 1 && row_ok && (!a.mask || a.mask[row])) {
-                tok = a.tokens[row];
-                gs = a.g[row] * a.inv_tau;
-                off = log2f(fabsf(gs)) - a.lse[row] * kLog2e;     // -gs * 2^(y - Y) = -+ 2^(y - Y + log2|gs|)
+            const int src = (EPI == 1 && row_ok && a.in_map) ? a.in_map[row] : row;
+            if (EPI == 1 && row_ok && (!a.mask || a.mask[src])) {
+                tok = a.tokens[src];
+                gs = a.g[src] * a.inv_tau;
+                off = log2f(fabsf(gs)) - a.lse[src] * kLog2e;     // -gs * 2^(y - Y) = -+ 2^(y - Y + log2|gs|)
                 neg = gs > 0.f;
             }
             const uint32_t buf = tc & 1;
             wait(&sm.tmem_full[buf], (tc >> 1) & 1, a.status);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t taddr = tmem_base + buf * kBlockN + ((uint32_t)(q * 32) << 16);
-            __nv_bfloat16 *orow = a.out + (size_t)(row_ok ? row : 0) * a.Ndim;
+            __nv_bfloat16 *orow = a.out + (size_t)(row_ok ? (a.out_map ? a.out_map[row] : row) : 0) * a.Ndim;
 #pragma unroll 1
             for (int cc = 0; cc < kBlockN / 32; ++cc) {
                 uint32_t r[32];
@@ -318,8 +338,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                         }
                     }
                 } else {
+                    // (an empty contraction left the accumulator unwritten: the result is 0)
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+                    for (int j = 0; j < 32; ++j) v[j] = k_blocks > 0 ? __uint_as_float(r[j]) : 0.f;
                 }
                 // Ndim is a multiple of 8: whole 16-byte groups are inside or outside the row
 #pragma unroll
@@ -381,6 +402,18 @@ static int make_map(CUtensorMap *map, const void *base, uint64_t inner, uint64_t
     return r == CUDA_SUCCESS ? PPO_OK : (int)cudaErrorInvalidValue;
 }
 
+// zero rows [*n, next multiple of 128) of a [M, row16 * 16 bytes] matrix (at most 127 rows, none beyond M)
+__global__ void __launch_bounds__(256)
+zero_tail_rows_kernel(uint4 *__restrict__ base, int row16, const int *__restrict__ n, int M)
+{
+    const int rows = max(0, min(*n, M));
+    const int j = rows + blockIdx.x;
+    if (j >= M || j >= ((rows + kBlockM - 1) / kBlockM) * kBlockM) return;
+    uint4 *dst = base + (size_t)j * row16;
+    const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+    for (int i = threadIdx.x; i < row16; i += blockDim.x) dst[i] = z;
+}
+
 template <bool A_MN, bool B_MN, int EPI>
 static int launch_gemm(const CUtensorMap &ma, const CUtensorMap &mb, Args a, int gm, int gn, cudaStream_t s)
 {
@@ -429,8 +462,33 @@ extern "C" int ppo_lmhead_bwd(const void *H, const void *W, int64_t M, int64_t K
     bwd::Args a = {};
     a.status = status;
 
+    // With a mask (and more than one row tile) the rows with mask 0 are taken out of all three passes: the other
+    // rows of H are packed into the workspace, pass 1 writes their gradient rows packed at the front of dlogits
+    // (its per-row inputs are read through the row order), pass 2 writes each row of dH at its original place
+    // (dH is cleared first) and pass 3 contracts over the packed rows only. Their number is known on the device:
+    // the kernels read it from the workspace header. Rows of the packed H and D between that number and the next
+    // multiple of 128 are zero-filled, so the last contraction block of pass 3 adds nothing.
+    const bool packed = mask && M > bwd::kBlockM;
+    const int *n_rows = nullptr;
+    const int32_t *order = nullptr;
+    const void *Hp = H;
+    if (packed) {
+        const LmWorkspace lay = lm_workspace(M, K, V);
+        rc = launch_lm_pack_rows(H, M, K, mask, workspace, lay, s);
+        if (rc) return rc;
+        unsigned char *ws = reinterpret_cast<unsigned char *>(workspace);
+        n_rows = &ws_header(workspace)->n_tokens;
+        order = reinterpret_cast<const int32_t *>(ws + lay.order_off);
+        Hp = ws + lay.packed_off;
+        bwd::zero_tail_rows_kernel<<<bwd::kBlockM, 256, 0, s>>>(reinterpret_cast<uint4 *>(dlogits), (int)(V / 8), n_rows,
+                                                              (int)M);
+        rc = launch_status();
+        if (rc) return rc;
+        if (dH) PPO_RETURN_IF_CUDA(cudaMemsetAsync(dH, 0, (size_t)M * (size_t)K * 2, s));
+    }
+
     // pass 1: D = epilogue(H W): A = H [M,K] K-major, B = W [K,V] MN-major
-    rc = bwd::make_map(&ma, H, (uint64_t)K, (uint64_t)M, bwd::kBlockM);
+    rc = bwd::make_map(&ma, Hp, (uint64_t)K, (uint64_t)M, bwd::kBlockM);
     if (rc) return rc;
     rc = bwd::make_map(&mb, W, (uint64_t)V, (uint64_t)K, 64);
     if (rc) return rc;
@@ -438,8 +496,10 @@ extern "C" int ppo_lmhead_bwd(const void *H, const void *W, int64_t M, int64_t K
     a.out = reinterpret_cast<__nv_bfloat16 *>(dlogits);
     a.tokens = tokens; a.mask = mask; a.lse = lse; a.g = dlogprob;
     a.c = kLog2e / temperature; a.inv_tau = 1.0f / temperature;
+    a.dev_rows = n_rows; a.rows_role = 1; a.in_map = order; a.out_map = nullptr;
     rc = bwd::launch_gemm<false, true, 1>(ma, mb, a, 37, 4, s);
     if (rc) return rc;
+    a.in_map = nullptr;
 
     if (dH) {   // pass 2: dH [M,K] = D [M,V] . W[K,V]^T: A = D K-major, B = W K-major; contraction over V
         rc = bwd::make_map(&ma, dlogits, (uint64_t)V, (uint64_t)M, bwd::kBlockM);
@@ -448,16 +508,19 @@ extern "C" int ppo_lmhead_bwd(const void *H, const void *W, int64_t M, int64_t K
         if (rc) return rc;
         a.Mdim = (int)M; a.Ndim = (int)K; a.Kc = (int)V;
         a.out = reinterpret_cast<__nv_bfloat16 *>(dH);
+        a.out_map = order;
         rc = bwd::launch_gemm<false, false, 0>(ma, mb, a, 37, 4, s);
         if (rc) return rc;
+        a.out_map = nullptr;
     }
     if (dW) {   // pass 3: dW [K,V] = H[M,K]^T . D [M,V]: A = H MN-major, B = D MN-major; contraction over M
-        rc = bwd::make_map(&ma, H, (uint64_t)K, (uint64_t)M, 64);
+        rc = bwd::make_map(&ma, Hp, (uint64_t)K, (uint64_t)M, 64);
         if (rc) return rc;
         rc = bwd::make_map(&mb, dlogits, (uint64_t)V, (uint64_t)M, 64);
         if (rc) return rc;
         a.Mdim = (int)K; a.Ndim = (int)V; a.Kc = (int)M;
         a.out = reinterpret_cast<__nv_bfloat16 *>(dW);
+        a.rows_role = 2;
         rc = bwd::launch_gemm<true, true, 0>(ma, mb, a, 8, 18, s);
         if (rc) return rc;
     }

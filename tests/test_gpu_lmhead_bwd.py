@@ -29,6 +29,18 @@ def _wide(t):
     return t.detach().double().cpu().numpy()
 
 
+def _rows_in_place(dlogits, mask):
+    """dlogits as [M, V] with every row at its own place. Given a mask (and more than one 128-row tile) the call
+    leaves the gradient rows of the rows with mask 1 packed at the front of the buffer, in row order; the rest of
+    the buffer is scratch."""
+    if mask is None or dlogits.shape[0] <= 128:
+        return dlogits
+    rows = torch.nonzero(mask).flatten()
+    full = torch.zeros_like(dlogits)
+    full[rows] = dlogits[: rows.numel()]
+    return full
+
+
 def _check(P, M, K, V, seed, with_mask=True, tau=0.7):
     g = torch.Generator(device="cuda").manual_seed(seed)
     H = torch.randn((M, K), generator=g, device="cuda").to(torch.bfloat16)
@@ -44,12 +56,12 @@ def _check(P, M, K, V, seed, with_mask=True, tau=0.7):
     assert P.last_device_status(ws) == 0
     ref = B.lmhead_bwd(_wide(H), _wide(W), tok.cpu().numpy(), up.cpu().numpy().astype(np.float64), tau,
                        mask=None if mask is None else mask.cpu().numpy())
-    D, dH, dW = _wide(o["dlogits"]), _wide(o["dH"]), _wide(o["dW"])
+    D, dH, dW = _wide(_rows_in_place(o["dlogits"], mask)), _wide(o["dH"]), _wide(o["dW"])
     assert np.isfinite(D).all() and np.isfinite(dH).all() and np.isfinite(dW).all()
     bad = np.abs(D - ref["D"]) > REL * np.abs(ref["D"]) + 1e-6
     assert not bad.any(), "dlogits: %d off, worst %.3e" % (bad.sum(), np.abs(D - ref["D"])[bad].max())
     if mask is not None:
-        assert not D[mask.cpu().numpy() == 0].any()
+        assert not D[mask.cpu().numpy() == 0].any() and not dH[mask.cpu().numpy() == 0].any()
     assert not D[0].any()
     for name, got, want, scale in (("dH", dH, ref["dH"], ref["dH_abs"]), ("dW", dW, ref["dW"], ref["dW_abs"])):
         bad = np.abs(got - want) > REL * scale + REL * np.abs(want) + 1e-6
@@ -109,12 +121,16 @@ def test_lmhead_bwd_config4_full_size_sampled(P):
     idx = torch.from_numpy(rows).cuda()
     ref = B.lmhead_bwd(_wide(H[idx]), Wd, tok[idx].cpu().numpy(), up[idx].cpu().numpy().astype(np.float64), tau,
                        mask=mask[idx].cpu().numpy())
-    D, dH = _wide(o["dlogits"][idx]), _wide(o["dH"][idx])
+    n_real = len(real)
+    packed_at = torch.from_numpy(np.searchsorted(real, rows)).cuda()       # where a real row's gradient row was packed
+    D = _wide(o["dlogits"][packed_at.clamp_max(n_real - 1)])
+    D[mask[idx].cpu().numpy() == 0] = 0.0                                   # (rows with mask 0 have none)
+    dH = _wide(o["dH"][idx])
     bad = np.abs(D - ref["D"]) > REL * np.abs(ref["D"]) + 1e-9
     assert not bad.any(), "dlogits rows: %d off, worst %.3e" % (bad.sum(), np.abs(D - ref["D"])[bad].max())
     bad = np.abs(dH - ref["dH"]) > REL * ref["dH_abs"] + REL * np.abs(ref["dH"]) + 1e-9
     assert not bad.any(), "dH rows: %d off, worst %.3e" % (bad.sum(), np.abs(dH - ref["dH"])[bad].max())
-    assert not _wide(o["dlogits"][mask == 0][:64]).any()
+    assert not _wide(o["dH"][mask == 0][:64]).any()
     dW = o["dW"].float()
     assert torch.isfinite(dW).all()
     # rows of dW sum to zero up to the bf16 rounding of its 50304 entries
@@ -123,14 +139,16 @@ def test_lmhead_bwd_config4_full_size_sampled(P):
     cols = torch.from_numpy(np.sort(rng.choice(V, 64, replace=False))).cuda()
     u = torch.randn((K,), generator=g, device="cuda", dtype=torch.float64)
     lhs = u @ dW.double()[:, cols]
-    Dc = o["dlogits"][:, cols].double()
-    rhs = (H.double() @ u) @ Dc
-    scale = (H.double().abs() @ u.abs()) @ Dc.abs()      # sum_k |u_k| (|H|^T |D|)[k, v]: the scale of dW's rounding
+    Dc = o["dlogits"][:n_real, cols].double()                              # packed rows <-> H[real]
+    Hr = H[torch.from_numpy(real).cuda()].double()
+    rhs = (Hr @ u) @ Dc
+    scale = (Hr.abs() @ u.abs()) @ Dc.abs()      # sum_k |u_k| (|H|^T |D|)[k, v]: the scale of dW's rounding
     assert float(((lhs - rhs).abs() / scale.clamp_min(1e-30)).max()) < 2.0 ** -8
 
 
-def test_lmhead_bwd_all_rows_masked(P):
-    M, K, V = 200, 128, 1000
+@pytest.mark.parametrize("M", [100, 200])
+def test_lmhead_bwd_all_rows_masked(P, M):
+    K, V = 128, 1000
     H = torch.randn((M, K), device="cuda").to(torch.bfloat16)
     W = torch.randn((K, V), device="cuda").to(torch.bfloat16)
     tok = torch.randint(0, V, (M,), device="cuda", dtype=torch.int32)
@@ -139,5 +157,29 @@ def test_lmhead_bwd_all_rows_masked(P):
     o = P.lmhead_bwd(H, W, tok, lse, torch.ones(M, device="cuda"), 0.7, ws,
                      mask=torch.zeros(M, dtype=torch.uint8, device="cuda"))
     torch.cuda.synchronize()
-    assert not o["dlogits"].float().any() and not o["dH"].float().any() and not o["dW"].float().any()
+    # (M = 200 takes the packed path: no gradient row is written, dlogits is scratch)
+    assert (M > 128 or not o["dlogits"].float().any()) and not o["dH"].float().any() and not o["dW"].float().any()
+    assert P.last_device_status(ws) == 0
+
+
+def test_lmhead_bwd_packed_rows_equal_the_dense_call(P):
+    """Taking the rows with mask 0 out of the three passes must not change a bit of dH (row-local) and must give the
+    dW of the dense call up to the order of the fp32 sums over rows, which does not change either: the packed rows
+    keep their order and the rows left out contributed exact zeros."""
+    M, K, V = 900, 128, 1032
+    g = torch.Generator(device="cuda").manual_seed(11)
+    H = torch.randn((M, K), generator=g, device="cuda").to(torch.bfloat16)
+    W = (torch.randn((K, V), generator=g, device="cuda") * 0.2).to(torch.bfloat16)
+    tok = torch.randint(0, V, (M,), generator=g, device="cuda", dtype=torch.int32)
+    up = torch.randn((M,), generator=g, device="cuda")
+    mask = (torch.rand((M,), generator=g, device="cuda") < 0.5).to(torch.uint8)
+    ws = P.new_workspace(P.lmhead_workspace_bytes(M, K, V))
+    _, _, lse = P.lmhead_logprob_entropy(H, W, tok, 0.7, ws, want_lse=True)
+    dense = P.lmhead_bwd(H, W, tok, lse, up * mask, 0.7, ws)               # zero gradient on the rows left out
+    packed = P.lmhead_bwd(H, W, tok, lse, up, 0.7, ws, mask=mask)
+    torch.cuda.synchronize()
+    assert torch.equal(_rows_in_place(packed["dlogits"], mask), dense["dlogits"])
+    assert torch.equal(packed["dH"], dense["dH"])
+    rel = (packed["dW"].double() - dense["dW"].double()).abs().max() / dense["dW"].double().abs().max()
+    assert float(rel) < 2.0 ** -7
     assert P.last_device_status(ws) == 0
