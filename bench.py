@@ -517,7 +517,7 @@ def run_lmhead(args, cfg):
                              (M * K * 2 / 1e6, K * V * 2 / 1e6),
                        "lmhead_ms": lm_ms, "lmhead_bwd_ms": bwd_ms,
                        "real_tokens": n_real,
-                       "lmhead_bwd_tflops": None if bwd_ms is None else 3.0 * 2.0 * M * K * V / (bwd_ms * 1e-3) / 1e12,
+                       "lmhead_bwd_tflops": None if bwd_ms is None else 3.0 * flops / (bwd_ms * 1e-3) / 1e12,
                        "device_status": status},
             "roofline": {"bound": "tensor", "kernel": "lmhead_kernel (ppo_lmhead_logprob_entropy)", "achieved": tf,
                          "peak": peak, "peak_kind": kind + " (sustained)", "unit": "TFLOP/s", "frac": tf / peak,
@@ -525,7 +525,7 @@ def run_lmhead(args, cfg):
                          "timing": "CUDA events around the C-ABI call (row order, packing of the real rows, GEMM kernel, "
                                    "finalize kernel); flops = 2 x real rows x K x V"},
             "clocks": clk.summary(), "e2e": None, "cpu_baseline": None,
-            "gpu_launches": (13 + (3 if bwd_out is not None else 0)) * K_steps,
+            "gpu_launches": (13 + (6 if bwd_out is not None else 0)) * K_steps,
         }
         print(json.dumps(line), flush=True)
     if distributed:

@@ -364,9 +364,15 @@ int ppo_lmhead_logprob_entropy(const void *H, const void *W, int64_t M, int64_t 
  *   H [M,K], W [K,V]  bf16 as in ppo_lmhead_logprob_entropy;  tokens [M] i32;  mask nullable [M] u8
  *   lse [M] f32       the `lse` output of ppo_lmhead_logprob_entropy for the same H, W, temperature
  *   dlogprob [M] f32  upstream gradient (rows with mask 0 or dlogprob 0 give zero rows)
- *   dlogits [M,V] bf16  required scratch AND output: the only intermediate written to memory
- *   dH [M,K], dW [K,V]  bf16 outputs, each nullable (its pass is skipped)
- *   workspace  required (status word only), 256-byte aligned
+ *   dlogits [M,V] bf16  required scratch AND output: the only intermediate written to memory.
+ *                       Without a mask, or with M <= 128: every row at its place.  With a mask and
+ *                       M > 128 the rows with mask 0 are taken out of all three passes, and the
+ *                       buffer returns the gradient rows of the rows with mask 1 PACKED at its
+ *                       front, in row order (the rest of it is scratch)
+ *   dH [M,K], dW [K,V]  bf16 outputs, each nullable (its pass is skipped); rows of dH with mask 0
+ *                       are 0
+ *   workspace  required, ppo_lmhead_workspace_bytes(M, K, V) bytes (status word, row order, packed
+ *              copy of H), 256-byte aligned
  * Requirements: K % 8 == 0, V % 8 == 0, all matrices 16-byte aligned; else PPO_ERR_UNSUPPORTED /
  * PPO_ERR_ALIGN.  Token ids are assumed valid (the forward call reports bad ones).
  */
