@@ -320,7 +320,9 @@ def run_ours(args, cfg):
         devbuf = {k: torch.empty_like(v, device=dev) for k, v in host.items()}
         res_names = ["losses", "dvalues", "advantages_whitened", "returns", "logprob", "ref_logprob"]
         host_res = {k: torch.empty_like(hp.out[k], device="cpu").pin_memory() for k in res_names}
-        h2d = sum(v.numel() * v.element_size() for v in host.values())
+        # the call copies, of the two logits tensors, the real rows only (padding rows are never read)
+        h2d = sum(v.numel() * v.element_size() for k, v in host.items() if not k.endswith("logits"))
+        h2d += 2 * n_real * V * esize
         d2h = sum(v.numel() * v.element_size() for v in host_res.values())
         host_io = binding.PPOStepIO.from_tensors({**host, **host_res}, cuda=False)
         dev_io = hp.step_io(devbuf)

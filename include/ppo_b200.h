@@ -401,7 +401,9 @@ int ppo_lmhead_bwd(const void *H, const void *W, int64_t M, int64_t K, int64_t V
  *
  * ppo_step_host: `host` is a host struct of HOST pointers (pinned memory makes the copies
  * asynchronous), `dev` a host struct of DEVICE pointers used as staging and output buffers.  Copies
- * every input host -> device, runs ppo_step on `dev`, copies back each output whose pointer in
+ * every input host -> device (of the logits tensors only the rows ppo_step reads: each response's
+ * positions up to its first EOS, found from host->responses; the other rows of the staging buffers
+ * are left as they are), runs ppo_step on `dev`, copies back each output whose pointer in
  * `host` is not NULL, and waits for the stream.  Inputs that are NULL in `host` (loss_logits,
  * old_logprob) are treated as in ppo_step.
  */

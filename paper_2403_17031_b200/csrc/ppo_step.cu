@@ -64,6 +64,26 @@ int copy_in(void *dst, const void *src, size_t bytes, cudaStream_t s)
     return PPO_OK;
 }
 
+// A [B, T, V] logits tensor: only the rows that ppo_step reads are copied - of each response the positions up to
+// and including its first EOS (the EOS trick masks the rest out of every step; found here from the host's tokens).
+int copy_in_real_rows(void *dst, const void *src, const int32_t *responses, int32_t B, int32_t T, size_t row_bytes,
+                      int32_t eos_id, cudaStream_t s)
+{
+    if (!src) return PPO_OK;
+    if (!dst) return PPO_ERR_NULL;
+    for (int32_t b = 0; b < B; ++b) {
+        const int32_t *r = responses + (size_t)b * T;
+        int32_t L = T;
+        for (int32_t t = 0; t < T; ++t)
+            if (r[t] == eos_id) { L = t + 1; break; }
+        const size_t off = (size_t)b * T * row_bytes;
+        PPO_RETURN_IF_CUDA(cudaMemcpyAsync(static_cast<unsigned char *>(dst) + off,
+                                           static_cast<const unsigned char *>(src) + off, (size_t)L * row_bytes,
+                                           cudaMemcpyHostToDevice, s));
+    }
+    return PPO_OK;
+}
+
 int copy_out(void *dst, const void *src, size_t bytes, cudaStream_t s)
 {
     if (!dst) return PPO_OK;          // the caller does not want this output on the host
@@ -93,9 +113,12 @@ extern "C" int ppo_step_host(const ppo_step_io *host, const ppo_step_io *dev, in
     const size_t bt = (size_t)B * (size_t)T, es = dtype == PPO_F32 ? 4 : 2;
     const size_t logits_bytes = bt * (size_t)V * es;
     // device staging buffers are written here, so drop the const the struct carries for inputs
-    PPO_TRY(copy_in(const_cast<void *>(dev->policy_logits), host->policy_logits, logits_bytes, s));
-    PPO_TRY(copy_in(const_cast<void *>(dev->ref_logits), host->ref_logits, logits_bytes, s));
-    PPO_TRY(copy_in(const_cast<void *>(dev->loss_logits), host->loss_logits, logits_bytes, s));
+    PPO_TRY(copy_in_real_rows(const_cast<void *>(dev->policy_logits), host->policy_logits, host->responses, B, T,
+                              (size_t)V * es, p->eos_id, s));
+    PPO_TRY(copy_in_real_rows(const_cast<void *>(dev->ref_logits), host->ref_logits, host->responses, B, T,
+                              (size_t)V * es, p->eos_id, s));
+    PPO_TRY(copy_in_real_rows(const_cast<void *>(dev->loss_logits), host->loss_logits, host->responses, B, T,
+                              (size_t)V * es, p->eos_id, s));
     PPO_TRY(copy_in(const_cast<int32_t *>(dev->responses), host->responses, bt * 4, s));
     PPO_TRY(copy_in(const_cast<float *>(dev->scores), host->scores, (size_t)B * 4, s));
     PPO_TRY(copy_in(const_cast<float *>(dev->values), host->values, bt * 4, s));
