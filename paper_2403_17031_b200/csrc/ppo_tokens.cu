@@ -268,7 +268,7 @@ loss_prepare_kernel(const uint8_t *__restrict__ mask, int64_t rows, WorkspaceHea
 }
 
 // ---------------------------------------------------------------- fused launch of ppo_step
-// Everything token-level in one launch, after the log-prob launch (which does not need the mask):
+// Everything token-level in one launch, after the log-prob launch (which finds the padding rows by itself):
 // one warp per sequence runs the EOS trick, the KL rewards and GAE; one extra block runs the loss
 // prologue (token count, row order) as soon as every sequence has had the EOS trick, and the last
 // sequence block to finish whitens the advantages of the whole batch - each with exactly the code and
