@@ -377,6 +377,9 @@ def run_ours(args, cfg):
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": "config%d %s" % (cfg.index, cfg.name), "B_per_gpu": B, "T": T, "V": V,
                        "logits_dtype": cfg.dtype, "real_tokens": n_real,
+                       # `value` counts all B*T response positions of the batch (padding after the first EOS
+                       # included, as the workload is stated); this one counts the positions before it only
+                       "real_tokens_per_s": n_real * world / (ms_per_step * 1e-3),
                        "l2": "inputs larger than L2 (%.0f MB of logits read on the %d real rows, 3 tensors, + %.0f MB "
                              "of gradient written per step; padding rows are not read)" %
                              (3 * n_real * V * esize / 1e6, n_real, R / 1e6),
