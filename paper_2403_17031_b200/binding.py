@@ -195,6 +195,12 @@ def lmhead_workspace_bytes(M: int, K: int, V: int) -> int:
     return int(lib().ppo_lmhead_workspace_bytes(M, K, V))
 
 
+def _need_workspace(workspace: torch.Tensor, nbytes: int, what: str) -> None:
+    """The C entry points take no workspace size; refuse a buffer that is too small before the call."""
+    if workspace is None or workspace.numel() * workspace.element_size() < nbytes:
+        raise ValueError("%s needs a workspace of %d bytes (lmhead_workspace_bytes)" % (what, nbytes))
+
+
 def new_workspace(nbytes: int, device="cuda") -> torch.Tensor:
     """Allocate (torch) and clear a workspace of at least `nbytes`."""
     ws = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
@@ -374,6 +380,7 @@ def lmhead_logprob_entropy(H, W, tokens, temperature: float, workspace, mask=Non
         out = (torch.empty(M, dtype=torch.float32, device=dev), torch.empty(M, dtype=torch.float32, device=dev),
                torch.empty(M, dtype=torch.float32, device=dev) if want_lse else None)
     lp, ent, lse = out
+    _need_workspace(workspace, lmhead_workspace_bytes(M, K, V), "lmhead_logprob_entropy")
     rc = lib().ppo_lmhead_logprob_entropy(_ptr(H, torch.bfloat16, "H"), _ptr(W, torch.bfloat16, "W"), M, K, V,
                                           _ptr(tokens, torch.int32, "tokens"), _ptr(mask, torch.uint8),
                                           float(temperature), _ptr(lp, torch.float32), _ptr(ent, torch.float32),
@@ -439,6 +446,7 @@ def lmhead_bwd(H, W, tokens, lse, dlogprob, temperature: float, workspace, mask=
     if out is None:
         out = {"dlogits": dlogits if dlogits is not None else torch.empty((M, V), dtype=torch.bfloat16, device=H.device),
                "dH": torch.empty_like(H) if want_dH else None, "dW": torch.empty_like(W) if want_dW else None}
+    _need_workspace(workspace, lmhead_workspace_bytes(M, K, V), "lmhead_bwd")
     rc = lib().ppo_lmhead_bwd(_ptr(H, torch.bfloat16), _ptr(W, torch.bfloat16), M, K, V, _ptr(tokens, torch.int32),
                               _ptr(mask, torch.uint8), _ptr(lse, torch.float32), _ptr(dlogprob, torch.float32),
                               float(temperature), _ptr(out["dlogits"], torch.bfloat16), _ptr(out["dH"]),

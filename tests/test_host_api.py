@@ -49,6 +49,15 @@ def test_workspace_sizes(L):
     assert binding.workspace_bytes(0, 53, 50304) == 256
     assert binding.workspace_bytes(512, 53, 50304) % 256 == 0
     assert binding.lmhead_workspace_bytes(27136, 4096, 50304) % 256 == 0
+    # header | 16 bytes per (row of a 128-row tile, chunk of 6 x 256 vocabulary columns) | row order | packed copy of H
+    a256 = lambda x: (x + 255) // 256 * 256
+    M, K, V = 1000, 512, 5000
+    tiles, chunks = (M + 127) // 128, ((V + 255) // 256 + 5) // 6
+    assert binding.lmhead_workspace_bytes(M, K, V) == 256 + a256(tiles * 128 * chunks * 16) + a256(M * 4) + a256(M * K * 2)
+    import pytest
+    import torch
+    with pytest.raises(ValueError):     # the binding refuses a workspace that is too small before any call
+        binding._need_workspace(torch.empty(1024, dtype=torch.uint8), binding.lmhead_workspace_bytes(M, K, V), "x")
 
 
 FAKE = 0x10000   # a non-null, 256-byte aligned address that is never dereferenced on these paths
