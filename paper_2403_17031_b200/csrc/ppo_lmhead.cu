@@ -20,6 +20,10 @@
 // workspace; a second small kernel merges a row's partials in chunk order and writes log-prob,
 // entropy and lse.
 //
+// Given a mask, the call first packs the rows with mask 1 into the workspace (row order and count found on the
+// device) and this kernel multiplies only those; it reads the row count from the workspace header, so its unit
+// list is as long as the packed rows need, and the second kernel writes each result at its original row.
+//
 // Every wait is bounded; a wait that runs out sets PPO_DEV_TIMEOUT and the block carries on with the
 // same control flow, so it still reaches the end, frees its tensor memory and returns.
 #include <cuda.h>

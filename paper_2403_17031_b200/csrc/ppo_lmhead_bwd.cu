@@ -10,7 +10,8 @@
 //   pass 2  dH = D W^T   (A = D, contraction over the vocabulary; both operands K-major);
 //   pass 3  dW = H^T D   (A = H^T, contraction over the rows; both operands MN-major, read as stored).
 // D is the only intermediate that touches HBM (M*V*2 bytes, written once and read by passes 2 and 3);
-// the logits themselves never do.
+// the logits themselves never do. Given a mask, the rows with mask 0 (zero rows of D) are taken out of all three
+// passes: H is packed first, D is written packed, and the kernels take the row count from the workspace header.
 //
 // Kernel structure (same as the forward kernel): one persistent block per SM, 192 threads: warp 0 = TMA
 // producer (4-stage ring, 128-byte swizzle), warp 1 = tcgen05.mma issuer (M = 128, N = 256, K = 16 per
