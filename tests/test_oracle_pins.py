@@ -119,6 +119,30 @@ def test_mask_neg_inf_and_bad_token(oracle):
     assert math.isnan(lp[2]) and math.isnan(H[2])
 
 
+def test_masked_rows_are_not_read_and_change_nothing_downstream(oracle):
+    """The chained path gives step 1 the mask of the EOS trick: rows with mask 0 output exactly 0 whatever they
+    hold (NaN included, and no status for a bad token there), rows with mask 1 are untouched by the option, and the
+    KL rewards built from either version are identical (step 3 multiplies by the same mask)."""
+    rng = np.random.default_rng(12)
+    x = rng.normal(0, 2, (6, 40)).astype(np.float32)
+    tok = np.array([3, 7, 1, 39, 0, 11], np.int32)
+    mask = np.array([1, 1, 0, 1, 0, 0], np.uint8)
+    full = oracle.logprob_entropy(x, tok, 0.7)
+    y = x.copy()
+    y[mask == 0] = np.nan
+    tok2 = tok.copy()
+    tok2[2] = 1000                                    # outside the vocabulary, but on a row with mask 0
+    part = oracle.logprob_entropy(y, tok2, 0.7, mask=mask)
+    for a, b in zip(full, part):
+        assert np.array_equal(a[mask == 1], b[mask == 1])
+        assert not b[mask == 0].any()
+    ref = full[0] - 0.01
+    m2, L = mask.reshape(1, 6).copy(), np.array([6], np.int32)
+    kl_a, rew_a = oracle.kl_rewards(full[0].reshape(1, 6), ref.reshape(1, 6), m2, L, np.array([0.5]), 0.05)
+    kl_b, rew_b = oracle.kl_rewards(part[0].reshape(1, 6), (ref * mask).reshape(1, 6), m2, L, np.array([0.5]), 0.05)
+    assert np.array_equal(kl_a, kl_b) and np.array_equal(rew_a, rew_b)
+
+
 # ---------------------------------------------------------------- step 2: EOS trick
 def test_truncate_hand_rows(oracle):
     E, P = 0, 1
