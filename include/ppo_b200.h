@@ -59,6 +59,7 @@ extern "C" {
 #define PPO_DEV_EMPTY_MASK 2     /* mask selected no element: statistics / losses are 0 */
 #define PPO_DEV_TIMEOUT 4        /* a bounded wait inside a kernel gave up; outputs are invalid */
 #define PPO_DEV_BAD_ROW 8        /* ppo_sample_logprob_entropy: a row had a NaN / +inf or no finite logit: token -1 */
+#define PPO_DEV_BAD_REUSE 16     /* ppo_loss_fwd_bwd_next_epoch: the workspace does not hold this mask's row order; nothing was written */
 
 /* indices into the losses[8] output of ppo_loss_fwd_bwd */
 enum { PPO_LOSS_PG = 0, PPO_LOSS_VF = 1, PPO_LOSS_TOTAL = 2, PPO_LOSS_APPROX_KL = 3,
@@ -220,6 +221,23 @@ int ppo_whiten(const float *x, const uint8_t *mask, int64_t n_elems, int shift_m
  * Per-row partial sums are reduced in a fixed order in fp64, so results are bit-reproducible.
  */
 int ppo_loss_fwd_bwd(const void *logits, int dtype, int32_t B, int32_t T, int64_t V,
+                     const int32_t *tokens, const uint8_t *mask, const float *old_logprob,
+                     const float *advantages, const float *values_new, const float *values_old,
+                     const float *returns, const ppo_params *p /* host */, float *losses,
+                     void *dlogits, float *dvalues, float *new_logprob, float *entropy,
+                     float *dlogprob, void *workspace, void *stream);
+
+/*
+ * The same call for the later PPO epochs of a batch (the paper's table: 4 epochs per batch): it must follow a
+ * ppo_loss_fwd_bwd, ppo_loss_fwd_bwd_next_epoch or ppo_step call on the same workspace with the same mask
+ * pointer, B and T, with no other call that uses this workspace in between.  The token count and row order
+ * that call left in the workspace are reused, which saves the prologue launch; all other arguments (logits,
+ * old_logprob, ...) may differ, the results are those of ppo_loss_fwd_bwd.  The kernel checks that the
+ * order in the workspace was built from this mask pointer, row count and workspace; if not, it sets
+ * PPO_DEV_BAD_REUSE in the device status and writes nothing.  The CONTENT of mask must not have changed
+ * since (not checked).
+ */
+int ppo_loss_fwd_bwd_next_epoch(const void *logits, int dtype, int32_t B, int32_t T, int64_t V,
                      const int32_t *tokens, const uint8_t *mask, const float *old_logprob,
                      const float *advantages, const float *values_new, const float *values_old,
                      const float *returns, const ppo_params *p /* host */, float *losses,

@@ -83,6 +83,8 @@ _SIGS = {
                              C.c_void_p, C.c_void_p]),
     "ppo_loss_fwd_bwd": (C.c_int, [C.c_void_p, C.c_int, C.c_int32, C.c_int32, C.c_int64] + [C.c_void_p] * 7 +
                          [C.POINTER(PPOParams)] + [C.c_void_p] * 8),
+    "ppo_loss_fwd_bwd_next_epoch": (C.c_int, [C.c_void_p, C.c_int, C.c_int32, C.c_int32, C.c_int64] +
+                                    [C.c_void_p] * 7 + [C.POINTER(PPOParams)] + [C.c_void_p] * 8),
     "ppo_loss_from_logprob": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32] + [C.c_void_p] * 6 +
                               [C.POINTER(PPOParams)] + [C.c_void_p] * 5),
     "ppo_loss_from_logprob_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32] + [C.c_void_p] * 6 +
@@ -297,8 +299,10 @@ def whiten(x, mask=None, shift_mean: bool = True, eps: float = 1e-8, workspace=N
 
 
 def loss_fwd_bwd(logits, tokens, mask, old_logprob, advantages, values_new, values_old, returns,
-                 params: PPOParams, workspace, want_dlogits: bool = True, want_aux: bool = True, out=None):
-    """Returns dict(losses[8], dlogits, dvalues, new_logprob, entropy, dlogprob)."""
+                 params: PPOParams, workspace, want_dlogits: bool = True, want_aux: bool = True, out=None,
+                 next_epoch: bool = False):
+    """Returns dict(losses[8], dlogits, dvalues, new_logprob, entropy, dlogprob). next_epoch: this call follows a
+    loss call (or step) on the same workspace with the same mask tensor and reuses its row order."""
     B, T, V = logits.shape
     dev = logits.device
     if out is None:
@@ -311,13 +315,12 @@ def loss_fwd_bwd(logits, tokens, mask, old_logprob, advantages, values_new, valu
             "dlogprob": torch.empty((B, T), dtype=torch.float32, device=dev) if want_aux else None,
         }
     f32 = torch.float32
-    rc = lib().ppo_loss_fwd_bwd(_ptr(logits, None, "logits"), _logits_dtype(logits), B, T, V,
-                                _ptr(tokens, torch.int32, "tokens"), _ptr(mask, torch.uint8, "mask"),
-                                _ptr(old_logprob, f32), _ptr(advantages, f32), _ptr(values_new, f32),
-                                _ptr(values_old, f32), _ptr(returns, f32), C.byref(params),
-                                _ptr(out["losses"], f32), _ptr(out["dlogits"], logits.dtype),
-                                _ptr(out["dvalues"], f32), _ptr(out["new_logprob"], f32), _ptr(out["entropy"], f32),
-                                _ptr(out["dlogprob"], f32), _ptr(workspace), _stream())
+    fn = lib().ppo_loss_fwd_bwd_next_epoch if next_epoch else lib().ppo_loss_fwd_bwd
+    rc = fn(_ptr(logits, None, "logits"), _logits_dtype(logits), B, T, V, _ptr(tokens, torch.int32, "tokens"),
+            _ptr(mask, torch.uint8, "mask"), _ptr(old_logprob, f32), _ptr(advantages, f32), _ptr(values_new, f32),
+            _ptr(values_old, f32), _ptr(returns, f32), C.byref(params), _ptr(out["losses"], f32),
+            _ptr(out["dlogits"], logits.dtype), _ptr(out["dvalues"], f32), _ptr(out["new_logprob"], f32),
+            _ptr(out["entropy"], f32), _ptr(out["dlogprob"], f32), _ptr(workspace), _stream())
     _check("ppo_loss_fwd_bwd", rc)
     return out
 

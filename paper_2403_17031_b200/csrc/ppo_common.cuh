@@ -1,6 +1,7 @@
 // Shared device/host helpers of the PPO hot-path kernels (sm_100a).
 #pragma once
 
+#include <cstddef>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <math.h>
@@ -25,8 +26,13 @@ struct WorkspaceHeader {
     int order_ready;   // n_tokens + 1 once token count, counters and row order of the loss call in flight are written
     int adv_ready;     // 1 once the advantages / returns that the loss call reads are written
     int step_blocks2;  // second ticket of ppo_step's token-level kernel (resets itself)
-    int reserved[55];
+    int reserved[9];
+    // what the row order in this workspace was built from: mask pointer, number of rows, order pointer. A loss call
+    // that reuses the order (ppo_loss_fwd_bwd_next_epoch) checks its own arguments against these.
+    unsigned long long order_sig[3];
+    int reserved2[40];
 };
+static_assert(offsetof(WorkspaceHeader, order_sig) % 8 == 0, "aligned 64-bit words");
 static_assert(sizeof(WorkspaceHeader) == 256, "header is one 256-byte block");
 
 constexpr int kPartialsPerToken = 8;   // pg, vf, kl, pg_clipped, vf_clipped, entropy, unused, unused
@@ -397,7 +403,7 @@ int loss_fwd_bwd_prepared(const void *logits, int dtype, int32_t B, int32_t T, i
                           const uint8_t *mask, const float *old_logprob, const float *advantages,
                           const float *values_new, const float *values_old, const float *returns, const ppo_params *p,
                           float *losses, void *dlogits, float *dvalues, float *new_logprob, float *entropy,
-                          float *dlogprob, void *workspace, void *stream, bool prepared);
+                          float *dlogprob, void *workspace, void *stream, bool prepared, bool reuse = false);
 int launch_loss_prepare(const uint8_t *mask, int64_t rows, void *workspace, cudaStream_t s);
 // the same prologue with the order array at a place of the caller's choice: hdr->n_tokens = number of rows with
 // mask 1, order[0 .. n_tokens) = those rows (ascending), order[n_tokens .. rows) = the other rows

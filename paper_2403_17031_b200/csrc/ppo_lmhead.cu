@@ -397,8 +397,11 @@ __global__ void __launch_bounds__(256)
 lmhead_finalize_kernel(const float4 *__restrict__ partials, int M, int V, int n_chunks, const int32_t *__restrict__ tokens,
                        const uint8_t *__restrict__ mask, const int32_t *__restrict__ order,
                        const int *__restrict__ m_eff, float c, float *__restrict__ logprob,
-                       float *__restrict__ entropy, float *__restrict__ lse, int *status)
+                       float *__restrict__ entropy, float *__restrict__ lse, int *status,
+                       unsigned long long *order_sig)
 {
+    // the partials of this call lie where a loss call keeps its row order: that order is void from here on
+    if (blockIdx.x == 0 && threadIdx.x == 0) order_sig[0] = 0ull;
     const int packed = blockIdx.x * blockDim.x + threadIdx.x;
     if (packed >= M) return;
     const int row = order ? order[packed] : packed;
@@ -585,6 +588,7 @@ extern "C" int ppo_lmhead_logprob_entropy(const void *H, const void *W, int64_t 
     rc = launch_status();
     if (rc) return rc;
     lmhead_finalize_kernel<<<(unsigned)((M + 255) / 256), 256, 0, s>>>(a.partials, a.M, a.V, a.n_chunks, tokens, mask, a.order,
-                                                                       a.m_eff, a.c, logprob, entropy, lse, a.status);
+                                                                       a.m_eff, a.c, logprob, entropy, lse, a.status,
+                                                                       ws_header(workspace)->order_sig);
     return launch_status();
 }

@@ -392,11 +392,24 @@ extern "C" int ppo_loss_fwd_bwd(const void *logits, int dtype, int32_t B, int32_
                                  false);
 }
 
+extern "C" int ppo_loss_fwd_bwd_next_epoch(const void *logits, int dtype, int32_t B, int32_t T, int64_t V,
+                                           const int32_t *tokens, const uint8_t *mask, const float *old_logprob,
+                                           const float *advantages, const float *values_new,
+                                           const float *values_old, const float *returns, const ppo_params *p,
+                                           float *losses, void *dlogits, float *dvalues, float *new_logprob,
+                                           float *entropy, float *dlogprob, void *workspace, void *stream)
+{
+    return loss_fwd_bwd_prepared(logits, dtype, B, T, V, tokens, mask, old_logprob, advantages, values_new, values_old,
+                                 returns, p, losses, dlogits, dvalues, new_logprob, entropy, dlogprob, workspace, stream,
+                                 false, true);
+}
+
 int ppo::loss_fwd_bwd_prepared(const void *logits, int dtype, int32_t B, int32_t T, int64_t V, const int32_t *tokens,
                                const uint8_t *mask, const float *old_logprob, const float *advantages,
                                const float *values_new, const float *values_old, const float *returns,
                                const ppo_params *p, float *losses, void *dlogits, float *dvalues, float *new_logprob,
-                               float *entropy, float *dlogprob, void *workspace, void *stream, bool prepared)
+                               float *entropy, float *dlogprob, void *workspace, void *stream, bool prepared,
+                               bool reuse)
 {
     if (dtype != PPO_F32 && dtype != PPO_BF16) return PPO_ERR_DTYPE;
     if (B <= 0 || T <= 0 || V <= 0 || V >= ((int64_t)1 << 31) || (int64_t)B * T >= ((int64_t)1 << 31))
@@ -414,7 +427,9 @@ int ppo::loss_fwd_bwd_prepared(const void *logits, int dtype, int32_t B, int32_t
     if (dlogits == logits) return PPO_ERR_PARAM;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     const int64_t rows = (int64_t)B * T;
-    int rc = prepared ? PPO_OK : launch_loss_prepare(mask, rows, workspace, s);
+    // reuse: the row order of the previous loss call on this workspace serves this call too (same mask): the bulk
+    // engine starts at once; the kernels that cannot check this run the prologue as usual
+    int rc = (prepared || reuse) ? PPO_OK : launch_loss_prepare(mask, rows, workspace, s);
     if (rc) return rc;
     LossArgs a;
     a.logits = logits;
@@ -443,8 +458,12 @@ int ppo::loss_fwd_bwd_prepared(const void *logits, int dtype, int32_t B, int32_t
     a.c1 = p->vf_coef;
     rc = PPO_ERR_UNSUPPORTED;
     if (option_value(PPO_OPT_ROW_ENGINE) != 1) {
-        rc = launch_loss_bulk(a, dtype, workspace, losses, p->vf_coef, true, s);
+        rc = launch_loss_bulk(a, dtype, workspace, losses, p->vf_coef, !reuse, s, reuse);
         if (rc != PPO_ERR_UNSUPPORTED) return rc;      // the engine reduces the partials itself
+    }
+    if (reuse) {
+        rc = launch_loss_prepare(mask, rows, workspace, s);
+        if (rc) return rc;
     }
     rc = dtype == PPO_F32 ? launch_loss<float>(a, s) : launch_loss<__nv_bfloat16>(a, s);
     if (rc) return rc;

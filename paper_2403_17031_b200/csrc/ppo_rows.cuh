@@ -252,7 +252,9 @@ int launch_logprob_bulk(const void *logits, int dtype, int64_t rows, int V, int6
 // (the engine's loss kernel also reduces the partials and writes `losses` itself)
 // `dependent`: launch so that the kernel may start while the kernel before it in the stream still runs (it
 // waits for the workspace header's flags before it reads that kernel's results)
+// `reuse`: no prologue ran for this call; the kernel checks that the order in the workspace was built from this
+// call's mask (PPO_DEV_BAD_REUSE and nothing written otherwise)
 int launch_loss_bulk(const LossArgs &a, int dtype, void *workspace, float *losses, float vf_coef, bool dependent,
-                     cudaStream_t s);
+                     cudaStream_t s, bool reuse = false);
 
 }   // namespace ppo

@@ -44,6 +44,7 @@ struct EngineSmem {
     int is_last;
     int ring[4];           // row of the block's k-th item at [k % 4], -1 = no further item
     int n_tokens;          // step 6: number of mask==1 rows of the call
+    int abort;             // step 6: the order that this call was told to reuse is not the one of its mask
     double lred[6 * 32];
     alignas(128) unsigned char zeros[kZeroBytes];
 };
@@ -281,6 +282,7 @@ struct EngineArgs {
     float *losses;
     float vf_coef;
     int wait_flags;         // the launch overlaps the kernel that produces order / advantages: poll the header's flags
+    int reuse;              // no prologue ran for this call: the order in the workspace must be the one of this mask
 };
 
 template <int CONS>
@@ -304,6 +306,12 @@ __device__ __forceinline__ void engine_epilogue(const EngineArgs &a, EngineSmem 
     __threadfence();
     reduce_loss_partials<CONS + 64>(a.loss.partials, a.loss.rows, sm.n_tokens, a.vf_coef, a.losses, sm.lred,
                                     (int)threadIdx.x, [] { block_sync_all<CONS>(); });
+    // every block is past the work counters: leave them ready for a call that reuses this order
+    if (threadIdx.x == 0) {
+        a.hdr->masked_next = 0;
+        a.hdr->real_next = 0;
+        a.hdr->done_blocks = 0;
+    }
 }
 
 // sign flip of a packed gradient (both bf16 halves of each word, or each fp32 word)
@@ -372,9 +380,20 @@ row_engine_kernel(const EngineArgs a)
     // step 6 inside ppo_step: this kernel may have been launched while the token-level kernel is still at
     // work; everything above touched shared memory only, from here on it reads what that kernel publishes
     // (the first flag carries the token count)
-    if (MODE == 1 && threadIdx.x == 0)
+    if (MODE == 1 && threadIdx.x == 0) {
+        sm.abort = 0;
+        if (a.reuse) {   // the order must have been built from this mask, for this many rows, at this place
+            const unsigned long long *sig = a.hdr->order_sig;
+            if (sig[0] != (unsigned long long)reinterpret_cast<uintptr_t>(a.mask) || sig[1] != (unsigned long long)a.rows ||
+                sig[2] != (unsigned long long)reinterpret_cast<uintptr_t>(a.order)) {
+                atomicOr(status, PPO_DEV_BAD_REUSE);
+                sm.abort = 1;
+            }
+        }
         sm.n_tokens = a.wait_flags ? max(flag_wait(&a.hdr->order_ready, status) - 1, 0) : a.hdr->n_tokens;
+    }
     __syncthreads();
+    if (MODE == 1 && sm.abort) return;   // nothing is read or written through an order that is not this call's
     // number of work items of the streaming phase
     const int64_t n_items = MODE == 0 ? a.rows : (int64_t)sm.n_tokens;
 
@@ -787,7 +806,7 @@ int launch_logprob_bulk(const void *logits, int dtype, int64_t rows, int V, int6
 }
 
 int launch_loss_bulk(const LossArgs &la, int dtype, void *workspace, float *losses, float vf_coef, bool dependent,
-                     cudaStream_t s)
+                     cudaStream_t s, bool reuse)
 {
     if (!la.dlogits || !aligned16(la.dlogits)) return PPO_ERR_UNSUPPORTED;
     EngineArgs a = {};
@@ -805,6 +824,7 @@ int launch_loss_bulk(const LossArgs &la, int dtype, void *workspace, float *loss
     a.losses = losses;
     a.vf_coef = vf_coef;
     a.wait_flags = dependent ? 1 : 0;
+    a.reuse = reuse ? 1 : 0;
     if (dtype == PPO_F32) {
         if (!bulk_ok<float>(la.logits, la.V, la.V)) return PPO_ERR_UNSUPPORTED;
         return launch_engine<float, 1, true>(a, la.rows, dependent, s);

@@ -224,6 +224,9 @@ __device__ __forceinline__ void loss_prepare_block(const uint8_t *mask, int64_t 
             hdr->masked_next = 0;
             hdr->real_next = 0;
             hdr->done_blocks = 0;
+            hdr->order_sig[0] = (unsigned long long)reinterpret_cast<uintptr_t>(mask);
+            hdr->order_sig[1] = (unsigned long long)rows;
+            hdr->order_sig[2] = (unsigned long long)reinterpret_cast<uintptr_t>(order);
             if (wi == 0 && flag_empty) atomicOr(&hdr->status, PPO_DEV_EMPTY_MASK);
         }
     }

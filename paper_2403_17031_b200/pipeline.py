@@ -62,11 +62,14 @@ class PPOHotPath:
                   out=o["advantages_whitened"], stats=o["whiten_stats"])
         return o
 
-    def loss(self, logits, responses, old_logprob, values_new, values_old):
-        """Step 6 on the loss-time logits, using the advantages/returns of rollout_stats."""
+    def loss(self, logits, responses, old_logprob, values_new, values_old, next_epoch: bool = False):
+        """Step 6 on the loss-time logits, using the advantages/returns of rollout_stats or step.
+        next_epoch: a later PPO epoch on the same batch (the call before this one on this object was loss() or
+        step()): the row order left in the workspace is reused, one launch less."""
         o = self.out
         _b.loss_fwd_bwd(logits, responses, o["mask"], old_logprob, o["advantages_whitened"], values_new,
-                        values_old, o["returns"], self.params, self.workspace, out=self._loss_out)
+                        values_old, o["returns"], self.params, self.workspace, out=self._loss_out,
+                        next_epoch=next_epoch)
         return o
 
     def step(self, policy_logits, ref_logits, responses, scores, values, values_new, old_logprob=None,

@@ -420,3 +420,76 @@ def test_step_never_reads_padding_rows(P, B, T, V, dtype):
     for k in names:
         assert torch.equal(a.out[k], b.out[k]), k
     assert b.device_status() == 0
+
+
+@pytest.mark.parametrize("B,T,V,dtype", [(64, 53, 50304, "bf16"), (37, 53, 2048, "bf16"), (5, 16, 1001, "f32")])
+def test_loss_next_epoch_reuses_the_row_order(P, B, T, V, dtype):
+    """Later PPO epochs of a batch (4 per batch in the paper's table) call the loss again on new logits with the same
+    mask: ppo_loss_fwd_bwd_next_epoch skips the prologue launch and must give the bits of the full call - after a
+    loss call, after another next-epoch call and after ppo_step. Told to reuse an order that was built from another
+    mask tensor, or that a fused LM-head call has overwritten, it must write nothing and raise PPO_DEV_BAD_REUSE."""
+    import dataclasses
+    from paper_2403_17031_b200 import binding
+    from paper_2403_17031_b200.pipeline import PPOHotPath
+    from paper_2403_17031_b200.synthetic import CONFIGS, make_batch
+    cfg = dataclasses.replace(CONFIGS[0], B=B, T=T, V=V, dtype=dtype, n_no_eos_exact=None)
+    batch = make_batch(cfg, "cuda")
+    pp = _params(P, cfg.hyper)
+    names = ("losses", "dlogits", "dvalues", "new_logprob", "new_entropy", "dlogprob")
+    g = torch.Generator(device="cuda").manual_seed(5)
+    epochs = []
+    for e in range(3):      # logits and stored log-probs of three epochs
+        lg = (batch["policy_logits"].float() + 0.05 * e * torch.randn(batch["policy_logits"].shape, generator=g,
+                                                                      device="cuda")).to(batch["policy_logits"].dtype)
+        epochs.append(lg)
+    a = PPOHotPath(B, T, V, cfg.torch_dtype, pp)
+    o = a.rollout_stats(batch["policy_logits"], batch["ref_logits"], batch["responses"], batch["scores"], batch["values"])
+    old = (o["logprob"] + batch["old_logprob_noise"]).contiguous()
+    want = []
+    for lg in epochs:       # the full call, every epoch
+        a.loss(lg, batch["responses"], old, batch["values_new"], batch["values"])
+        torch.cuda.synchronize()
+        want.append({k: a.out[k].clone() for k in names})
+    b = PPOHotPath(B, T, V, cfg.torch_dtype, pp)
+    b.rollout_stats(batch["policy_logits"], batch["ref_logits"], batch["responses"], batch["scores"], batch["values"])
+    for e, lg in enumerate(epochs):
+        for k in names:
+            b.out[k].fill_(7)
+        b.loss(lg, batch["responses"], old, batch["values_new"], batch["values"], next_epoch=e > 0)
+        torch.cuda.synchronize()
+        for k in names:
+            assert torch.equal(b.out[k], want[e][k]), (k, "after loss", e)
+    # after the single-call step
+    c = PPOHotPath(B, T, V, cfg.torch_dtype, pp)
+    c.step(batch["policy_logits"], batch["ref_logits"], batch["responses"], batch["scores"], batch["values"],
+           batch["values_new"], old_logprob=old)
+    c.loss(epochs[1], batch["responses"], old, batch["values_new"], batch["values"], next_epoch=True)
+    torch.cuda.synchronize()
+    for k in names:
+        assert torch.equal(c.out[k], want[1][k]), (k, "after step")
+    assert b.device_status() == 0 and c.device_status() == 0
+    if V % 8:
+        return              # (the kernels of this shape run the prologue themselves: nothing to refuse)
+    # an order built from another mask tensor is refused, nothing is written
+    other = c.out["mask"].clone()
+    for k in names:
+        c.out[k].fill_(7)
+    binding.loss_fwd_bwd(epochs[2], batch["responses"], other, old, c.out["advantages_whitened"], batch["values_new"],
+                         batch["values"], c.out["returns"], pp, c.workspace, out=c._loss_out, next_epoch=True)
+    torch.cuda.synchronize()
+    assert c.device_status() == 16
+    for k in names:
+        assert bool((c.out[k] == 7).all()), k
+    # ... and so is one that a fused LM-head call on the same workspace has overwritten
+    M, K = 256, 64
+    ws = P.new_workspace(max(P.lmhead_workspace_bytes(M, K, 512), P.workspace_bytes(B, T, V)))
+    d = PPOHotPath(B, T, V, cfg.torch_dtype, pp)
+    d.workspace = ws
+    d.step(batch["policy_logits"], batch["ref_logits"], batch["responses"], batch["scores"], batch["values"],
+           batch["values_new"], old_logprob=old)
+    P.lmhead_logprob_entropy(torch.randn((M, K), device="cuda").to(torch.bfloat16),
+                             torch.randn((K, 512), device="cuda").to(torch.bfloat16),
+                             torch.zeros(M, dtype=torch.int32, device="cuda"), 0.7, ws)
+    d.loss(epochs[1], batch["responses"], old, batch["values_new"], batch["values"], next_epoch=True)
+    torch.cuda.synchronize()
+    assert d.device_status() == 16
