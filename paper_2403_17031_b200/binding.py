@@ -17,7 +17,7 @@ PPO_F32, PPO_BF16 = 0, 1
 OPT_LOSS_ROW_CACHE = 1
 OPT_ROW_ENGINE = 2
 LOSS_NAMES = ("pg_loss", "vf_loss", "loss", "approx_kl", "pg_clipfrac", "vf_clipfrac", "entropy", "n")
-DEV_BAD_TOKEN, DEV_EMPTY_MASK, DEV_TIMEOUT = 1, 2, 4
+DEV_BAD_TOKEN, DEV_EMPTY_MASK, DEV_TIMEOUT, DEV_BAD_ROW, DEV_BAD_REUSE = 1, 2, 4, 8, 16
 
 _ERR = {-1: "PPO_ERR_NULL", -2: "PPO_ERR_SHAPE", -3: "PPO_ERR_PARAM", -4: "PPO_ERR_ALIGN", -5: "PPO_ERR_DTYPE",
         -6: "PPO_ERR_UNSUPPORTED"}
