@@ -134,3 +134,36 @@ def test_lmhead_mask_takes_rows_out_of_the_gemm(P, oracle, M, K, V, pattern):
         assert_abs(npy(got[0])[sel], rlp, TOL_LOGPROB, "logprob")
         assert_abs(npy(got[1])[sel], rent, TOL_LOGPROB, "entropy")
         assert_abs(npy(got[2])[sel], rlse, TOL_LOGPROB, "lse")
+
+
+def test_lmhead_config4_full_size_with_the_eos_trick_mask(P, oracle):
+    """Config 4 as the benchmark runs it: the call is given the mask of the EOS trick and multiplies the real rows
+    only. Real rows: bits of the call without a mask, and a sample of them against the oracle; padding rows: 0."""
+    from paper_2403_17031_b200.synthetic import CONFIGS, make_lmhead_batch
+    cfg = CONFIGS[4]
+    h = cfg.hyper
+    b = make_lmhead_batch(cfg, "cuda")
+    M, K = b["H"].shape
+    V = b["W"].shape[1]
+    _, _, _, mask, _ = P.truncate_and_score(b["responses"], b["scores"], h.eos_id, h.pad_id, h.no_eos_score)
+    mask = mask.reshape(-1)
+    tok = b["responses"].reshape(-1)
+    ws = P.new_workspace(P.lmhead_workspace_bytes(M, K, V))
+    dense = [t.clone() for t in P.lmhead_logprob_entropy(b["H"], b["W"], tok, h.temperature, ws)]
+    got = P.lmhead_logprob_entropy(b["H"], b["W"], tok, h.temperature, ws, mask=mask)
+    torch.cuda.synchronize()
+    assert P.last_device_status(ws) == 0
+    m = mask.bool()
+    assert 0.3 * M < int(m.sum()) < 0.8 * M
+    for a, d, name in zip(got, dense, ("logprob", "entropy", "lse")):
+        assert torch.equal(a[m], d[m]), name
+        assert not a[~m].any(), name
+    rng = np.random.default_rng(6)
+    real = np.flatnonzero(npy(mask))
+    sel = np.sort(rng.choice(real, 24, replace=False)).astype(np.int64)
+    sel[0], sel[-1] = real[0], real[-1]
+    rlp, rent, rlse = oracle.lmhead_logprob_entropy(host_logits(b["H"]), host_logits(b["W"]), npy(tok),
+                                                    np.float32(h.temperature), sel_rows=sel)
+    assert_abs(npy(got[0])[sel], rlp, TOL_LOGPROB, "logprob (sampled)")
+    assert_abs(npy(got[1])[sel], rent, TOL_LOGPROB, "entropy (sampled)")
+    assert_abs(npy(got[2])[sel], rlse, TOL_LOGPROB, "lse (sampled)")
