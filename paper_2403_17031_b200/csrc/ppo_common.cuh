@@ -26,7 +26,8 @@ struct WorkspaceHeader {
     int order_ready;   // n_tokens + 1 once token count, counters and row order of the loss call in flight are written
     int adv_ready;     // 1 once the advantages / returns that the loss call reads are written
     int step_blocks2;  // second ticket of ppo_step's token-level kernel (resets itself)
-    int reserved[9];
+    int masked_tail;   // work counter of the masked rows kept back for blocks that run out of real rows (reset by every loss call)
+    int reserved[8];
     // what the row order in this workspace was built from: mask pointer, number of rows, order pointer. A loss call
     // that reuses the order (ppo_loss_fwd_bwd_next_epoch) checks its own arguments against these.
     unsigned long long order_sig[3];

@@ -32,6 +32,16 @@ namespace ppo {
 // CONS + 64 threads per block (+ one producer warp + one filler warp); two packs per consumer thread
 // and chunk, i.e. chunks of CONS * 32 bytes (16 KB / 30 KB).
 constexpr int kZeroBytes = 4096;                    // shared zeros, source of the bulk zero-fill stores
+// A loss call that starts with nothing to wait for (a later PPO epoch: order and advantages are already there) keeps
+// this many masked rows per block (at most half of them) away from the filler threads. They are zero-filled by the
+// consumer warps of blocks that have run out of real rows, so the last row time of the kernel, in which fewer and fewer
+// blocks still hold a real row, is filled with finely divisible work (3.4% at B = 64, T = 53; nothing at large batches,
+// where the amount is a small part of the masked rows). A call that overlaps its producer kernel keeps nothing back:
+// there the fillers use the time in which the consumers still wait for the advantages.
+#ifndef PPO_REUSE_RESERVE_ROWS
+#define PPO_REUSE_RESERVE_ROWS 3
+#endif
+constexpr int kReuseReserveRows = PPO_REUSE_RESERVE_ROWS;
 constexpr int kMaxChunks = 14;                      // barriers provided per block
 constexpr size_t kMaxRowBytes = 224 * 1024;         // the largest row one block can hold
 constexpr uint32_t kWaitTries = 1u << 20;           // x ~1 us per try
@@ -283,7 +293,15 @@ struct EngineArgs {
     float vf_coef;
     int wait_flags;         // the launch overlaps the kernel that produces order / advantages: poll the header's flags
     int reuse;              // no prologue ran for this call: the order in the workspace must be the one of this mask
+    int fill_reserve_rows;  // masked rows per block that the filler threads leave to the consumers' zero-fill phase
 };
+
+// number of masked rows that the filler threads may take
+__device__ __forceinline__ int64_t filler_share(int64_t n_masked, int reserve_rows)
+{
+    const int64_t keep = (int64_t)reserve_rows * gridDim.x;
+    return n_masked - (keep < n_masked / 2 ? keep : n_masked / 2);
+}
 
 template <int CONS>
 __device__ __forceinline__ void block_sync_all() { asm volatile("bar.sync 2, %0;" ::"r"(CONS + 64) : "memory"); }
@@ -309,6 +327,7 @@ __device__ __forceinline__ void engine_epilogue(const EngineArgs &a, EngineSmem 
     // every block is past the work counters: leave them ready for a call that reuses this order
     if (threadIdx.x == 0) {
         a.hdr->masked_next = 0;
+        a.hdr->masked_tail = 0;
         a.hdr->real_next = 0;
         a.hdr->done_blocks = 0;
     }
@@ -404,9 +423,10 @@ row_engine_kernel(const EngineArgs a)
         const LossArgs &la = a.loss;
         const int64_t n_masked = la.rows - n_items;
         const size_t row_bytes = (size_t)V * sizeof(T);
+        const int64_t n_fill = filler_share(n_masked, a.fill_reserve_rows);
         for (;;) {
             const int64_t j = atomicAdd(&a.hdr->masked_next, 1);
-            if (j >= n_masked) break;
+            if (j >= n_fill) break;
             const int64_t row = a.order[la.rows - 1 - j];
             unsigned char *dst = reinterpret_cast<unsigned char *>(reinterpret_cast<T *>(la.dlogits) + row * (int64_t)V);
             for (size_t off = 0; off < row_bytes; off += kZeroBytes) {
@@ -710,12 +730,24 @@ row_engine_kernel(const EngineArgs a)
         const LossArgs &la = a.loss;
         const int64_t n_masked = a.loss.rows - n_items;
         const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+        // masked item j is row order[rows - 1 - j]: the fillers draw j in [0, n_fill) from masked_next, the rows kept
+        // back are j in [n_fill, n_masked) and are drawn from masked_tail; once those are gone the consumers help
+        // with whatever the fillers have left
+        const int64_t n_fill = filler_share(n_masked, a.fill_reserve_rows);
+        bool tail = n_fill < n_masked;
         for (;;) {
             consumer_sync<CONS>();
-            if (ct == 0) sm.next_item = atomicAdd(&a.hdr->masked_next, 1);
+            if (ct == 0)
+                sm.next_item = tail ? (int)n_fill + atomicAdd(&a.hdr->masked_tail, 1) : atomicAdd(&a.hdr->masked_next, 1);
             consumer_sync<CONS>();
             const int64_t j = sm.next_item;
-            if (j >= n_masked) break;
+            if (tail) {
+                if (j >= n_masked) {
+                    tail = false;
+                    continue;
+                }
+            } else if (j >= n_fill)
+                break;
             const int64_t row = a.order[a.loss.rows - 1 - j];
             uint4 *dst4 = reinterpret_cast<uint4 *>(reinterpret_cast<T *>(la.dlogits) + row * (int64_t)V);
             for (int i = ct; i < nvec; i += kConsumers) st_stream(dst4 + i, z);
@@ -825,6 +857,7 @@ int launch_loss_bulk(const LossArgs &la, int dtype, void *workspace, float *loss
     a.vf_coef = vf_coef;
     a.wait_flags = dependent ? 1 : 0;
     a.reuse = reuse ? 1 : 0;
+    a.fill_reserve_rows = reuse ? kReuseReserveRows : 0;
     if (dtype == PPO_F32) {
         if (!bulk_ok<float>(la.logits, la.V, la.V)) return PPO_ERR_UNSUPPORTED;
         return launch_engine<float, 1, true>(a, la.rows, dependent, s);

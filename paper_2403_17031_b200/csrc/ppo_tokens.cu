@@ -222,6 +222,7 @@ __device__ __forceinline__ void loss_prepare_block(const uint8_t *mask, int64_t 
         if (lane == 31) {
             hdr->n_tokens = wi;
             hdr->masked_next = 0;
+            hdr->masked_tail = 0;
             hdr->real_next = 0;
             hdr->done_blocks = 0;
             hdr->order_sig[0] = (unsigned long long)reinterpret_cast<uintptr_t>(mask);
