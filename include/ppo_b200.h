@@ -423,7 +423,11 @@ int ppo_lmhead_bwd(const void *H, const void *W, int64_t M, int64_t K, int64_t V
  * positions up to its first EOS, found from host->responses; the other rows of the staging buffers
  * are left as they are), runs ppo_step on `dev`, copies back each output whose pointer in
  * `host` is not NULL, and waits for the stream.  Inputs that are NULL in `host` (loss_logits,
- * old_logprob) are treated as in ppo_step.
+ * old_logprob) are treated as in ppo_step.  The copies of the reference tensor are queued on a
+ * side stream of the library (one per device, created by the first call on that device and kept
+ * until the process exits) that is ordered after the work already in `stream` and before the
+ * kernels of this call, so that two copy queues keep the host link busy; the call is safe from
+ * several host threads.
  */
 typedef struct ppo_step_io {
     const void *policy_logits, *ref_logits, *loss_logits;

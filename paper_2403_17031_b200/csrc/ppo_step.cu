@@ -2,6 +2,8 @@
 // steps (the token-level ones fused into one launch that overlaps its neighbours) plus the host<->device copies.
 #include "ppo_common.cuh"
 
+#include <mutex>
+
 using namespace ppo;
 
 extern "C" int ppo_step(const ppo_step_io *io, int dtype, int32_t B, int32_t T, int64_t V, const ppo_params *p,
@@ -66,21 +68,60 @@ int copy_in(void *dst, const void *src, size_t bytes, cudaStream_t s)
 
 // A [B, T, V] logits tensor: only the rows that ppo_step reads are copied - of each response the positions up to
 // and including its first EOS (the EOS trick masks the rest out of every step; found here from the host's tokens).
+// A response without EOS ends where the next one starts, so the two go out as one copy.
 int copy_in_real_rows(void *dst, const void *src, const int32_t *responses, int32_t B, int32_t T, size_t row_bytes,
                       int32_t eos_id, cudaStream_t s)
 {
     if (!src) return PPO_OK;
     if (!dst) return PPO_ERR_NULL;
+    size_t run_off = 0, run_bytes = 0;   // copy being collected
     for (int32_t b = 0; b < B; ++b) {
         const int32_t *r = responses + (size_t)b * T;
         int32_t L = T;
         for (int32_t t = 0; t < T; ++t)
             if (r[t] == eos_id) { L = t + 1; break; }
         const size_t off = (size_t)b * T * row_bytes;
-        PPO_RETURN_IF_CUDA(cudaMemcpyAsync(static_cast<unsigned char *>(dst) + off,
-                                           static_cast<const unsigned char *>(src) + off, (size_t)L * row_bytes,
-                                           cudaMemcpyHostToDevice, s));
+        if (run_bytes && run_off + run_bytes != off) {
+            PPO_RETURN_IF_CUDA(cudaMemcpyAsync(static_cast<unsigned char *>(dst) + run_off,
+                                               static_cast<const unsigned char *>(src) + run_off, run_bytes,
+                                               cudaMemcpyHostToDevice, s));
+            run_bytes = 0;
+        }
+        if (!run_bytes) run_off = off;
+        run_bytes += (size_t)L * row_bytes;
     }
+    if (run_bytes)
+        PPO_RETURN_IF_CUDA(cudaMemcpyAsync(static_cast<unsigned char *>(dst) + run_off,
+                                           static_cast<const unsigned char *>(src) + run_off, run_bytes,
+                                           cudaMemcpyHostToDevice, s));
+    return PPO_OK;
+}
+
+// Second copy queue of ppo_step_host. One queue leaves the link idle between two copies (about 4 us per copy, 8% of
+// the transfer time at 128 copies of 2.5 MB); with the policy tensor on the caller's stream and the reference tensor
+// on a side stream the gaps of one queue are filled by the other. One side stream and two events per device, created
+// on the first call on that device and kept until the process exits.
+struct CopyLane {
+    cudaStream_t side = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
+};
+std::mutex g_lane_mutex;   // held while a call enqueues its fork / join, so that two host threads cannot interleave them
+
+int copy_lane(CopyLane **out)
+{
+    static CopyLane lanes[64];
+    int dev = 0;
+    PPO_RETURN_IF_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return PPO_ERR_UNSUPPORTED;
+    CopyLane &l = lanes[dev];
+    if (!l.side) {
+        cudaStream_t st = nullptr;
+        PPO_RETURN_IF_CUDA(cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking));
+        PPO_RETURN_IF_CUDA(cudaEventCreateWithFlags(&l.fork, cudaEventDisableTiming));
+        PPO_RETURN_IF_CUDA(cudaEventCreateWithFlags(&l.join, cudaEventDisableTiming));
+        l.side = st;
+    }
+    *out = &l;
     return PPO_OK;
 }
 
@@ -113,12 +154,24 @@ extern "C" int ppo_step_host(const ppo_step_io *host, const ppo_step_io *dev, in
     const size_t bt = (size_t)B * (size_t)T, es = dtype == PPO_F32 ? 4 : 2;
     const size_t logits_bytes = bt * (size_t)V * es;
     // device staging buffers are written here, so drop the const the struct carries for inputs
-    PPO_TRY(copy_in_real_rows(const_cast<void *>(dev->policy_logits), host->policy_logits, host->responses, B, T,
-                              (size_t)V * es, p->eos_id, s));
-    PPO_TRY(copy_in_real_rows(const_cast<void *>(dev->ref_logits), host->ref_logits, host->responses, B, T,
-                              (size_t)V * es, p->eos_id, s));
-    PPO_TRY(copy_in_real_rows(const_cast<void *>(dev->loss_logits), host->loss_logits, host->responses, B, T,
-                              (size_t)V * es, p->eos_id, s));
+    {
+        // the reference tensor goes through the side queue, everything else through the caller's stream; the side
+        // queue starts after the work already in the stream (which may still read the staging buffers) and the
+        // stream continues after the side queue's last copy
+        std::lock_guard<std::mutex> guard(g_lane_mutex);
+        CopyLane *lane = nullptr;
+        PPO_TRY(copy_lane(&lane));
+        PPO_RETURN_IF_CUDA(cudaEventRecord(lane->fork, s));
+        PPO_RETURN_IF_CUDA(cudaStreamWaitEvent(lane->side, lane->fork, 0));
+        PPO_TRY(copy_in_real_rows(const_cast<void *>(dev->ref_logits), host->ref_logits, host->responses, B, T,
+                                  (size_t)V * es, p->eos_id, lane->side));
+        PPO_RETURN_IF_CUDA(cudaEventRecord(lane->join, lane->side));
+        PPO_TRY(copy_in_real_rows(const_cast<void *>(dev->policy_logits), host->policy_logits, host->responses, B, T,
+                                  (size_t)V * es, p->eos_id, s));
+        PPO_TRY(copy_in_real_rows(const_cast<void *>(dev->loss_logits), host->loss_logits, host->responses, B, T,
+                                  (size_t)V * es, p->eos_id, s));
+        PPO_RETURN_IF_CUDA(cudaStreamWaitEvent(s, lane->join, 0));
+    }
     PPO_TRY(copy_in(const_cast<int32_t *>(dev->responses), host->responses, bt * 4, s));
     PPO_TRY(copy_in(const_cast<float *>(dev->scores), host->scores, (size_t)B * 4, s));
     PPO_TRY(copy_in(const_cast<float *>(dev->values), host->values, bt * 4, s));
