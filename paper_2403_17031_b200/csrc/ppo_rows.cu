@@ -458,7 +458,7 @@ int ppo::loss_fwd_bwd_prepared(const void *logits, int dtype, int32_t B, int32_t
     a.c1 = p->vf_coef;
     rc = PPO_ERR_UNSUPPORTED;
     if (option_value(PPO_OPT_ROW_ENGINE) != 1) {
-        rc = launch_loss_bulk(a, dtype, workspace, losses, p->vf_coef, !reuse, s, reuse);
+        rc = launch_loss_bulk(a, dtype, workspace, losses, p->vf_coef, !reuse, s, reuse, !prepared);
         if (rc != PPO_ERR_UNSUPPORTED) return rc;      // the engine reduces the partials itself
     }
     if (reuse) {

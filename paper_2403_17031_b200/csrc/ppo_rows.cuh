@@ -254,7 +254,9 @@ int launch_logprob_bulk(const void *logits, int dtype, int64_t rows, int V, int6
 // waits for the workspace header's flags before it reads that kernel's results)
 // `reuse`: no prologue ran for this call; the kernel checks that the order in the workspace was built from this
 // call's mask (PPO_DEV_BAD_REUSE and nothing written otherwise)
+// `keep_back`: leave a few masked rows per block to the blocks that run out of real rows (calls that do not overlap
+// a long producer kernel)
 int launch_loss_bulk(const LossArgs &a, int dtype, void *workspace, float *losses, float vf_coef, bool dependent,
-                     cudaStream_t s, bool reuse = false);
+                     cudaStream_t s, bool reuse = false, bool keep_back = false);
 
 }   // namespace ppo

@@ -32,12 +32,12 @@ namespace ppo {
 // CONS + 64 threads per block (+ one producer warp + one filler warp); two packs per consumer thread
 // and chunk, i.e. chunks of CONS * 32 bytes (16 KB / 30 KB).
 constexpr int kZeroBytes = 4096;                    // shared zeros, source of the bulk zero-fill stores
-// A loss call that starts with nothing to wait for (a later PPO epoch: order and advantages are already there) keeps
+// A stand-alone loss call (its advantages are there from the start; a later PPO epoch finds the row order too) keeps
 // this many masked rows per block (at most half of them) away from the filler threads. They are zero-filled by the
 // consumer warps of blocks that have run out of real rows, so the last row time of the kernel, in which fewer and fewer
 // blocks still hold a real row, is filled with finely divisible work (3.4% at B = 64, T = 53; nothing at large batches,
-// where the amount is a small part of the masked rows). A call that overlaps its producer kernel keeps nothing back:
-// there the fillers use the time in which the consumers still wait for the advantages.
+// where the amount is a small part of the masked rows). The call inside ppo_step, which overlaps the kernels that
+// produce its advantages, keeps nothing back: there the fillers use the time in which the consumers still wait.
 #ifndef PPO_REUSE_RESERVE_ROWS
 #define PPO_REUSE_RESERVE_ROWS 3
 #endif
@@ -838,7 +838,7 @@ int launch_logprob_bulk(const void *logits, int dtype, int64_t rows, int V, int6
 }
 
 int launch_loss_bulk(const LossArgs &la, int dtype, void *workspace, float *losses, float vf_coef, bool dependent,
-                     cudaStream_t s, bool reuse)
+                     cudaStream_t s, bool reuse, bool keep_back)
 {
     if (!la.dlogits || !aligned16(la.dlogits)) return PPO_ERR_UNSUPPORTED;
     EngineArgs a = {};
@@ -857,7 +857,7 @@ int launch_loss_bulk(const LossArgs &la, int dtype, void *workspace, float *loss
     a.vf_coef = vf_coef;
     a.wait_flags = dependent ? 1 : 0;
     a.reuse = reuse ? 1 : 0;
-    a.fill_reserve_rows = reuse ? kReuseReserveRows : 0;
+    a.fill_reserve_rows = keep_back ? kReuseReserveRows : 0;
     if (dtype == PPO_F32) {
         if (!bulk_ok<float>(la.logits, la.V, la.V)) return PPO_ERR_UNSUPPORTED;
         return launch_engine<float, 1, true>(a, la.rows, dependent, s);
