@@ -33,7 +33,7 @@ import torch  # noqa: E402
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the committed ncu capture of the same
 # configuration (profiles/loss_fwd_bwd_row_engine_config1.md, profiles/dpo_step_config5.md); None where no capture
 # of the current kernel exists.
-NCU_TRAFFIC_BYTES = {1: 160.003e6 + 282.884e6, 5: 109.9e6 + 965.3e6}
+NCU_TRAFFIC_BYTES = {1: 160.007e6 + 283.877e6, 5: 109.9e6 + 965.3e6}
 LAUNCHES_PER_STEP = 3   # ppo_step: logprob pair (policy + reference), rollout (token-level steps + loss prologue), row_engine (loss)
 
 
