@@ -174,6 +174,21 @@ int ppo_kl_rewards(const float *logprob, const float *ref_logprob, const uint8_t
                    float kl_coef, float *kl, float *rewards, void *stream);
 
 /*
+ * The three curves of the paper's figure of PPO learning curves, from the outputs of steps 2 and 3:
+ *     out3[0] = mean over b of R_b,  R_b = scores[b] - kl_coef * sum_t kl[b,t]   (Eq. "RL" with the
+ *               KL of a response estimated by its summed per-token k1 terms)
+ *     out3[1] = mean over b of sum_t kl[b,t]   ("the mean of the sum of per-token KL divergence
+ *               between the RL and SFT policies")
+ *     out3[2] = mean over b of scores[b]       (pass step 2's scores_out for what PPO optimises)
+ * kl [B,T] f32 (step 3), scores [B] f32, out3 [3] f32, all device.  mask [B,T] u8 is nullable: with
+ * it, positions with mask 0 are left out of the sums; without it every position counts (step 3
+ * already writes 0 behind the responses).  Means are over the B responses.  One block, fp64 sums in
+ * a fixed order.  B, T >= 1; errors: PPO_ERR_SHAPE, PPO_ERR_NULL, PPO_ERR_PARAM (kl_coef not finite).
+ */
+int ppo_rollout_curves(const float *kl, const uint8_t *mask, const float *scores, int32_t B, int32_t T,
+                       float kl_coef, float *out3, void *stream);
+
+/*
  * Step 4, GAE with the table's gamma and lambda.  The episode ends after the last real token
  * (the value function predicts the end-of-episode return, section "Value model initializes
  * from the reward model"), so nothing is bootstrapped beyond seq_len-1:

@@ -4,9 +4,9 @@ fails loudly if it is missing (there is no CPU or PyTorch fallback)."""
 from .binding import (PPOParams, PPOStepIO, step, step_host, default_params, gae, kl_rewards, last_device_status, lib, lmhead_logprob_entropy,
                       lmhead_workspace_bytes, logprob_entropy, loss_from_logprob, loss_from_logprob_static, loss_fwd_bwd, new_workspace,
                       set_option, truncate_and_score, version, whiten, workspace_bytes, PPOError, LOSS_NAMES,
-                      logprob_bwd, pairwise_loss, dpo_loss, lmhead_bwd, sample_logprob_entropy, logprob_entropy_pair)
+                      logprob_bwd, pairwise_loss, dpo_loss, lmhead_bwd, sample_logprob_entropy, logprob_entropy_pair, rollout_curves)
 
 __all__ = ["PPOParams", "PPOStepIO", "step", "step_host", "default_params", "gae", "kl_rewards", "last_device_status", "lib",
            "lmhead_logprob_entropy", "lmhead_workspace_bytes", "logprob_entropy", "loss_from_logprob", "loss_from_logprob_static",
            "loss_fwd_bwd", "new_workspace", "set_option", "truncate_and_score", "version", "whiten",
-           "workspace_bytes", "PPOError", "LOSS_NAMES", "logprob_bwd", "pairwise_loss", "dpo_loss", "lmhead_bwd", "sample_logprob_entropy", "logprob_entropy_pair"]
+           "workspace_bytes", "PPOError", "LOSS_NAMES", "logprob_bwd", "pairwise_loss", "dpo_loss", "lmhead_bwd", "sample_logprob_entropy", "logprob_entropy_pair", "rollout_curves"]

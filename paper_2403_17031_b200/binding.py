@@ -77,6 +77,8 @@ _SIGS = {
                                          C.c_void_p]),
     "ppo_kl_rewards": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                  C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "ppo_rollout_curves": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float, C.c_void_p,
+                                     C.c_void_p]),
     "ppo_gae": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float, C.c_float,
                           C.c_void_p, C.c_void_p, C.c_void_p]),
     "ppo_whiten": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_float, C.c_void_p, C.c_void_p,
@@ -272,6 +274,17 @@ def kl_rewards(logprob, ref_logprob, mask, seq_len, scores, kl_coef: float, out=
                               _ptr(mask, torch.uint8), _ptr(seq_len, torch.int32), _ptr(scores, torch.float32),
                               B, T, float(kl_coef), _ptr(kl, torch.float32), _ptr(rew, torch.float32), _stream())
     _check("ppo_kl_rewards", rc)
+    return out
+
+
+def rollout_curves(kl, mask, scores, kl_coef: float, out=None):
+    """Mean RLHF reward, mean summed per-token KL, mean score of a batch; returns a [3] f32 tensor."""
+    B, T = kl.shape
+    if out is None:
+        out = torch.empty(3, dtype=torch.float32, device=kl.device)
+    rc = lib().ppo_rollout_curves(_ptr(kl, torch.float32), None if mask is None else _ptr(mask, torch.uint8),
+                                  _ptr(scores, torch.float32), B, T, float(kl_coef), _ptr(out, torch.float32), _stream())
+    _check("ppo_rollout_curves", rc)
     return out
 
 
