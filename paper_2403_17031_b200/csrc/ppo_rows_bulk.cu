@@ -13,8 +13,8 @@
 //     the space, one chunk behind, with the next row. Rows whose mask is 0 are only zero-filled: a
 //     filler thread per block takes them from a shared work counter and writes them with bulk
 //     shared->global copies of a small block of zeros while the consumers work on real rows (the
-//     real-row phase alone leaves HBM bandwidth idle); consumers that run out of real rows join in a
-//     stand-alone call keeps a few masked rows per block back for them, so that the end of the kernel stays busy;
+//     real-row phase alone leaves HBM bandwidth idle); consumers that run out of real rows join in (a
+//     stand-alone call keeps a few masked rows per block back for them, so that the end of the kernel stays busy);
 //   * step 6 hands its rows out dynamically (a counter in the workspace header; the row index reaches
 //     the consumers through a small ring in shared memory), since SMs do not stream at equal speed;
 //   * two blocks per SM while a row is <= 110 KB (bf16, V = 50304), one otherwise;
