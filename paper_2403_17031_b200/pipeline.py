@@ -104,6 +104,12 @@ class PPOHotPath:
         t["workspace"] = self.workspace
         return _b.PPOStepIO.from_tensors(t, cuda)
 
+    def curves(self):
+        """The three statistics the paper plots per PPO update, from the outputs of the last rollout_stats() / step():
+        [mean RLHF reward, mean summed per-token KL, mean score] as a [3] f32 tensor (one small launch)."""
+        o = self.out
+        return _b.rollout_curves(o["kl"], o["mask"], o["scores_out"], self.params.kl_coef)
+
     def device_status(self) -> int:
         return _b.last_device_status(self.workspace)
 

@@ -83,3 +83,23 @@ def test_curves_argument_errors(P):
     L = binding.lib()
     assert L.ppo_rollout_curves(None, None, s.data_ptr(), 2, 3, 0.05, s.data_ptr(), None) == -1
     assert L.ppo_rollout_curves(kl.data_ptr(), None, s.data_ptr(), 0, 3, 0.05, s.data_ptr(), None) == -2
+
+
+def test_curves_after_the_single_call_step(P):
+    """PPOHotPath.curves() after ppo_step on a small TL;DR-shaped batch equals the oracle on the step's own outputs."""
+    import dataclasses
+    from oracle import curves_oracle as Q
+    from paper_2403_17031_b200 import binding
+    from paper_2403_17031_b200.pipeline import PPOHotPath
+    from paper_2403_17031_b200.synthetic import CONFIGS, make_batch
+    cfg = dataclasses.replace(CONFIGS[1], B=16, V=2048)
+    batch = make_batch(cfg, "cuda")
+    hp = PPOHotPath(cfg.B, cfg.T, cfg.V, cfg.torch_dtype, binding.params_from(cfg.hyper))
+    o = hp.step(batch["policy_logits"], batch["ref_logits"], batch["responses"], batch["scores"], batch["values"],
+                batch["values_new"])
+    got = hp.curves().double().cpu().numpy()
+    want = Q.rollout_curves(o["kl"].cpu().numpy(), o["mask"].cpu().numpy(), o["scores_out"].cpu().numpy(),
+                            cfg.hyper.kl_coef)
+    for i, k in enumerate(("rlhf_reward", "kl", "score")):
+        assert abs(got[i] - want[k]) <= TOL_ABS, k
+    assert abs(got[0] - float(o["rewards"].double().sum(dim=1).mean())) <= TOL_ABS
