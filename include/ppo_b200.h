@@ -177,8 +177,8 @@ int ppo_kl_rewards(const float *logprob, const float *ref_logprob, const uint8_t
  * The three curves of the paper's figure of PPO learning curves, from the outputs of steps 2 and 3:
  *     out3[0] = mean over b of R_b,  R_b = scores[b] - kl_coef * sum_t kl[b,t]   (Eq. "RL" with the
  *               KL of a response estimated by its summed per-token k1 terms)
- *     out3[1] = mean over b of sum_t kl[b,t]   ("the mean of the sum of per-token KL divergence
- *               between the RL and SFT policies")
+ *     out3[1] = mean over b of sum_t kl[b,t]   (the figure's KL curve: per-token KL terms between RL
+ *               and SFT policy summed per response, then averaged over the responses)
  *     out3[2] = mean over b of scores[b]       (pass step 2's scores_out for what PPO optimises)
  * kl [B,T] f32 (step 3), scores [B] f32, out3 [3] f32, all device.  mask [B,T] u8 is nullable: with
  * it, positions with mask 0 are left out of the sums; without it every position counts (step 3

@@ -8,8 +8,9 @@ The caption of the paper's figure of PPO learning curves names them:
                 R = r(x, y) - beta * KL, with the KL of one response estimated by the sum over its
                 real tokens of the per-token k1 terms (log pi - log pi_SFT at the sampled token),
                 averaged over the responses of the batch
-  kl            "the mean of the sum of per-token KL divergence between the RL and SFT policies":
-                the same sum, averaged over the responses
+  kl            per response, the per-token KL terms between the RL policy and the SFT policy are
+                summed; the curve is the mean of those sums over the responses (caption of the figure
+                of PPO learning curves)
   score         the scores obtained from the reward model, averaged over the responses (here the
                 score array that is passed in; the PPO loop passes the scores after the EOS trick)
 Plain definitions: one loop over responses, one over tokens.

@@ -62,5 +62,27 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB_PATH
 
 
+def build_variant(out_path: str, defines, only=None) -> str:
+    """A second copy of the library compiled with extra -D macros (tests of the bounded waits use one in which the
+    hand-over flags are withheld). `only`: basenames of the sources to compile; objects go next to `out_path`."""
+    obj_dir = out_path + ".obj"
+    os.makedirs(obj_dir, exist_ok=True)
+    srcs = [s for s in sources() if only is None or os.path.basename(s) in only]
+    procs, objs = [], []
+    for src in srcs:
+        obj = os.path.join(obj_dir, os.path.basename(src)[:-3] + ".o")
+        cmd = [_nvcc(), *NVCC_FLAGS, *["-D" + d for d in defines], "-I", INCLUDE, "-I", CSRC, "-c", src, "-o", obj]
+        procs.append(subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True))
+        objs.append(obj)
+    for p in procs:
+        out, _ = p.communicate()
+        if p.returncode != 0:
+            sys.stderr.write(out)
+            raise RuntimeError("nvcc failed")
+    subprocess.check_call([_nvcc(), "-shared", "-o", out_path, *objs, "-cudart", "static", *ARCH_FLAGS,
+                           "-Xcompiler", "-fPIC"])
+    return out_path
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

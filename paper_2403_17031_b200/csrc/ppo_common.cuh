@@ -345,16 +345,29 @@ __device__ __forceinline__ void reduce_loss_partials(const float *partials, int6
 // while the token-level kernel before it is still running, see launch_dependent): the writer publishes
 // with flag_set after its data, the reader polls with flag_wait before it touches them. The wait is
 // bounded (~1 s); when it runs out the status word gets PPO_DEV_TIMEOUT and the caller carries on.
-__device__ __forceinline__ void flag_set(int *flag, int value = 1 /* non-zero */)
+// PPO_TEST_WITHHOLD_FLAGS (never defined in the product build): a test build in which the flags whose bit is set
+// (1 = order_ready, 2 = adv_ready) are never published, so that the bounded waits of the reader run out.
+#ifndef PPO_TEST_WITHHOLD_FLAGS
+#define PPO_TEST_WITHHOLD_FLAGS 0
+#endif
+enum FlagKind { kFlagOrder = 1, kFlagAdv = 2 };
+
+__device__ __forceinline__ void flag_set(int *flag, int value /* non-zero */, FlagKind kind)
 {
+    if (PPO_TEST_WITHHOLD_FLAGS & kind) return;
     __threadfence();
     asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(flag), "r"(value) : "memory");
 }
 
+#ifndef PPO_WAIT_TRIES
+constexpr uint32_t kFlagWaitTries = 1u << 20;
+#else
+constexpr uint32_t kFlagWaitTries = PPO_WAIT_TRIES;   // a test build makes the waits short
+#endif
 // returns the flag's (non-zero) value, or 0 after the wait ran out
 __device__ __forceinline__ int flag_wait(const int *flag, int *status)
 {
-    for (uint32_t it = 0; it < (1u << 20); ++it) {
+    for (uint32_t it = 0; it < kFlagWaitTries; ++it) {
         int v;
         asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
         if (v) return v;

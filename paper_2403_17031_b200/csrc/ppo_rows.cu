@@ -84,10 +84,18 @@ logprob_pair_kernel(const T *__restrict__ policy_logits, const T *__restrict__ r
                     float *__restrict__ ref_logprob, int *status, int *flags2)
 {
     __shared__ float red[96];
-    // ppo_step: the hand-over flags between the two kernels that follow start at 0 (nothing runs beside this
-    // kernel on the stream, and the next kernel starts after it has ended)
-    if (flags2 && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) { flags2[0] = 0; flags2[1] = 0; }
-    grid_dependents_may_launch();   // the token-level kernel may be scheduled as this grid drains; it waits for its end
+    // ppo_step: the hand-over flags between the two kernels that follow start at 0. The token-level kernel may be
+    // scheduled as soon as every block of this grid has passed the trigger below, and part of it runs before it
+    // waits for this grid's end, so the block that clears the flags makes the stores visible before its trigger.
+    if (flags2 && blockIdx.x == 0 && blockIdx.y == 0) {
+        if (threadIdx.x == 0) {
+            flags2[0] = 0;
+            flags2[1] = 0;
+            __threadfence();
+        }
+        __syncthreads();
+    }
+    grid_dependents_may_launch();   // the token-level kernel may be scheduled as this grid drains
     if (seq_T > 0) {
         const int64_t row = blockIdx.x;
         const int t = (int)(row % seq_T);

@@ -45,7 +45,10 @@ constexpr int kZeroBytes = 4096;                    // shared zeros, source of t
 constexpr int kReuseReserveRows = PPO_REUSE_RESERVE_ROWS;
 constexpr int kMaxChunks = 14;                      // barriers provided per block
 constexpr size_t kMaxRowBytes = 224 * 1024;         // the largest row one block can hold
-constexpr uint32_t kWaitTries = 1u << 20;           // x ~1 us per try
+#ifndef PPO_WAIT_TRIES
+#define PPO_WAIT_TRIES (1u << 20)
+#endif
+constexpr uint32_t kWaitTries = PPO_WAIT_TRIES;     // x ~1 us per try (a test build makes the waits short)
 
 struct EngineSmem {
     unsigned long long full[kMaxChunks];
@@ -410,7 +413,18 @@ row_engine_kernel(const EngineArgs a)
                 sm.abort = 1;
             }
         }
-        sm.n_tokens = a.wait_flags ? max(flag_wait(&a.hdr->order_ready, status) - 1, 0) : a.hdr->n_tokens;
+        if (a.wait_flags) {
+            // a wait that ran out: nobody may have written the row order, so nothing may be indexed through it
+            const int v = flag_wait(&a.hdr->order_ready, status);
+            if (v == 0) {
+                sm.abort = 1;
+                if (blockIdx.x == 0)   // the status word says why; the scalars must not look like a result
+                    for (int q = 0; q < 8; ++q) a.losses[q] = __int_as_float(0x7fc00000);
+            }
+            sm.n_tokens = max(v - 1, 0);
+        } else {
+            sm.n_tokens = a.hdr->n_tokens;
+        }
     }
     __syncthreads();
     if (MODE == 1 && sm.abort) return;   // nothing is read or written through an order that is not this call's
@@ -547,6 +561,10 @@ row_engine_kernel(const EngineArgs a)
                 }
                 asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
             }
+            // The consumers have seen every chunk land, unless one of their waits ran out: make sure (bounded) that
+            // no copy into this block's shared memory is still in flight when the block retires.
+            if (k > 0)
+                for (int c = 0; c < nch; ++c) mbar_wait(&sm.full[c], (k - 1) & 1, status);
         }
         if (MODE == 1) {
             __syncwarp();

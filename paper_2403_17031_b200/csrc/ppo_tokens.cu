@@ -250,7 +250,7 @@ __device__ __forceinline__ void loss_prepare_block(const uint8_t *mask, int64_t 
     if (!publish) return;
     __syncthreads();
     // a loss kernel that is already running may go on; the flag carries the token count (+1) it needs first
-    if (threadIdx.x == 0) flag_set(&hdr->order_ready, *reinterpret_cast<volatile int *>(&hdr->n_tokens) + 1);
+    if (threadIdx.x == 0) flag_set(&hdr->order_ready, *reinterpret_cast<volatile int *>(&hdr->n_tokens) + 1, kFlagOrder);
 }
 
 __global__ void __launch_bounds__(kReduceThreads)
@@ -268,7 +268,7 @@ loss_prepare_kernel(const uint8_t *__restrict__ mask, int64_t rows, WorkspaceHea
     __syncthreads();
     grid_dependents_may_launch();
     loss_prepare_block(mask, rows, hdr, order, warp_tot, true, flag_empty != 0);
-    if (threadIdx.x == 0) flag_set(&hdr->adv_ready);   // stand-alone loss call: its other inputs exist already
+    if (threadIdx.x == 0) flag_set(&hdr->adv_ready, 1, kFlagAdv);   // stand-alone loss call: its other inputs exist already
 }
 
 // ---------------------------------------------------------------- fused launch of ppo_step
@@ -344,7 +344,7 @@ rollout_kernel(const int32_t *responses, int B, int T, int eos_id, int pad_id, c
         __syncthreads();
         whiten_block(advantages, mask, rows, 1, eps, whitened, stats3, &hdr->status, red);
         __syncthreads();
-        if (threadIdx.x == 0) flag_set(&hdr->adv_ready);
+        if (threadIdx.x == 0) flag_set(&hdr->adv_ready, 1, kFlagAdv);
         return;
     }
 
@@ -406,7 +406,7 @@ rollout_kernel(const int32_t *responses, int B, int T, int eos_id, int pad_id, c
     }
     whiten_block(advantages, mask, rows, 1, eps, whitened, stats3, &hdr->status, red);
     __syncthreads();
-    if (threadIdx.x == 0) flag_set(&hdr->adv_ready);
+    if (threadIdx.x == 0) flag_set(&hdr->adv_ready, 1, kFlagAdv);
 }
 
 // Sum the per-token partials (fixed thread assignment, fp64) and write the eight loss scalars.

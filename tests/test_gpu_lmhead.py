@@ -167,3 +167,85 @@ def test_lmhead_config4_full_size_with_the_eos_trick_mask(P, oracle):
     assert_abs(npy(got[0])[sel], rlp, TOL_LOGPROB, "logprob (sampled)")
     assert_abs(npy(got[1])[sel], rent, TOL_LOGPROB, "entropy (sampled)")
     assert_abs(npy(got[2])[sel], rlse, TOL_LOGPROB, "lse (sampled)")
+
+
+def test_config4_chained_path_against_the_oracle(P, oracle):
+    """Config 4 as the benchmark times it, call by call: EOS trick -> fused LM head of policy and reference with the
+    EOS-trick mask -> KL rewards -> GAE -> whitening -> loss at log-prob level. Log-probs and entropy on a row sample
+    (the oracle forms each logits row by fp64 dot products), every [B,T] array of the later steps in full, each fed
+    the GPU's own upstream fp32 values, and the loss through the oracle's own loss arithmetic."""
+    from parity import TOL_REL, assert_rel, f32, near_kink
+    from paper_2403_17031_b200 import binding
+    from paper_2403_17031_b200.synthetic import CONFIGS, make_lmhead_batch
+    cfg = CONFIGS[4]
+    h = cfg.hyper
+    p = binding.params_from(h)
+    b = make_lmhead_batch(cfg, "cuda")
+    M, K = b["H"].shape
+    V = b["W"].shape[1]
+    B, T = b["responses"].shape
+    ws = P.new_workspace(max(P.lmhead_workspace_bytes(M, K, V), P.workspace_bytes(B, T, V)))
+    tok = b["responses"].reshape(-1)
+    ro, ei, sl, mask, so = P.truncate_and_score(b["responses"], b["scores"], h.eos_id, h.pad_id, h.no_eos_score)
+    lp, ent, lse = P.lmhead_logprob_entropy(b["H"], b["W"], tok, h.temperature, ws, mask=mask.view(-1))
+    rlp, _, _ = P.lmhead_logprob_entropy(b["H"], b["W_ref"], tok, h.temperature, ws, mask=mask.view(-1))
+    lp, ent, rlp = lp.view(B, T), ent.view(B, T), rlp.view(B, T)
+    kl, rew = P.kl_rewards(lp, rlp, mask, sl, so, h.kl_coef)
+    adv, ret = P.gae(rew, b["values"], sl, h.gamma, h.lam)
+    aw, st = P.whiten(adv, mask, True, h.whiten_eps, workspace=ws)
+    old = (lp + b["old_logprob_noise"]).contiguous()
+    out = P.loss_from_logprob(lp, ent, mask, old, aw, b["values_new"], b["values"], ret, p, ws)
+    torch.cuda.synchronize()
+    assert P.last_device_status(ws) == 0
+
+    # EOS trick: exact
+    resp = npy(b["responses"])
+    o_ro, o_ei, o_sl, o_m, o_so = oracle.truncate_and_score(resp, h.eos_id, h.pad_id, npy(b["scores"]),
+                                                           np.float32(h.no_eos_score))
+    for got, want in ((ro, o_ro), (ei, o_ei), (sl, o_sl), (mask, o_m)):
+        assert np.array_equal(npy(got), want)
+    assert np.array_equal(npy(so).astype(np.float64), o_so)
+    m = o_m.astype(bool)
+    n = float(m.sum())
+    # fused LM head on a sample of real rows, both weight matrices; padding rows are 0
+    rng = np.random.default_rng(44)
+    real = np.flatnonzero(m.reshape(-1)).astype(np.int64)
+    sel = np.unique(np.concatenate([rng.choice(real, 96, replace=False), real[:1], real[-1:]]))
+    Hh = host_logits(b["H"])
+    tau = np.float32(h.temperature)
+    o_lp, o_ent, _ = oracle.lmhead_logprob_entropy(Hh, host_logits(b["W"]), npy(tok), tau, sel_rows=sel)
+    o_rlp, _, _ = oracle.lmhead_logprob_entropy(Hh, host_logits(b["W_ref"]), npy(tok), tau, sel_rows=sel)
+    assert_abs(npy(lp).reshape(-1)[sel], o_lp, TOL_LOGPROB, "logprob (sampled)")
+    assert_abs(npy(ent).reshape(-1)[sel], o_ent, TOL_LOGPROB, "entropy (sampled)")
+    assert_abs(npy(rlp).reshape(-1)[sel], o_rlp, TOL_LOGPROB, "ref_logprob (sampled)")
+    for t in (lp, ent, rlp):
+        assert not npy(t)[~m].any()
+        assert np.isfinite(npy(t)).all()
+    # token-level steps in full
+    o_kl, o_rew = oracle.kl_rewards(npy(lp), npy(rlp), o_m, o_sl, f32(o_so), np.float32(h.kl_coef))
+    assert_abs(npy(kl), o_kl, TOL_LOGPROB, "kl")
+    assert_rel(npy(rew), o_rew, TOL_REL, "rewards")
+    o_adv, o_ret = oracle.gae(npy(rew), npy(b["values"]), o_sl, np.float32(h.gamma), np.float32(h.lam))
+    assert_rel(npy(adv), o_adv, TOL_REL, "advantages")
+    assert_rel(npy(ret), o_ret, TOL_REL, "returns")
+    o_aw, o_st = oracle.whiten(npy(adv), o_m, True, np.float32(h.whiten_eps))
+    assert_rel(npy(aw), o_aw, TOL_REL, "whitened advantages")
+    assert_rel(npy(st), o_st, TOL_REL, "whiten stats")
+    # the loss: a two-entry vocabulary (x, 0) at temperature 1 whose log-softmax at entry 0 is the given log-prob
+    nlp = npy(lp).astype(np.float64)
+    pt = np.exp(np.minimum(nlp, -1e-12))
+    x = np.where(m, np.log(pt) - np.log1p(-pt), 0.0)
+    ref = oracle.loss_fwd_bwd(np.stack([x, np.zeros_like(x)], -1).astype(np.float32), np.zeros((B, T), np.int32), o_m,
+                              npy(old), npy(aw), npy(b["values_new"]), npy(b["values"]), npy(ret), 1.0,
+                              np.float32(h.cliprange), np.float32(h.cliprange_value), np.float32(h.vf_coef),
+                              want_dlogits=False)
+    kink = near_kink(nlp, npy(old), h.cliprange) & m
+    got = npy(out["losses"]).astype(np.float64)
+    assert got[7] == n
+    for i, name in enumerate(oracle.LOSS_NAMES[:6]):
+        tol = TOL_LOGPROB + (int(kink.sum()) / n if name == "pg_clipfrac" else 0.0)
+        assert abs(got[i] - ref["losses"][i]) <= tol, (name, got[i], ref["losses"][i])
+    assert abs(got[6] - npy(ent).astype(np.float64)[m].sum() / n) <= 1e-5
+    assert 0 < ref["losses"][4] < 1 and 0 < ref["losses"][5] < 1
+    assert_abs(n * npy(out["dvalues"]), n * ref["dvalues"], 1e-4, "n*dvalues")
+    assert_abs((n * npy(out["dlogprob"]).astype(np.float64))[~kink], (n * ref["dlogprob"])[~kink], 1e-4, "n*dlogprob")

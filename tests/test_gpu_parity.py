@@ -159,25 +159,26 @@ def test_config1_pythia_rollout_shape(P, oracle):
     _check_stagewise(P, oracle, cfg, batch, n_grad_rows=96)
 
 
-def test_config2_full_ppo_batch_sampled_rows(P, oracle):
-    """B=512 at full size: integer steps exact on everything; the logits-bound calls are checked on
-    a row sample (the oracle computes each sampled row on its own)."""
+def test_config2_full_ppo_batch_every_row(P, oracle):
+    """B=512 at full size, through the separate calls and through the single-call step the benchmark times: integer
+    steps exact; log-probs and entropy of every real row of both tensors against the oracle; every [B,T] array; the
+    loss scalars and per-token gradients of every row through the oracle's own loss; every gradient row validated
+    on the device; a sample of gradient rows element by element."""
     from paper_2403_17031_b200.synthetic import CONFIGS, make_batch
     cfg = CONFIGS[2]
-    h = cfg.hyper
     batch = make_batch(cfg, "cuda")
-    _check_sampled(P, oracle, cfg, batch, n_rows=160, seed=2)
+    _check_full_size(P, oracle, cfg, batch, n_grad_rows=160, seed=2)
 
 
-def test_config3_long_response_stress_sampled_rows(P, oracle):
-    """B=256, T=512, fp32 logits (26 GB per tensor): full-size launch, sampled-row parity."""
+def test_config3_long_response_stress_every_row(P, oracle):
+    """B=256, T=512, fp32 logits (26 GB per tensor): the same checks as config 2 at full size."""
     from paper_2403_17031_b200.synthetic import CONFIGS, make_batch
     cfg = CONFIGS[3]
     free, _ = torch.cuda.mem_get_info()
     if free < 100e9:
         pytest.skip("needs ~90 GB of free device memory")
     batch = make_batch(cfg, "cuda", chunk_rows=4096)
-    _check_sampled(P, oracle, cfg, batch, n_rows=96, seed=3)
+    _check_full_size(P, oracle, cfg, batch, n_grad_rows=512, seed=3)
 
 
 def test_config3_shape_small_batch_all_steps(P, oracle):
@@ -189,42 +190,91 @@ def test_config3_shape_small_batch_all_steps(P, oracle):
     _check_stagewise(P, oracle, replace(cfg, B=4), batch, n_grad_rows=48)
 
 
-def _check_sampled(P, O, cfg, batch, n_rows, seed):
+_STEP_OUTPUTS = ("responses_out", "eos_index", "seq_len", "mask", "scores_out", "logprob", "entropy", "ref_logprob", "kl",
+                 "rewards", "advantages", "returns", "advantages_whitened", "losses", "dvalues", "new_logprob",
+                 "new_entropy", "dlogprob")
+
+
+def _poison(hp):
+    """Fill every output with a pattern no kernel writes: a row that a launch skipped stays visible."""
+    for k, t in hp.out.items():
+        if t is None or k == "whiten_stats":
+            continue
+        if t.is_floating_point():
+            t.fill_(float("nan"))
+        else:
+            t.fill_(-77 if t.dtype != torch.uint8 else 201)
+
+
+def _row_checksums(dl, chunk=4096):
+    """One int64 per gradient row: the sum of the row's bit patterns (any changed bit changes it)."""
+    rows = dl.shape[0]
+    out = torch.empty(rows, dtype=torch.int64, device=dl.device)
+    it = torch.int16 if dl.dtype == torch.bfloat16 else torch.int32
+    for r0 in range(0, rows, chunk):
+        out[r0:r0 + chunk] = dl[r0:r0 + chunk].view(it).sum(-1, dtype=torch.int64)
+    return out
+
+
+def _oracle_logprob_rows(O, logits2d, rows_idx, tokens, tau, chunk=4096):
+    """The oracle's step 1 on the given rows of a device tensor [rows, V], copied to the host chunk by chunk."""
+    lp = np.empty(len(rows_idx)); ent = np.empty(len(rows_idx))
+    for i0 in range(0, len(rows_idx), chunk):
+        idx = rows_idx[i0:i0 + chunk]
+        x = host_logits(logits2d[torch.from_numpy(idx).to(logits2d.device)])
+        lp[i0:i0 + chunk], ent[i0:i0 + chunk], _ = O.logprob_entropy(x, tokens[idx], tau)
+    return lp, ent
+
+
+def _check_full_size(P, O, cfg, batch, n_grad_rows, seed):
     from paper_2403_17031_b200.pipeline import PPOHotPath
     h = cfg.hyper
     B, T, V = batch["policy_logits"].shape
+    rows = B * T
     bf16 = batch["policy_logits"].dtype == torch.bfloat16
     rng = np.random.default_rng(seed)
+    tau = np.float32(h.temperature)
     hp = PPOHotPath(B, T, V, batch["policy_logits"].dtype, _params(P, h))
-    o = hp.rollout_stats(batch["policy_logits"], batch["ref_logits"], batch["responses"], batch["scores"],
-                         batch["values"])
+    args = (batch["policy_logits"], batch["ref_logits"], batch["responses"], batch["scores"], batch["values"])
+
+    # ---- the separate calls
+    _poison(hp)
+    o = hp.rollout_stats(*args)
     old = (o["logprob"] + batch["old_logprob_noise"]).contiguous()
     o = hp.loss(batch["policy_logits"], batch["responses"], old, batch["values_new"], batch["values"])
     torch.cuda.synchronize()
     assert hp.device_status() == 0
-    # integer step: exact, everywhere
+    sep = {k: o[k].clone() for k in _STEP_OUTPUTS}
+    dl2 = o["dlogits"].view(rows, V)
+    sep_sums = _row_checksums(dl2)
+
+    # ---- integer step: exact, everywhere
     resp = npy(batch["responses"])
     ro, ei, sl, m, so = O.truncate_and_score(resp, h.eos_id, h.pad_id, npy(batch["scores"]), np.float32(h.no_eos_score))
     for k, want in (("responses_out", ro), ("eos_index", ei), ("seq_len", sl), ("mask", m)):
         assert np.array_equal(npy(o[k]), want), k
+    assert np.array_equal(npy(o["scores_out"]).astype(np.float64), so)
     mask_np = m.astype(bool)
+    flat_mask = mask_np.reshape(-1)
     n = float(mask_np.sum())
     assert float(o["losses"][7]) == n
-    # sampled rows of the logits-bound steps
-    real = np.flatnonzero(mask_np.reshape(-1))
-    sel = np.sort(rng.choice(real, min(n_rows, len(real)), replace=False)).astype(np.int64)
-    sel_t = torch.from_numpy(sel).cuda()
-    tau = np.float32(h.temperature)
-    tok = resp.reshape(-1)[sel]
-    pl = host_logits(batch["policy_logits"].reshape(-1, V)[sel_t])
-    rl = host_logits(batch["ref_logits"].reshape(-1, V)[sel_t])
-    lp, ent, _ = O.logprob_entropy(pl, tok, tau)
-    rlp, _, _ = O.logprob_entropy(rl, tok, tau)
-    assert_abs(npy(o["logprob"]).reshape(-1)[sel], lp, TOL_LOGPROB, "logprob (sampled)")
-    assert_abs(npy(o["entropy"]).reshape(-1)[sel], ent, TOL_LOGPROB, "entropy (sampled)")
-    assert_abs(npy(o["ref_logprob"]).reshape(-1)[sel], rlp, TOL_LOGPROB, "ref_logprob (sampled)")
-    assert_abs(npy(o["new_logprob"]).reshape(-1)[sel], lp, TOL_LOGPROB, "new_logprob (sampled)")
-    # token-level steps: whole arrays, each fed the GPU's own upstream fp32 outputs
+    real = np.flatnonzero(flat_mask).astype(np.int64)
+    masked = np.flatnonzero(~flat_mask).astype(np.int64)
+
+    # ---- step 1 on EVERY real row of both tensors (and the loss kernel's own log-prob / entropy of the policy rows)
+    tok_flat = resp.reshape(-1)
+    lp, ent = _oracle_logprob_rows(O, batch["policy_logits"].view(rows, V), real, tok_flat, tau)
+    rlp, _ = _oracle_logprob_rows(O, batch["ref_logits"].view(rows, V), real, tok_flat, tau)
+    pick = lambda name: npy(o[name]).reshape(-1)
+    assert_abs(pick("logprob")[real], lp, TOL_LOGPROB, "logprob (every real row)")
+    assert_abs(pick("entropy")[real], ent, TOL_LOGPROB, "entropy (every real row)")
+    assert_abs(pick("ref_logprob")[real], rlp, TOL_LOGPROB, "ref_logprob (every real row)")
+    assert_abs(pick("new_logprob")[real], lp, TOL_LOGPROB, "new_logprob (every real row)")
+    assert_abs(pick("new_entropy")[real], ent, TOL_LOGPROB, "new_entropy (every real row)")
+    for k in ("logprob", "entropy", "ref_logprob", "new_logprob", "new_entropy", "dlogprob", "dvalues"):
+        assert not pick(k)[masked].any(), k + " must be 0 on padding rows"
+
+    # ---- token-level steps: whole arrays, each fed the GPU's own upstream fp32 outputs
     kl, rew = O.kl_rewards(npy(o["logprob"]), npy(o["ref_logprob"]), m, sl, f32(so), np.float32(h.kl_coef))
     assert_abs(npy(o["kl"]), kl, TOL_LOGPROB, "kl")
     assert_rel(npy(o["rewards"]), rew, TOL_REL, "rewards")
@@ -233,31 +283,102 @@ def _check_sampled(P, O, cfg, batch, n_rows, seed):
     assert_rel(npy(o["returns"]), ret, TOL_REL, "returns")
     aw, st = O.whiten(npy(o["advantages"]), m, True, np.float32(h.whiten_eps))
     assert_rel(npy(o["advantages_whitened"]), aw, TOL_REL, "whitened advantages")
-    # loss gradients of the sampled rows: the oracle runs on the sample as a [1, k, V] batch, whose
+
+    # ---- loss scalars and per-token gradients of EVERY row through the oracle's own loss: a two-entry
+    # vocabulary (x, 0) at temperature 1 whose log-softmax at entry 0 is the GPU's new_logprob (x = logit(p))
+    nlp_gpu = npy(o["new_logprob"]).astype(np.float64)
+    p_tok = np.exp(np.minimum(nlp_gpu, -1e-12))
+    x = np.where(mask_np, np.log(p_tok) - np.log1p(-p_tok), 0.0)
+    lg2 = np.stack([x, np.zeros_like(x)], -1)
+    # (the oracle widens fp32 logits; x in fp32 moves new_logprob by <= 6e-8 * |x|, far inside the tolerance)
+    old_np = npy(old)
+    ref2 = O.loss_fwd_bwd(lg2.astype(np.float32), np.zeros((B, T), np.int32), m, old_np, npy(o["advantages_whitened"]),
+                          npy(batch["values_new"]), npy(batch["values"]), npy(o["returns"]), 1.0,
+                          np.float32(h.cliprange), np.float32(h.cliprange_value), np.float32(h.vf_coef),
+                          want_dlogits=False)
+    assert_abs(ref2["new_logprob"][mask_np], nlp_gpu[mask_np], 2e-5, "two-entry construction reproduces new_logprob")
+    kink = near_kink(nlp_gpu, old_np, h.cliprange) & mask_np
+    got_l = npy(o["losses"]).astype(np.float64)
+    for i, name in enumerate(O.LOSS_NAMES[:6]):
+        tol = TOL_LOGPROB + (int(kink.sum()) / n if name == "pg_clipfrac" else 0.0)
+        assert abs(got_l[i] - ref2["losses"][i]) <= tol, (name, got_l[i], ref2["losses"][i])
+    assert abs(got_l[6] - ent.sum() / n) <= TOL_LOGPROB, "mean entropy"
+    assert 0 < ref2["losses"][4] < 1 and 0 < ref2["losses"][5] < 1          # both clip branches fire
+    assert_abs(n * npy(o["dvalues"]), n * ref2["dvalues"], 1e-4, "n*dvalues (every row)")
+    assert_abs((n * npy(o["dlogprob"]).astype(np.float64))[~kink], (n * ref2["dlogprob"])[~kink], 1e-4,
+               "n*dlogprob (every row)")
+
+    # ---- every gradient row, on the device: finite; padding rows all zero; a real row sums to ~0, its entry at
+    # the sampled token is g/tau * (1 - p_tok), and its absolute values sum to 2 |g|/tau (1 - p_tok)
+    tok_d = batch["responses"].reshape(-1).long()
+    g_d = o["dlogprob"].reshape(-1).double() / float(tau)
+    onem_p = -torch.expm1(o["new_logprob"].reshape(-1).double())
+    mask_d = o["mask"].reshape(-1).bool()
+    # tolerances: one rounding to the output type (2^-9 relative for bf16) on every entry, plus the fp32 evaluation
+    # error of the probabilities (a few 1e-6 of |g|/tau, which matters where 1 - p_tok is tiny)
+    rel = 2.0 ** -7 if bf16 else 1e-4
+    for r0 in range(0, rows, 4096):
+        c = dl2[r0:r0 + 4096]
+        mk = mask_d[r0:r0 + 4096]
+        assert bool(torch.isfinite(c).all()), "non-finite gradient rows in [%d, %d)" % (r0, r0 + 4096)
+        cd = c.double()
+        assert not bool(cd[~mk].any()), "padding rows of dlogits must be zero"
+        want_tok = (g_d[r0:r0 + 4096] * onem_p[r0:r0 + 4096])
+        got_tok = cd.gather(1, tok_d[r0:r0 + 4096, None])[:, 0]
+        scale = n * want_tok.abs()
+        slack = 1e-5 * n * g_d[r0:r0 + 4096].abs()
+        assert bool(((n * (got_tok - want_tok)).abs() <= rel * scale + slack + 1e-6)[mk].all()), \
+            "dlogits at the sampled token"
+        assert bool(((n * cd.sum(1)).abs() <= rel * scale + slack + 1e-4)[mk].all()), "row sums"
+        assert bool(((n * cd.abs().sum(1) - 2 * scale).abs() <= 2 * (rel * scale + slack) + 1e-4)[mk].all()), \
+            "row L1 norms"
+        del cd
+
+    # ---- a sample of gradient rows element by element: the oracle runs on the sample as a [1, k, V] batch, whose
     # normaliser is k instead of n, so n*gradient of the full batch equals k*gradient of the sample
+    first_last = np.array([real[0], real[-1], real[real < T][-1], real[real >= (B - 1) * T][0]], np.int64)
+    sel = np.unique(np.concatenate([rng.choice(real, min(n_grad_rows, len(real)), replace=False), first_last]))
+    sel_t = torch.from_numpy(sel).cuda()
     k = len(sel)
-    pick = lambda name: npy(o[name]).reshape(-1)[sel][None]
-    sub = O.loss_fwd_bwd(pl[None], tok[None], np.ones((1, k), np.uint8), npy(old).reshape(-1)[sel][None],
-                         pick("advantages_whitened"), npy(batch["values_new"]).reshape(-1)[sel][None],
-                         npy(batch["values"]).reshape(-1)[sel][None], pick("returns"), tau,
+    pl = host_logits(batch["policy_logits"].view(rows, V)[sel_t])
+    pk = lambda name: pick(name)[sel][None]
+    sub = O.loss_fwd_bwd(pl[None], tok_flat[sel][None], np.ones((1, k), np.uint8), old_np.reshape(-1)[sel][None],
+                         pk("advantages_whitened"), npy(batch["values_new"]).reshape(-1)[sel][None],
+                         npy(batch["values"]).reshape(-1)[sel][None], pk("returns"), tau,
                          np.float32(h.cliprange), np.float32(h.cliprange_value), np.float32(h.vf_coef))
-    kink = near_kink(sub["new_logprob"], npy(old).reshape(-1)[sel][None], h.cliprange).reshape(-1)
-    dl = n * o["dlogits"].reshape(-1, V)[sel_t].float().cpu().numpy().astype(np.float64)
-    assert_grad(dl[~kink], k * sub["dlogits"][~kink], bf16, "n*dlogits (sampled)")
-    assert_abs(n * pick("dvalues")[0], k * sub["dvalues"][0], 1e-4, "n*dvalues (sampled)")
-    assert_abs((n * pick("dlogprob")[0])[~kink], (k * sub["dlogprob"][0])[~kink], 1e-4, "n*dlogprob (sampled)")
-    # masked rows: zero-filled (sample) and the loss scalars agree with the log-prob-level entry point
-    masked = np.flatnonzero(~mask_np.reshape(-1))
-    if len(masked):
-        ms = torch.from_numpy(np.sort(rng.choice(masked, min(64, len(masked)), replace=False))).cuda()
-        assert not o["dlogits"].reshape(-1, V)[ms].any().item()
+    kk = near_kink(sub["new_logprob"], old_np.reshape(-1)[sel][None], h.cliprange).reshape(-1)
+    dl = n * dl2[sel_t].float().cpu().numpy().astype(np.float64)
+    assert_grad(dl[~kk], k * sub["dlogits"][~kk], bf16, "n*dlogits (sampled rows)")
+
+    # ---- the log-prob-level entry point on the same per-token inputs: same bits
     o2 = P.loss_from_logprob(o["new_logprob"], o["new_entropy"], o["mask"], old, o["advantages_whitened"],
                              batch["values_new"], batch["values"], o["returns"], _params(P, h), hp.workspace)
     assert torch.equal(o2["losses"], o["losses"]) and torch.equal(o2["dvalues"], o["dvalues"])
     assert torch.equal(o2["dlogprob"], o["dlogprob"])
-    # and the scalars against the oracle's log-prob-level arithmetic on the GPU's own new_logprob is
-    # covered stage-wise at the smaller configs; here check the normaliser and finiteness
-    assert torch.isfinite(o["losses"]).all()
+
+    # ---- the single-call step (the launch configuration the benchmark times: overlapped launches, dynamic row
+    # hand-out), eager and as a replayed CUDA graph, then a later epoch: every output bit equal to the separate calls
+    step_args = args + (batch["values_new"],)
+    for how in ("eager", "graph", "next_epoch"):
+        _poison(hp)
+        if how == "eager":
+            hp.step(*step_args, old_logprob=old)
+        elif how == "graph":
+            graph = hp.capture_step(*step_args, old_logprob=old)
+            _poison(hp)
+            graph.replay()
+        else:
+            hp.step(*step_args, old_logprob=old)
+            for name in ("losses", "dlogits", "dvalues", "new_logprob", "new_entropy", "dlogprob"):
+                hp.out[name].fill_(float("nan"))
+            hp.loss(batch["policy_logits"], batch["responses"], old, batch["values_new"], batch["values"],
+                    next_epoch=True)
+        torch.cuda.synchronize()
+        assert hp.device_status() == 0, how
+        names = _STEP_OUTPUTS if how != "next_epoch" else ("losses", "dvalues", "new_logprob", "new_entropy", "dlogprob")
+        for name in names:
+            assert torch.equal(hp.out[name], sep[name]), (name, how)
+        assert torch.equal(_row_checksums(hp.out["dlogits"].view(rows, V)), sep_sums), ("dlogits", how)
 
 
 def test_single_call_step_and_host_step_match_the_separate_calls(P):

@@ -242,30 +242,61 @@ def test_gae_closed_forms(oracle):
 
 
 # ---------------------------------------------------------------- step 5: whitening
-def _paper_whiten(values, shift_mean=True):
-    """The whiten() semantics stated in the paper, evaluated with library mean/var."""
-    mean, var = values.mean(), values.var()          # numpy var is the biased one
-    w = (values - mean) / np.sqrt(var + 1e-8)
-    return w if shift_mean else w + mean
+def _moments_exact(values):
+    """Mean and population variance of integer-valued data from the raw power sums, in exact rational arithmetic
+    (one pass, var = E[x^2] - E[x]^2): structured unlike the oracle's two passes over centred values."""
+    from fractions import Fraction
+    xs = [Fraction(int(v)) for v in np.asarray(values).reshape(-1)]
+    n = len(xs)
+    s1, s2 = sum(xs), sum(v * v for v in xs)
+    mean = s1 / n
+    return mean, s2 / n - mean * mean
 
 
-def test_whiten_matches_paper_listing_semantics(oracle):
+def test_whiten_closed_forms_and_properties(oracle):
+    """Listing "whiten" and detail "Advantage whitening": population (not sample) variance, 1e-8 inside the square
+    root, zero mean by default and the mean added back on request."""
+    # two points 0 and 2: mean 1, population variance 1 (the sample variance would be 2)
+    y, st = oracle.whiten(np.array([0.0, 2.0]), None, True, 1e-8)
+    assert st.tolist() == [1.0, 1.0, 2.0]
+    assert np.allclose(y, np.array([-1.0, 1.0]) / np.sqrt(1.0 + 1e-8), atol=1e-15)
+    y, _ = oracle.whiten(np.array([0.0, 2.0]), None, False, 1e-8)
+    assert np.allclose(y, 1.0 + np.array([-1.0, 1.0]) / np.sqrt(1.0 + 1e-8), atol=1e-15)
+    # a constant array: variance 0, so the 1e-8 alone keeps the division finite and the result is 0 (or the mean)
+    y, st = oracle.whiten(np.full(7, 4.0), None, True, 1e-8)
+    assert st[1] == 0.0 and not y.any()
+    y, _ = oracle.whiten(np.full(7, 4.0), None, False, 1e-8)
+    assert np.array_equal(y, np.full(7, 4.0))
+    # integer-valued data against exact rational moments
     rng = np.random.default_rng(8)
-    x = rng.normal(3.0, 2.0, (16, 53))
+    x = rng.integers(-50, 50, (16, 53)).astype(np.float64)
+    mean_q, var_q = _moments_exact(x)
     for sm in (True, False):
         y, st = oracle.whiten(x, None, sm, 1e-8)
-        assert np.allclose(y, _paper_whiten(x, sm), atol=1e-12)
-        assert abs(st[0] - x.mean()) < 1e-12 and abs(st[1] - x.var()) < 1e-12 and st[2] == x.size
+        assert abs(st[0] - float(mean_q)) < 1e-13 and abs(st[1] - float(var_q)) < 1e-11 and st[2] == x.size
+        want = (x - float(mean_q)) / np.sqrt(float(var_q) + 1e-8) + (0.0 if sm else float(mean_q))
+        assert np.allclose(y, want, atol=1e-12)
+        # properties: mean 0 (or the input's mean), variance var / (var + 1e-8)
+        assert abs(y.mean() - (0.0 if sm else float(mean_q))) < 1e-12
+        assert abs(((y - y.mean()) ** 2).mean() - float(var_q) / (float(var_q) + 1e-8)) < 1e-12
     # masked: statistics over mask==1 entries only, zeros elsewhere
     m = (rng.random((16, 53)) < 0.6).astype(np.uint8)
-    y, st = oracle.whiten(x, m, True, 1e-8)
     sel = m.astype(bool)
-    assert np.allclose(y[sel], _paper_whiten(x[sel]), atol=1e-12)
+    y, st = oracle.whiten(x, m, True, 1e-8)
+    mq, vq = _moments_exact(x[sel])
+    assert abs(st[0] - float(mq)) < 1e-13 and abs(st[1] - float(vq)) < 1e-11 and st[2] == sel.sum()
+    assert np.allclose(y[sel], (x[sel] - float(mq)) / np.sqrt(float(vq) + 1e-8), atol=1e-12)
     assert not y[~sel].any()
     assert abs(y[sel].mean()) < 1e-12
-    assert abs(y[sel].var() - st[1] / (st[1] + 1e-8)) < 1e-12
-    y2, _ = oracle.whiten(-3.0 * x + 7.0, m, True, 1e-8)         # affine map with a < 0 flips sign
-    assert np.allclose(y2, -y, atol=1e-7)
+    assert abs((y[sel] ** 2).mean() - st[1] / (st[1] + 1e-8)) < 1e-12
+    # entries behind the mask do not matter
+    x2 = x.copy()
+    x2[~sel] = 1e9
+    y2, st2 = oracle.whiten(x2, m, True, 1e-8)
+    assert np.array_equal(y2, y) and np.array_equal(st2, st)
+    # an affine map a*x + b with a < 0 flips the sign and nothing else (variance far above 1e-8)
+    y3, _ = oracle.whiten(-3.0 * x + 7.0, m, True, 1e-8)
+    assert np.allclose(y3, -y, atol=1e-7)
     y1, _ = oracle.whiten(np.array([2.5, 9.0]), np.array([1, 0], np.uint8), True, 1e-8)   # n = 1
     assert y1.tolist() == [0.0, 0.0]
 
