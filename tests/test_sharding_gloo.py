@@ -82,3 +82,27 @@ def test_two_rank_sharded_rows_equal_unsharded(oracle):
         L_cat += L
         assert tmax == 2.0 and units == 6 * cfg.T
     assert lp_cat == lp_full.tolist() and L_cat == L_full.tolist()
+
+
+def test_bench_starts_its_own_ranks_and_prints_one_line():
+    """`bench.py --gpus 2` without a launcher starts two ranks itself; the plumbing arm runs the launch, the process
+    group and the reduction of the timing without any kernel (gloo here), and rank 0 alone prints the JSON line."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    env["CUDA_VISIBLE_DEVICES"] = ""
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--impl", "plumbing"],
+                         capture_output=True, text=True, timeout=240, env=env)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, out.stdout
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["ranks_seen"] == 2 and d["sequences_owned_total"] == 512
+    assert d["max_ms"] >= 19.0          # the slower rank's time (rank 1 sleeps 20 ms), not rank 0's
+    # a rank count that contradicts the launcher is refused
+    env2 = dict(env, RANK="0", WORLD_SIZE="1", LOCAL_RANK="0")
+    bad = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--impl", "plumbing"],
+                         capture_output=True, text=True, timeout=120, env=env2)
+    assert bad.returncode != 0 and "ranks" in bad.stderr
