@@ -11,9 +11,18 @@ kernel can be compared with it token by token:
     offset high), output word = element index % 4;
   * uniform: u = (floor(x / 2^9) + 1/2) * 2^-23 for a 32-bit word x, so u lies strictly inside (0, 1) and is an
     fp32 number;
-  * draw: the token of row r is argmax_j [ y_j - log2(-log2 u_j) ] with y_j = logit_j * log2(e) / tau (the
-    Gumbel-max rule in base 2; equivalently the index that minimises the exponential variate -log2(u_j)
-    divided by the unnormalised probability 2^(y_j)); exact ties go to the lowest index.
+  * draw, in two levels (an exponential race may be run group by group: the group whose total weight wins
+    its race is the group of the overall winner with the right probability, and inside a group the members
+    race with their own weights). The V elements are dealt into C = 256 classes in runs of 8:
+    class(j) = floor(j / 8) mod 256.
+      level 1: W_c = sum over the class of 2^(y_j), y_j = logit_j * log2(e) / tau; the class is
+               argmax_c [ log2 W_c - log2(-log2 v_c) ] over the classes with W_c > 0, ties to the lowest c, with
+               v_c the uniform of word c % 4 of the counter (2^31 + floor(c / 4), row, offset low, offset high);
+      level 2: the token is argmax_j [ y_j - log2(-log2 u_j) ] over the elements j of that class, ties to the
+               lowest j, with u_j the uniform of word j % 4 of the counter (floor(j / 4), row, offset low, offset high).
+    (log2 W - log2(-log2 u) is the Gumbel-max form, in base 2, of minimising the exponential variate -log2(u)
+    divided by the weight.) Every element is drawn with probability 2^(y_j) / sum_k 2^(y_k) = softmax(logits / tau)_j.
+    Only 256 + V/256 uniforms per row decide the draw, so a kernel needs the generator for the winning class only.
 """
 from __future__ import annotations
 
@@ -50,12 +59,51 @@ def uniforms(rows: int, V: int, seed: int, offset: int = 0, row0: int = 0):
     return ((x >> np.uint32(9)).astype(np.float64) + 0.5) * 2.0 ** -23
 
 
+N_CLASSES = 256
+RUN = 8
+CLASS_COUNTER_BASE = 1 << 31
+
+
+def class_of(V: int):
+    """class(j) for j = 0 .. V-1."""
+    return (np.arange(V) // RUN) % N_CLASSES
+
+
+def class_uniforms(rows: int, seed: int, offset: int = 0, row0: int = 0):
+    """v [rows, 256] float64: the uniforms of level 1."""
+    c = np.arange(N_CLASSES, dtype=np.uint64)
+    r = (np.arange(rows, dtype=np.uint64) + np.uint64(row0))[:, None]
+    words = philox4x32_10((np.uint64(CLASS_COUNTER_BASE) + (c >> np.uint64(2)))[None, :], r,
+                          np.uint64(offset & 0xFFFFFFFF), np.uint64((offset >> 32) & 0xFFFFFFFF), seed & 0xFFFFFFFF,
+                          (seed >> 32) & 0xFFFFFFFF)
+    sel = (c & np.uint64(3)).astype(np.int64)[None, :]
+    x = np.choose(np.broadcast_to(sel, words[0].shape), words)
+    return ((x >> np.uint32(9)).astype(np.float64) + 0.5) * 2.0 ** -23
+
+
 def sample(logits, temperature: float, seed: int, offset: int = 0):
-    """logits [rows, V] float64 (already widened). Returns (tokens int64 [rows], keys [rows, V] float64): the
-    perturbed base-2 scores whose argmax is the token."""
+    """logits [rows, V] float64 (already widened). Returns (tokens int64 [rows], keys1 [rows, 256], keys2 [rows, V],
+    cls [V]): keys1 are the perturbed base-2 scores of the classes (-inf for a class without weight), keys2 those of the
+    elements; the token is the argmax of keys2 over the class that is the argmax of keys1."""
     x = np.asarray(logits, np.float64)
+    rows, V = x.shape
     y = x * (np.log2(np.e) / float(temperature))
-    u = uniforms(x.shape[0], x.shape[1], seed, offset)
-    with np.errstate(divide="ignore"):
-        keys = y - np.log2(-np.log2(u))
-    return keys.argmax(axis=1), keys
+    cls = class_of(V)
+    u = uniforms(rows, V, seed, offset)
+    v = class_uniforms(rows, seed, offset)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        keys2 = y - np.log2(-np.log2(u))
+        keys1 = np.full((rows, N_CLASSES), -np.inf)
+        tokens = np.empty(rows, np.int64)
+        for r in range(rows):
+            ymax = y[r].max()
+            if not np.isfinite(ymax):                      # no element with weight (or a +inf / NaN): nothing is drawn
+                tokens[r] = -1
+                continue
+            W = np.bincount(cls, weights=np.exp2(y[r] - ymax), minlength=N_CLASSES)    # the class sums
+            has = W > 0
+            keys1[r, has] = (ymax + np.log2(W[has])) - np.log2(-np.log2(v[r, has]))
+            c_star = int(keys1[r].argmax())
+            inside = np.where(cls == c_star, keys2[r], -np.inf)
+            tokens[r] = int(inside.argmax())
+    return tokens, keys1, keys2, cls
