@@ -285,9 +285,16 @@ int ppo_logprob_entropy_pair(const void *policy_logits, const void *ref_logits, 
  * Temperature sampling fused with step 1 (Table "PPO hyperparameters": temperature): draws one token
  * per row from softmax(logits / temperature) and returns its log-prob, the row's entropy and
  * log-sum-exp from the same single pass over HBM.  The draw is reproducible and defined as follows:
- *   word(j)  = Philox4x32-10 with key = seed, counter = (j / 4, row, offset low, offset high), output j % 4
- *   u_j      = (floor(word(j) / 2^9) + 1/2) * 2^-23            (an fp32 number in (0, 1))
- *   token    = argmax_j [ logit_j * log2(e) / temperature - log2(-log2 u_j) ], ties to the lowest j
+ *   uniform(w) = (floor(w / 2^9) + 1/2) * 2^-23 for a 32-bit word w    (an fp32 number in (0, 1))
+ *   words come from Philox4x32-10 with key = seed; y_j = logit_j * log2(e) / temperature
+ *   The row is dealt into 256 classes in runs of 8 elements, class(j) = (j / 8) mod 256, and an exponential
+ *   race (the Gumbel-max rule) is run in two levels:
+ *   level 1:  W_c = sum of 2^(y_j) over class c;  v_c = uniform(word c % 4 of counter (2^31 + c / 4, row,
+ *             offset low, offset high));  class = argmax_c [ log2 W_c - log2(-log2 v_c) ], ties to the lowest c
+ *   level 2:  u_j = uniform(word j % 4 of counter (j / 4, row, offset low, offset high));
+ *             token = argmax over the class's j of [ y_j - log2(-log2 u_j) ], ties to the lowest j
+ *   Element j is drawn with probability softmax(logits / temperature)_j; only the winning class needs its
+ *   elements' uniforms, which is why the call runs at the speed of ppo_logprob_entropy.
  * Use a new `offset` for every call that must be independent of the previous ones with the same seed.
  *   logits [rows, V] dtype, row pitch row_stride >= V elements
  *   tokens_out [rows] i32; logprob, entropy, lse nullable [rows] f32 (as in ppo_logprob_entropy)

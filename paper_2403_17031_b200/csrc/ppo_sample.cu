@@ -4,18 +4,24 @@
 // streamed from HBM once for both.
 //
 // The draw is defined so that it can be reproduced on a CPU token by token:
-//   * Philox4x32-10 (counter-based; Salmon et al., SC'11): key = seed, counter = (j / 4, row, offset low,
-//     offset high), word j % 4 belongs to element j of the row;
-//   * u_j = (floor(word / 2^9) + 1/2) * 2^-23, an fp32 number strictly inside (0, 1);
-//   * the token is the j that minimises E_j / 2^(y_j) with E_j = -log2(u_j) (an exponential race; the
-//     same as the Gumbel-max rule argmax_j [y_j - log2(-log2 u_j)]), y_j = logit_j * log2(e) / tau.
-//     Candidates are compared by cross-multiplication (E_j * e_best < E_best * e_j with e = 2^(y - max)),
-//     so the race costs no division and reuses the exponential that the softmax sums need anyway;
-//     exact ties go to the lowest index.
-// One block per row, one pass: the exponentials are taken relative to the maximum of the row's first pack
-// (any reference serves the race and the sums); a row whose sums overflow that way, or that holds a NaN or
-// an infinity, is repeated with its exact maximum. The generator dominates: ~10 integer instructions per
-// logit next to ~12 for everything else, so this kernel is bound by instruction issue, not by HBM.
+//   * Philox4x32-10 (counter-based; Salmon et al., SC'11), key = seed; a 32-bit word w gives the uniform
+//     (floor(w / 2^9) + 1/2) * 2^-23, an fp32 number strictly inside (0, 1);
+//   * an exponential race (the Gumbel-max rule) in two levels. The row is dealt into 256 classes in runs of 8
+//     elements, class(j) = (j / 8) mod 256, which is exactly the set of elements thread c of a 256-thread block
+//     streams. Level 1: class c has weight W_c = sum of 2^(y_j) over its elements (y_j = logit_j * log2(e) / tau:
+//     the thread's share of the softmax sum, needed anyway) and the uniform of word c % 4 of the counter
+//     (2^31 + c / 4, row, offset low, offset high); the class that minimises -log2(v_c) / W_c wins. Level 2: inside
+//     that class, element j has the uniform of word j % 4 of the counter (j / 4, row, offset low, offset high) and
+//     the element that minimises -log2(u_j) / 2^(y_j) is the token. Every element is drawn with probability
+//     softmax(logits / tau)_j, and only 256 + V / 256 uniforms per row are ever needed, so the generator costs
+//     nothing next to the stream of logits: the kernel runs at the speed of the plain log-prob pass.
+//     Candidates are compared by cross-multiplication (E_a * w_b < E_b * w_a), no division; exact ties go to
+//     the lowest index.
+// One block of 256 threads per row, one pass over the logits: the exponentials are taken relative to the maximum
+// of the row's first pack (any reference serves the race and the sums); a row whose sums overflow that way, or
+// that holds a NaN or an infinity (-inf included), is repeated with clamped values and its exact maximum. Then two short block-wide steps: the race
+// between the 256 class sums, and the race between the members of the winning class (one member per thread,
+// re-read from L2).
 #include "ppo_rows.cuh"
 
 namespace ppo {
@@ -23,29 +29,20 @@ namespace ppo {
 constexpr uint32_t kPhiloxM0 = 0xD2511F53u, kPhiloxM1 = 0xCD9E8D57u;
 constexpr uint32_t kPhiloxW0 = 0x9E3779B9u, kPhiloxW1 = 0xBB67AE85u;
 
-// the ten round keys depend on the seed only: computed once per thread (uniform across the grid)
-struct PhiloxKeys {
-    uint32_t k0[10], k1[10];
-    __device__ __forceinline__ void init(uint32_t a, uint32_t b)
-    {
-#pragma unroll
-        for (int r = 0; r < 10; ++r) {
-            k0[r] = a + (uint32_t)r * kPhiloxW0;
-            k1[r] = b + (uint32_t)r * kPhiloxW1;
-        }
-    }
-};
-
-__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, const PhiloxKeys &k,
+// (the round keys are derived on the fly: a thread runs the generator twice per row, and nothing of it should
+// occupy registers during the pass over the logits)
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1,
                                               uint32_t (&o)[4])
 {
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
         const uint64_t p0 = (uint64_t)kPhiloxM0 * c0, p1 = (uint64_t)kPhiloxM1 * c2;   // one wide multiply each
-        c0 = (uint32_t)(p1 >> 32) ^ c1 ^ k.k0[r];
+        c0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
         c1 = (uint32_t)p1;
-        c2 = (uint32_t)(p0 >> 32) ^ c3 ^ k.k1[r];
+        c2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
         c3 = (uint32_t)p0;
+        k0 += kPhiloxW0;
+        k1 += kPhiloxW1;
     }
     o[0] = c0; o[1] = c1; o[2] = c2; o[3] = c3;
 }
@@ -89,128 +86,174 @@ struct SampleArgs {
     int *status;
 };
 
+constexpr int kSampleThreads = 256;      // = number of classes of the draw
+constexpr int kRun = 8;                  // consecutive elements that go to the same class
+constexpr uint32_t kClassCounterBase = 0x80000000u;
+
 struct SampleSmem {
-    float rs[32], ru[32], re[32], rl[32];
-    int rj[32];
-    float bs, bu;
+    float rs[8], ru[8], re[8], rl[8];
+    int rj[8];
+    float bs, bu, be;
+    int bj;
     int redo;
 };
 
-// softmax sums and race of one row relative to the reference m (base-2 units); result in thread 0
-template <typename T, bool VECTOR, int THREADS>
-__device__ __forceinline__ void sums_and_race(const T *src, int V, float c, float m, uint32_t row, const SampleArgs &a,
-                                              const PhiloxKeys &keys, SampleSmem &sm, float &s_out, float &u_out,
-                                              Race &best_out)
+// block-wide race (fixed order: lanes, then warps); the winner is returned to every thread
+__device__ __forceinline__ Race block_race(Race best, SampleSmem &sm)
 {
-    constexpr int N = Pack<T>::N;
-    constexpr int WARPS = THREADS / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const float nm = -m;
-    float s0 = 0.f, s1 = 0.f, u0 = 0.f, u1 = 0.f;
-    Race best;
-    best.init();
-    if (VECTOR) {
-        const uint4 *src4 = reinterpret_cast<const uint4 *>(src);
-        const int nvec = V / N;
-        for (int i = threadIdx.x; i < nvec; i += THREADS) {
-            float x[N];
-            Pack<T>::unpack_clamped(src4[i], x);
-#pragma unroll
-            for (int h = 0; h < N / 4; ++h) {
-                uint32_t w[4];
-                philox4x32_10((uint32_t)(i * (N / 4) + h), row, a.off_lo, a.off_hi, keys, w);
-#pragma unroll
-                for (int q = 0; q < 4; q += 2) {   // packed fp32x2 arithmetic: two elements per instruction
-                    const float2 t = __ffma2_rn(make_float2(x[h * 4 + q], x[h * 4 + q + 1]), make_float2(c, c),
-                                                make_float2(nm, nm));
-                    const float2 e = make_float2(ex2(t.x), ex2(t.y));
-                    const float2 sn = __fadd2_rn(make_float2(s0, s1), e);
-                    const float2 un = __ffma2_rn(e, t, make_float2(u0, u1));
-                    s0 = sn.x; s1 = sn.y; u0 = un.x; u1 = un.y;
-                    best.offer(e.x, log2_uniform(w[q]), i * N + h * 4 + q);
-                    best.offer(e.y, log2_uniform(w[q + 1]), i * N + h * 4 + q + 1);
-                }
-            }
-        }
-    } else {
-        for (int j = threadIdx.x; j < V; j += THREADS) {
-            float x = Pack<T>::load1(src + j);
-            x = (x != x) ? x : fmaxf(x, kNegBig);
-            uint32_t w[4];
-            philox4x32_10((uint32_t)(j >> 2), row, a.off_lo, a.off_hi, keys, w);
-            const float t = fmaf(x, c, nm);
-            const float e = ex2(t);
-            s0 += e;
-            u0 = fmaf(e, t, u0);
-            best.offer(e, log2_uniform(w[j & 3]), j);
-        }
-    }
-    // block merge: sums by addition, race by comparison (fixed order: lanes, then warps)
-    float s = s0 + s1, u = u0 + u1;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
-        s += __shfl_xor_sync(0xffffffffu, s, off);
-        u += __shfl_xor_sync(0xffffffffu, u, off);
         Race o;
         o.e = __shfl_xor_sync(0xffffffffu, best.e, off);
         o.L = __shfl_xor_sync(0xffffffffu, best.L, off);
         o.j = __shfl_xor_sync(0xffffffffu, best.j, off);
         best.merge(o);
     }
-    __syncthreads();   // the arrays below may still be read from an earlier call
-    if (lane == 0) {
-        sm.rs[warp] = s; sm.ru[warp] = u; sm.re[warp] = best.e; sm.rl[warp] = best.L; sm.rj[warp] = best.j;
+    __syncthreads();   // the arrays below may still be read from the step before
+    if (lane == 0) { sm.re[warp] = best.e; sm.rl[warp] = best.L; sm.rj[warp] = best.j; }
+    __syncthreads();
+    Race w;
+    w.init();
+#pragma unroll
+    for (int k = 0; k < kSampleThreads / 32; ++k) {
+        Race o;
+        o.e = sm.re[k]; o.L = sm.rl[k]; o.j = sm.rj[k];
+        w.merge(o);
+    }
+    return w;
+}
+
+// The softmax sums of one row relative to the reference m (base-2 units), thread c summing class c, then the two
+// levels of the race. Returns the row sums (s, u) and the winning element to every thread.
+// CLAMP: -inf logits are clamped (first attempt without: 0 * -inf then turns the entropy sum into NaN and the row is repeated).
+template <typename T, bool VECTOR, bool CLAMP>
+__device__ __forceinline__ void sums_and_race(const T *src, int V, float c, float m, uint32_t row, const SampleArgs &a,
+                                              SampleSmem &sm, float &s_out, float &u_out, Race &best_out)
+{
+    constexpr int N = Pack<T>::N, PPR = kRun / N;   // packs per run: 1 (bf16) or 2 (fp32)
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const float nm = -m;
+    const int n_runs = (V + kRun - 1) / kRun;
+    FixedAcc acc;
+    acc.init();
+    if (VECTOR) {
+        const uint4 *src4 = reinterpret_cast<const uint4 *>(src);
+        const int nvec = V / N;
+        constexpr int UNROLL = 4 / PPR;             // four 16-byte loads in flight per thread
+        int g = threadIdx.x;
+        for (; g + (UNROLL - 1) * kSampleThreads < n_runs; g += UNROLL * kSampleThreads) {
+            uint4 v[UNROLL][PPR];
+            bool have[UNROLL][PPR];
+#pragma unroll
+            for (int k = 0; k < UNROLL; ++k)
+#pragma unroll
+                for (int h = 0; h < PPR; ++h) {
+                    const int i = (g + k * kSampleThreads) * PPR + h;
+                    have[k][h] = i < nvec;       // (fp32 with V % 8 == 4: the last run is half a run)
+                    if (have[k][h]) v[k][h] = ld_stream(src4 + i);
+                }
+#pragma unroll
+            for (int k = 0; k < UNROLL; ++k)
+#pragma unroll
+                for (int h = 0; h < PPR; ++h)
+                    if (have[k][h]) accumulate_fixed<T, true, CLAMP>(v[k][h], c, nm, acc);
+        }
+        for (; g < n_runs; g += kSampleThreads)
+#pragma unroll
+            for (int h = 0; h < PPR; ++h) {
+                const int i = g * PPR + h;
+                if (i < nvec) accumulate_fixed<T, true, CLAMP>(ld_stream(src4 + i), c, nm, acc);
+            }
+    } else {
+        for (int g = threadIdx.x; g < n_runs; g += kSampleThreads)
+            for (int q = 0; q < kRun; ++q) {
+                const int j = g * kRun + q;
+                if (j >= V) break;
+                float x = Pack<T>::load1(src + j);
+                x = (x != x) ? x : fmaxf(x, kNegBig);
+                const float t = fmaf(x, c, nm);
+                const float e = ex2(t);
+                acc.s0 += e;
+                acc.u0 = fmaf(e, t, acc.u0);
+            }
+    }
+    // ---- level 1: the class sums race with one uniform each; the row sums are merged on the way
+    const float W = acc.s0 + acc.s1;
+    float s = W, u = acc.u0 + acc.u1;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        s += __shfl_xor_sync(0xffffffffu, s, off);
+        u += __shfl_xor_sync(0xffffffffu, u, off);
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-        s = 0.f; u = 0.f;
-        best.init();
-        for (int w = 0; w < WARPS; ++w) {
-            s += sm.rs[w]; u += sm.ru[w];
-            Race o;
-            o.e = sm.re[w]; o.L = sm.rl[w]; o.j = sm.rj[w];
-            best.merge(o);
+    if (lane == 0) { sm.rs[warp] = s; sm.ru[warp] = u; }
+    uint32_t w[4];
+    philox4x32_10(kClassCounterBase + (threadIdx.x >> 2), row, a.off_lo, a.off_hi, a.k0, a.k1, w);
+    Race cls;
+    cls.e = W;
+    cls.L = log2_uniform(w[threadIdx.x & 3]);
+    cls.j = (int)threadIdx.x;
+    if (!(W > 0.f)) cls.init();                 // a class without weight (or with a NaN) never wins
+    cls = block_race(cls, sm);                  // (its barriers also publish rs / ru)
+    s = 0.f; u = 0.f;
+#pragma unroll
+    for (int k = 0; k < kSampleThreads / 32; ++k) { s += sm.rs[k]; u += sm.ru[k]; }
+    // ---- level 2: the members of the winning class race, one member per thread
+    Race best;
+    best.init();
+    if (cls.j != 0x7fffffff) {
+        const int c_star = cls.j;
+        for (int q = threadIdx.x;; q += kSampleThreads) {
+            const int run = c_star + (q / kRun) * kSampleThreads;
+            if (run >= n_runs) break;
+            const int j = run * kRun + (q % kRun);
+            if (j < V) {
+                float x = Pack<T>::load1(src + j);
+                x = (x != x) ? x : fmaxf(x, kNegBig);
+                const float e = ex2(fmaf(x, c, nm));
+                philox4x32_10((uint32_t)(j >> 2), row, a.off_lo, a.off_hi, a.k0, a.k1, w);
+                const uint32_t wj = (j & 2) ? ((j & 1) ? w[3] : w[2]) : ((j & 1) ? w[1] : w[0]);
+                if (e > 0.f) best.offer(e, log2_uniform(wj), j);
+            }
         }
     }
+    best = block_race(best, sm);
     s_out = s; u_out = u; best_out = best;
 }
 
-template <typename T, bool VECTOR, int THREADS>
-__global__ void __launch_bounds__(THREADS)
+template <typename T, bool VECTOR>
+__global__ void __launch_bounds__(kSampleThreads, 8)
 sample_kernel(const SampleArgs a)
 {
     constexpr int N = Pack<T>::N;
-    constexpr int WARPS = THREADS / 32;
+    constexpr int WARPS = kSampleThreads / 32;
     __shared__ SampleSmem sm;
     const int64_t row = blockIdx.x;
     const T *src = reinterpret_cast<const T *>(a.logits) + row * a.row_stride;
     const int V = a.V;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    PhiloxKeys keys;
-    keys.init(a.k0, a.k1);
 
     // First attempt with the maximum of the row's first pack as the reference of the exponentials (any
     // reference works for the race and the sums as long as nothing overflows): one pass over the row.
     float m = VECTOR ? row_reference<T>(src, a.c) : safe_reference(fmaxf(Pack<T>::load1(src), kNegBig), a.c);
     float s, u;
     Race best;
-    sums_and_race<T, VECTOR, THREADS>(src, V, a.c, m, (uint32_t)row, a, keys, sm, s, u, best);
-    if (threadIdx.x == 0) sm.redo = !(s < 1.0e37f) || !(fabsf(u) < 1.0e37f);
-    __syncthreads();
-    if (sm.redo) {
+    sums_and_race<T, VECTOR, false>(src, V, a.c, m, (uint32_t)row, a, sm, s, u, best);
+    if (!(s < 1.0e37f) || !(fabsf(u) < 1.0e37f)) {   // (s and u are the same in every thread)
         // a sum overflowed (an element lies more than ~2^127 above the reference) or the row holds a NaN or
         // +inf: take the exact maximum (NaN-blind; a NaN then shows up in the sums again) and repeat
         float mx = kNegBig;
         if (VECTOR) {
             const uint4 *src4 = reinterpret_cast<const uint4 *>(src);
             const int nvec = V / N;
-            for (int i = threadIdx.x; i < nvec; i += THREADS) {
+            for (int i = threadIdx.x; i < nvec; i += kSampleThreads) {
                 float x[N], xm;
                 Pack<T>::unpack(src4[i], x, xm);
                 mx = fmaxf(mx, xm);
             }
         } else {
-            for (int j = threadIdx.x; j < V; j += THREADS) mx = fmaxf(mx, fmaxf(Pack<T>::load1(src + j), kNegBig));
+            for (int j = threadIdx.x; j < V; j += kSampleThreads) mx = fmaxf(mx, fmaxf(Pack<T>::load1(src + j), kNegBig));
         }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
@@ -221,7 +264,8 @@ sample_kernel(const SampleArgs a)
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
         m = safe_reference(mx, a.c);
-        sums_and_race<T, VECTOR, THREADS>(src, V, a.c, m, (uint32_t)row, a, keys, sm, s, u, best);
+        __syncthreads();
+        sums_and_race<T, VECTOR, true>(src, V, a.c, m, (uint32_t)row, a, sm, s, u, best);
     }
     if (threadIdx.x == 0) {
         int tok = best.j;
@@ -277,16 +321,15 @@ extern "C" int ppo_sample_logprob_entropy(const void *logits, int dtype, int64_t
     a.lse = lse;
     a.status = workspace ? &ws_header(workspace)->status : nullptr;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    constexpr int THREADS = 256;
     const int n = dtype == PPO_F32 ? 4 : 8;
     const bool vec = aligned16(logits) && (row_stride * es) % 16 == 0 && V % n == 0;
     const unsigned grid = (unsigned)rows;
     if (dtype == PPO_F32) {
-        if (vec) sample_kernel<float, true, THREADS><<<grid, THREADS, 0, s>>>(a);
-        else sample_kernel<float, false, THREADS><<<grid, THREADS, 0, s>>>(a);
+        if (vec) sample_kernel<float, true><<<grid, kSampleThreads, 0, s>>>(a);
+        else sample_kernel<float, false><<<grid, kSampleThreads, 0, s>>>(a);
     } else {
-        if (vec) sample_kernel<__nv_bfloat16, true, THREADS><<<grid, THREADS, 0, s>>>(a);
-        else sample_kernel<__nv_bfloat16, false, THREADS><<<grid, THREADS, 0, s>>>(a);
+        if (vec) sample_kernel<__nv_bfloat16, true><<<grid, kSampleThreads, 0, s>>>(a);
+        else sample_kernel<__nv_bfloat16, false><<<grid, kSampleThreads, 0, s>>>(a);
     }
     return launch_status();
 }
