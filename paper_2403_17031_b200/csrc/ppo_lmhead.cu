@@ -26,9 +26,7 @@
 //
 // Every wait is bounded; a wait that runs out sets PPO_DEV_TIMEOUT and the block carries on with the
 // same control flow, so it still reaches the end, frees its tensor memory and returns.
-#include <cuda.h>
-
-#include "ppo_common.cuh"
+#include "ppo_tcgen05.cuh"
 
 namespace ppo {
 
@@ -50,8 +48,6 @@ template <int MT> struct LmShape {
 };
 constexpr int kTilesPerChunk = 6;                       // vocabulary tiles per work unit
 constexpr int kRowGroup = 37;                           // row tiles that sweep the vocabulary together
-constexpr int kTmemCols = 512;
-constexpr uint32_t kLmWaitTries = 1u << 19;         // x up to ~2 us per try
 constexpr uint32_t kAbsentBits = 0xffffffffu;           // "this chunk does not hold the sampled token"
 
 struct LmSmem {
@@ -59,83 +55,8 @@ struct LmSmem {
     uint32_t tmem_base;
 };
 
-__device__ __forceinline__ uint32_t lm_smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ bool lm_wait(unsigned long long *bar, uint32_t parity, int *status)
-{
-    const uint32_t addr = lm_smem_addr(bar);
-    for (uint32_t it = 0; it < kLmWaitTries; ++it) {
-        uint32_t ok;
-        asm volatile(
-            "{\n"
-            ".reg .pred p;\n"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
-            "selp.u32 %0, 1, 0, p;\n"
-            "}\n"
-            : "=r"(ok)
-            : "r"(addr), "r"(parity), "r"(2000u)
-            : "memory");
-        if (ok) return true;
-    }
-    atomicOr(status, PPO_DEV_TIMEOUT);
-    return false;
-}
-
-__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int x, int y, unsigned long long *bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(lm_smem_addr(dst)), "l"(map), "r"(x), "r"(y), "r"(lm_smem_addr(bar))
-        : "memory");
-}
-
-// shared-memory matrix descriptor: 128-byte swizzle, version 1; offsets in 16-byte units
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3fff);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3fff) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fff) << 32;
-    d |= (uint64_t)1 << 46;    // descriptor version (sm_100)
-    d |= (uint64_t)2 << 61;    // SWIZZLE_128B
-    return d;
-}
-
 // instruction descriptor: D fp32, A and B bf16, A K-major, B MN-major, M = 128, N = 256
-constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
-                                ((uint32_t)(kBlockN >> 3) << 17) | ((uint32_t)(kBlockM >> 4) << 24);
-
-__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n"
-        "}\n"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(kInstrDesc), "r"(accumulate), "r"(0u)
-        : "memory");
-}
-
-__device__ __forceinline__ void umma_commit(unsigned long long *bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(lm_smem_addr(bar))
-                 : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-}
+constexpr uint32_t kInstrDesc = tc::instr_desc(false, true, kBlockM, kBlockN);
 
 struct LmUnit {
     int m_tile, chunk;
@@ -177,7 +98,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__
     extern __shared__ __align__(1024) unsigned char lm_smem_raw[];
     __shared__ LmSmem sm;
     // the ring must start on a 1024-byte boundary (swizzle atoms)
-    unsigned char *ring = lm_smem_raw + ((1024u - (lm_smem_addr(lm_smem_raw) & 1023u)) & 1023u);
+    unsigned char *ring = lm_smem_raw + ((1024u - (tc::saddr(lm_smem_raw) & 1023u)) & 1023u);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int k_blocks = a.K / kBlockK;
     // every role walks the same unit list, derived from the same row count
@@ -190,21 +111,17 @@ lmhead_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(lm_smem_addr(&sm.full[s])) : "memory");
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(lm_smem_addr(&sm.empty[s])) : "memory");
+            tc::barrier_init(&sm.full[s], 1);
+            tc::barrier_init(&sm.empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) {
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(lm_smem_addr(&sm.tmem_full[b])) : "memory");
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(lm_smem_addr(&sm.tmem_empty[b])), "r"(4 * MT)
-                         : "memory");
+            tc::barrier_init(&sm.tmem_full[b], 1);
+            tc::barrier_init(&sm.tmem_empty[b], 4 * MT);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {   // one warp allocates all 512 columns of tensor memory
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(lm_smem_addr(&sm.tmem_base)),
-                     "r"((uint32_t)kTmemCols)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        tc::tmem_alloc_all(&sm.tmem_base);
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -221,18 +138,16 @@ lmhead_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__
                 for (int t = t0; t < t1; ++t) {
                     for (int kb = 0; kb < k_blocks; ++kb, ++it) {
                         const int s = it % kStages;
-                        if (it >= kStages) lm_wait(&sm.empty[s], ((it / kStages) - 1) & 1, a.status);
+                        if (it >= kStages) tc::wait(&sm.empty[s], ((it / kStages) - 1) & 1, a.status);
                         unsigned char *stage = ring + (size_t)s * kStageBytes;
-                        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(lm_smem_addr(&sm.full[s])),
-                                     "r"((uint32_t)kStageBytes)
-                                     : "memory");
+                        tc::barrier_expect_tx(&sm.full[s], (uint32_t)kStageBytes);
 #pragma unroll
                         for (int j = 0; j < MT; ++j)   // (a tile past the last row is filled with zeros)
-                            tma_load_2d(stage + j * kABytes, &map_h, kb * kBlockK, (un.m_tile * MT + j) * kBlockM,
+                            tc::tma_load_2d(stage + j * kABytes, &map_h, kb * kBlockK, (un.m_tile * MT + j) * kBlockM,
                                         &sm.full[s]);
 #pragma unroll
                         for (int j = 0; j < kBlockN / 64; ++j)
-                            tma_load_2d(stage + MT * kABytes + j * kBBoxBytes, &map_w, t * kBlockN + j * 64,
+                            tc::tma_load_2d(stage + MT * kABytes + j * kBBoxBytes, &map_w, t * kBlockN + j * 64,
                                         kb * kBlockK, &sm.full[s]);
                     }
                 }
@@ -248,30 +163,30 @@ lmhead_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__
                 const int t0 = un.chunk * kTilesPerChunk, t1 = min(t0 + kTilesPerChunk, a.n_tiles);
                 for (int t = t0; t < t1; ++t, ++tc) {
                     const uint32_t buf = tc % kSets;
-                    if (tc >= (uint32_t)kSets) lm_wait(&sm.tmem_empty[buf], ((tc / kSets) - 1) & 1, a.status);
+                    if (tc >= (uint32_t)kSets) tc::wait(&sm.tmem_empty[buf], ((tc / kSets) - 1) & 1, a.status);
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t tmem_d = tmem_base + buf * (MT * kBlockN);
                     for (int kb = 0; kb < k_blocks; ++kb, ++it) {
                         const int s = it % kStages;
-                        lm_wait(&sm.full[s], (it / kStages) & 1, a.status);
+                        tc::wait(&sm.full[s], (it / kStages) & 1, a.status);
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                        const uint32_t a_addr = lm_smem_addr(ring + (size_t)s * kStageBytes);
+                        const uint32_t a_addr = tc::saddr(ring + (size_t)s * kStageBytes);
                         const uint32_t b_addr = a_addr + MT * kABytes;
 #pragma unroll
                         for (int kk = 0; kk < kBlockK / 16; ++kk) {
                             // B: vocabulary-major; 64-column boxes 8192 B apart, 8 K-rows 1024 B apart;
                             //    16 K-rows = 2048 bytes further
-                            const uint64_t bd = smem_desc(b_addr + kk * 2048, kBBoxBytes, 1024);
+                            const uint64_t bd = tc::smem_desc(b_addr + kk * 2048, kBBoxBytes, 1024);
 #pragma unroll
                             for (int j = 0; j < MT; ++j) {
                                 // A: K-major, 8-row groups 1024 B apart; 16 K-elements = 32 bytes further
-                                const uint64_t ad = smem_desc(a_addr + j * kABytes + kk * 32, 16, 1024);
-                                umma(tmem_d + j * kBlockN, ad, bd, (kb | kk) ? 1u : 0u);
+                                const uint64_t ad = tc::smem_desc(a_addr + j * kABytes + kk * 32, 16, 1024);
+                                tc::mma(tmem_d + j * kBlockN, ad, bd, kInstrDesc, (kb | kk) ? 1u : 0u);
                             }
                         }
-                        umma_commit(&sm.empty[s]);            // ring slot is free once these MMAs have read it
+                        tc::commit(&sm.empty[s]);            // ring slot is free once these MMAs have read it
                     }
-                    umma_commit(&sm.tmem_full[buf]);          // accumulator complete
+                    tc::commit(&sm.tmem_full[buf]);          // accumulator complete
                 }
             }
         }
@@ -293,22 +208,20 @@ lmhead_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__
             uint32_t xtok_bits = kAbsentBits;
             for (int t = t0; t < t1; ++t, ++tc) {
                 const uint32_t buf = tc % kSets;
-                lm_wait(&sm.tmem_full[buf], (tc / kSets) & 1, a.status);
+                tc::wait(&sm.tmem_full[buf], (tc / kSets) & 1, a.status);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t taddr = tmem_base + buf * (MT * kBlockN) + acc * kBlockN + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
                 for (int cc = 0; cc < kBlockN / 32; ++cc) {
                     uint32_t r[32];
                     __syncwarp();                            // the aligned tensor-memory load needs a converged warp
-                    tmem_ld32(taddr + cc * 32, r);
+                    tc::tmem_ld32(taddr + cc * 32, r);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                     if (cc == kBlockN / 32 - 1) {
                         // all of this warp's reads of the accumulator are done: hand it back
                         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                         __syncwarp();
-                        if (lane == 0)
-                            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(lm_smem_addr(&sm.tmem_empty[buf]))
-                                         : "memory");
+                        if (lane == 0) tc::barrier_arrive(&sm.tmem_empty[buf]);
                     }
                     const int col0 = t * kBlockN + cc * 32;
                     if (col0 >= a.V) continue;
@@ -369,8 +282,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols)
-                     : "memory");
+        tc::tmem_free_all(tmem_base);
     }
 }
 
@@ -437,37 +349,7 @@ lmhead_finalize_kernel(const float4 *__restrict__ partials, int M, int V, int n_
 }
 
 // ---------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
-// 2-D bf16 tensor [outer, inner] (inner contiguous), box [box_outer, 64], 128-byte swizzle
-static int make_map(CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint32_t box_outer)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return (int)cudaErrorNotSupported;
-    const cuuint64_t dims[2] = {inner, outer};
-    const cuuint64_t strides[1] = {inner * 2};
-    const cuuint32_t box[2] = {64, box_outer};
-    const cuuint32_t elem[2] = {1, 1};
-    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, elem,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? PPO_OK : (int)cudaErrorInvalidValue;
-}
+using tc::make_map;
 
 static size_t lm_partials_bytes(int m_tiles, int n_chunks)
 {

@@ -19,9 +19,7 @@
 // (thread r owns row r of the tile, 32 columns per tcgen05.ld). Work unit = one 128 x 256 output tile
 // with its whole contraction; units are ordered in groups of gm x gn tiles that run at the same time
 // and share their operand panels through L2. Every wait is bounded (PPO_DEV_TIMEOUT on expiry).
-#include <cuda.h>
-
-#include "ppo_common.cuh"
+#include "ppo_tcgen05.cuh"
 
 namespace ppo {
 namespace bwd {
@@ -33,94 +31,13 @@ constexpr int kBoxBytes = 64 * kBlockK * 2;             // 8 KB: one 64 x 64 box
 constexpr int kBBytes = kBlockN * kBlockK * 2;          // 32 KB
 constexpr int kStageBytes = kABytes + kBBytes;          // 48 KB
 constexpr int kThreads = 192;
-constexpr int kTmemCols = 512;
-constexpr uint32_t kWaitTries = 1u << 19;               // x up to ~2 us per try
 
 struct Smem {
     unsigned long long full[kStages], empty[kStages], tmem_full[2], tmem_empty[2];
     uint32_t tmem_base;
 };
 
-__device__ __forceinline__ uint32_t saddr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ bool wait(unsigned long long *bar, uint32_t parity, int *status)
-{
-    const uint32_t addr = saddr(bar);
-    for (uint32_t it = 0; it < kWaitTries; ++it) {
-        uint32_t ok;
-        asm volatile(
-            "{\n"
-            ".reg .pred p;\n"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
-            "selp.u32 %0, 1, 0, p;\n"
-            "}\n"
-            : "=r"(ok)
-            : "r"(addr), "r"(parity), "r"(2000u)
-            : "memory");
-        if (ok) return true;
-    }
-    atomicOr(status, PPO_DEV_TIMEOUT);
-    return false;
-}
-
-__device__ __forceinline__ void tma_load(void *dst, const CUtensorMap *map, int x, int y, unsigned long long *bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(saddr(dst)), "l"(map), "r"(x), "r"(y), "r"(saddr(bar))
-        : "memory");
-}
-
-// shared-memory matrix descriptor: 128-byte swizzle, version 1; offsets in 16-byte units
-__device__ __forceinline__ uint64_t desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3fff);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3fff) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fff) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
-}
-
-// instruction descriptor: D fp32, A and B bf16, M = 128, N = 256; bits 15 / 16 = A / B is MN-major
-template <bool A_MN, bool B_MN>
-__device__ __forceinline__ constexpr uint32_t instr_desc()
-{
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16) |
-           ((uint32_t)(kBlockN >> 3) << 17) | ((uint32_t)(kBlockM >> 4) << 24);
-}
-
-__device__ __forceinline__ void mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n"
-        "}\n"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u)
-        : "memory");
-}
-
-__device__ __forceinline__ void commit(unsigned long long *bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(saddr(bar)) : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-}
+using namespace tc;
 
 struct Unit {
     int m_tile, n_tile;
@@ -199,20 +116,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(saddr(&sm.full[s])) : "memory");
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(saddr(&sm.empty[s])) : "memory");
+            barrier_init(&sm.full[s], 1);
+            barrier_init(&sm.empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) {
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(saddr(&sm.tmem_full[b])) : "memory");
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 4;" ::"r"(saddr(&sm.tmem_empty[b])) : "memory");
+            barrier_init(&sm.tmem_full[b], 1);
+            barrier_init(&sm.tmem_empty[b], 4);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(saddr(&sm.tmem_base)),
-                     "r"((uint32_t)kTmemCols)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        tmem_alloc_all(&sm.tmem_base);
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -230,22 +144,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     const int s = it % kStages;
                     if (it >= kStages) wait(&sm.empty[s], ((it / kStages) - 1) & 1, a.status);
                     unsigned char *stage = ring + (size_t)s * kStageBytes;
-                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(saddr(&sm.full[s])),
-                                 "r"((uint32_t)kStageBytes)
-                                 : "memory");
+                    barrier_expect_tx(&sm.full[s], (uint32_t)kStageBytes);
                     if (A_MN) {   // A stored [Kc, Mdim]: boxes of 64 (m) x 64 (k)
 #pragma unroll
                         for (int j = 0; j < kBlockM / 64; ++j)
-                            tma_load(stage + j * kBoxBytes, &map_a, m0 + j * 64, kb * kBlockK, &sm.full[s]);
+                            tma_load_2d(stage + j * kBoxBytes, &map_a, m0 + j * 64, kb * kBlockK, &sm.full[s]);
                     } else {      // A stored [Mdim, Kc]: one box of 64 (k) x 128 (m)
-                        tma_load(stage, &map_a, kb * kBlockK, m0, &sm.full[s]);
+                        tma_load_2d(stage, &map_a, kb * kBlockK, m0, &sm.full[s]);
                     }
                     if (B_MN) {   // B stored [Kc, Ndim]: boxes of 64 (n) x 64 (k)
 #pragma unroll
                         for (int j = 0; j < kBlockN / 64; ++j)
-                            tma_load(stage + kABytes + j * kBoxBytes, &map_b, n0 + j * 64, kb * kBlockK, &sm.full[s]);
+                            tma_load_2d(stage + kABytes + j * kBoxBytes, &map_b, n0 + j * 64, kb * kBlockK, &sm.full[s]);
                     } else {      // B stored [Ndim, Kc]: one box of 64 (k) x 256 (n)
-                        tma_load(stage + kABytes, &map_b, kb * kBlockK, n0, &sm.full[s]);
+                        tma_load_2d(stage + kABytes, &map_b, kb * kBlockK, n0, &sm.full[s]);
                     }
                 }
             }
@@ -254,7 +166,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = instr_desc<A_MN, B_MN>();
+            constexpr uint32_t idesc = instr_desc(A_MN, B_MN, kBlockM, kBlockN);
             uint32_t it = 0, tc = 0;
             for (int u = blockIdx.x; u < n_units; u += gridDim.x, ++tc) {
                 const uint32_t buf = tc & 1;
@@ -272,8 +184,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                         // K-major operand: 8-row groups 1024 B apart; 16 contraction elements = 32 bytes further.
                         // MN-major operand: 64-wide boxes 8192 B apart, 8 contraction rows 1024 B apart;
                         // 16 contraction rows = 2048 bytes further.
-                        const uint64_t ad = A_MN ? desc(a_addr + kk * 2048, kBoxBytes, 1024) : desc(a_addr + kk * 32, 16, 1024);
-                        const uint64_t bd = B_MN ? desc(b_addr + kk * 2048, kBoxBytes, 1024) : desc(b_addr + kk * 32, 16, 1024);
+                        const uint64_t ad = A_MN ? smem_desc(a_addr + kk * 2048, kBoxBytes, 1024) : smem_desc(a_addr + kk * 32, 16, 1024);
+                        const uint64_t bd = B_MN ? smem_desc(b_addr + kk * 2048, kBoxBytes, 1024) : smem_desc(b_addr + kk * 32, 16, 1024);
                         mma(tmem_d, ad, bd, idesc, (kb | kk) ? 1u : 0u);
                     }
                     commit(&sm.empty[s]);
@@ -316,8 +228,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 if (cc == kBlockN / 32 - 1) {
                     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                     __syncwarp();
-                    if (lane == 0)
-                        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(saddr(&sm.tmem_empty[buf])) : "memory");
+                    if (lane == 0) barrier_arrive(&sm.tmem_empty[buf]);
                 }
                 const int col0 = un.n_tile * kBlockN + cc * 32;
                 if (!row_ok || col0 >= a.Ndim) continue;
@@ -365,44 +276,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols)
-                     : "memory");
+        tmem_free_all(tmem_base);
     }
 }
 
 // ---------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
-// 2-D bf16 tensor [outer, inner] (inner contiguous), box [box_outer, 64], 128-byte swizzle, zero fill outside
-static int make_map(CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint32_t box_outer)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return (int)cudaErrorNotSupported;
-    const cuuint64_t dims[2] = {inner, outer};
-    const cuuint64_t strides[1] = {inner * 2};
-    const cuuint32_t box[2] = {64, box_outer};
-    const cuuint32_t elem[2] = {1, 1};
-    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, elem,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? PPO_OK : (int)cudaErrorInvalidValue;
-}
-
 // zero rows [*n, next multiple of 128) of a [M, row16 * 16 bytes] matrix (at most 127 rows, none beyond M)
 __global__ void __launch_bounds__(256)
 zero_tail_rows_kernel(uint4 *__restrict__ base, int row16, const int *__restrict__ n, int M)
