@@ -56,15 +56,18 @@ def _loss_kernel_hash():
     return h.hexdigest()
 
 
-def _ncu_traffic(key: str, algorithmic_bytes: float):
-    """DRAM bytes (read + write) per launch from the stored capture of workload `key`, scaled by the algorithmic
-    bytes when the capture was taken on a cut of the batch; None without a capture of the current kernel."""
+def _ncu_traffic(key: str, read_bytes: float, write_bytes: float):
+    """DRAM bytes (read + write) of one launch with the given algorithmic read / write bytes, from the stored capture
+    of workload `key` (taken on a cut of the batch): reads scale with the rows read, writes with the rows written, and
+    the tail of the write stream that was still in L2 when the captured launch ended is the same at any size. None
+    without a capture of the current kernel."""
     try:
         d = json.load(open(_TRAFFIC_FILE))
         e = d["captures"][key]
         if d["sources_sha256"] != _loss_kernel_hash():
             return None
-        return (e["dram_bytes_read"] + e["dram_bytes_write"]) * algorithmic_bytes / e["algorithmic_bytes"]
+        in_l2 = e["algorithmic_bytes_write"] - e["dram_bytes_write"]
+        return e["dram_bytes_read"] * read_bytes / e["algorithmic_bytes_read"] + max(write_bytes - in_l2, 0.0)
     except Exception:
         return None
 
@@ -373,7 +376,7 @@ def measure_ppo(cfg, args, D, K, warmup, target_s, full: bool):
     loss_gbs = loss_bytes / (next_ms * 1e-3) / 1e9
     # the step reads the logits of the real rows only (policy, reference, loss) and writes every gradient row
     path_bytes = 2 * n_real * V * esize + loss_bytes
-    traffic = _ncu_traffic("config%d" % cfg.index, loss_bytes)
+    traffic = _ncu_traffic("config%d" % cfg.index, n_real * V * esize, B * T * V * esize)
     roofline = {"bound": "hbm", "kernel": "row_engine_kernel (ppo_loss_fwd_bwd)", "achieved": loss_gbs,
                 "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": loss_gbs / peak,
                 "frac_of_8tbs": loss_gbs / 8000.0, "traffic": traffic,
@@ -791,7 +794,7 @@ def run_dpo(args):
                        "device_status": st.device_status()},
             "roofline": {"bound": "hbm", "kernel": "row_engine_kernel (ppo_logprob_bwd)", "achieved": bwd_gbs,
                          "peak": peak, "peak_kind": kind, "unit": "GB/s", "frac": bwd_gbs / peak,
-                         "frac_of_8tbs": bwd_gbs / 8000.0, "traffic": _ncu_traffic("config5", bwd_bytes),
+                         "frac_of_8tbs": bwd_gbs / 8000.0, "traffic": _ncu_traffic("config5", n_real * V * es, rows * V * es),
                          "algorithmic_bytes": bwd_bytes,
                          "timing": "CUDA events around the ppo_logprob_bwd call (prologue + row engine launches), "
                                    "right after the timed region"},
