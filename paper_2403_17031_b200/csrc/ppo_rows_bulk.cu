@@ -21,9 +21,11 @@
 //   * step 6 may be launched while the kernel that produces its row order and advantages is still
 //     running (programmatic dependent launch): it then polls two flags of the workspace header.
 //
-// Every wait is bounded: when it runs out the block records PPO_DEV_TIMEOUT in the status word
-// and carries on with the same control flow (so no barrier is left short), which makes the
-// outputs invalid but lets the kernel end.
+// Every wait is bounded: when it runs out the block records PPO_DEV_TIMEOUT in the status word. A block
+// that never learns the row order (step 6 launched early) returns before anything is indexed through it,
+// and block 0 writes NaN loss scalars; after any other run-out the block carries on with the same control
+// flow (so no barrier is left short), which makes the outputs invalid but lets the kernel end, and the
+// producer makes sure that none of its copies into shared memory is still in flight when the block retires.
 #include "ppo_rows.cuh"
 
 namespace ppo {
