@@ -486,11 +486,14 @@ def _lmhead_oracle_baseline(cfg, b, seconds=10.0):
     to_np = lambda t: t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
     H, W = to_np(b["H"]), to_np(b["W"])
     tok = b["responses"].reshape(-1).cpu().numpy()
-    n = max(O.num_threads(), 8)
-    sel = np.arange(0, H.shape[0], max(1, H.shape[0] // n))[:n].astype(np.int64)
-    t0 = time.perf_counter()
-    O.lmhead_logprob_entropy(H, W, tok, np.float32(cfg.hyper.temperature), sel_rows=sel)
-    dt = time.perf_counter() - t0
+    def timed(n):
+        sel = np.arange(0, H.shape[0], max(1, H.shape[0] // n))[:n].astype(np.int64)
+        t0 = time.perf_counter()
+        O.lmhead_logprob_entropy(H, W, tok, np.float32(cfg.hyper.temperature), sel_rows=sel)
+        return sel, time.perf_counter() - t0
+    sel, dt = timed(max(O.num_threads(), 8))                       # size probe
+    n = int(min(H.shape[0], max(len(sel), len(sel) * seconds / max(dt, 1e-3))))
+    sel, dt = timed(n)
     # one step of the config needs two such passes per real row (policy and reference unembedding)
     return {"value": len(sel) / dt / 2.0, "unit": "tokens/s", "cores": O.num_threads(), "kind": "oracle",
             "sample": "%d rows of H x W [%d, %d] in fp64 for one unembedding, %.1f s; halved for the two unembeddings of a "
@@ -585,24 +588,26 @@ def measure_lmhead(cfg, args, D, K, warmup, target_s, full: bool):
            "clocks": clk.summary(), "e2e": None, "cpu_baseline": None, "cpu_baseline_1thread": None,
            "gpu_launches": (13 + (6 if bwd_out is not None else 0)) * K * len(blocks)}
     if full and not args.no_e2e:
-        # end to end through the same C-ABI calls with host buffers: H, both unembeddings, tokens, scores and values
+        # end to end through ppo_lmhead_step_host: H (its real rows), both unembeddings, tokens, scores and values
         # start in pinned host memory and are copied in every step; the loss scalars and the [B,T] results come back
         names = ["H", "W", "W_ref", "responses", "scores", "values", "values_new"]
         host = {k: b[k].cpu().pin_memory() for k in names}
-        host_old = old.cpu().pin_memory()
-        outs = [loss_out["losses"], loss_out["dlogprob"], loss_out["dvalues"], o["aw"], o["ret"], o["lp"], o["rlp"]]
-        host_res = [torch.empty_like(t, device="cpu").pin_memory() for t in outs]
-        h2d = sum(v.numel() * v.element_size() for v in host.values()) + host_old.numel() * 4
-        d2h = sum(v.numel() * v.element_size() for v in host_res)
+        host["old_logprob"] = old.cpu().pin_memory()
+        dev_out = {"responses_out": o["ro"], "eos_index": o["ei"], "seq_len": o["sl"], "mask": o["mask"], "scores_out": o["so"],
+                   "logprob": o["lp"], "entropy": o["ent"], "lse": o["lse"], "ref_logprob": o["rlp"], "kl": o["kl"],
+                   "rewards": o["rew"], "advantages": o["adv"], "returns": o["ret"], "advantages_whitened": o["aw"],
+                   "whiten_stats": o["st"], "losses": loss_out["losses"], "dlogprob": loss_out["dlogprob"],
+                   "dvalues": loss_out["dvalues"]}
+        res_names = ["losses", "dlogprob", "dvalues", "advantages_whitened", "returns", "logprob", "ref_logprob"]
+        host_res = {k: torch.empty_like(dev_out[k], device="cpu").pin_memory() for k in res_names}
+        h2d = sum(v.numel() * v.element_size() for k, v in host.items() if k != "H") + n_real * Kd * 2
+        d2h = sum(v.numel() * v.element_size() for v in host_res.values())
+        host_io = binding.LMHeadStepIO.from_tensors({**host, **host_res}, cuda=False)
+        dev_io = binding.LMHeadStepIO.from_tensors({**{k: b[k] for k in names}, "old_logprob": old, **dev_out,
+                                                    "workspace": ws}, cuda=True)
 
         def e2e_step():
-            for k in names:
-                b[k].copy_(host[k], non_blocking=True)
-            old.copy_(host_old, non_blocking=True)
-            step(old)
-            for t, ht in zip(outs, host_res):
-                ht.copy_(t, non_blocking=True)
-            torch.cuda.current_stream().synchronize()
+            binding.lmhead_step_host(host_io, dev_io, B, T, Kd, V, p)
         Ke = max(3, min(K, args.e2e_steps))
         e2e_step()
         D.barrier()
@@ -615,8 +620,8 @@ def measure_lmhead(cfg, args, D, K, warmup, target_s, full: bool):
         e_ms = D.max_float(a.elapsed_time(c))
         res["e2e"] = {"value": n_real * world / (e_ms / Ke * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                       "d2h_bytes_per_step": d2h, "steps": Ke, "ms_per_step": e_ms / Ke,
-                      "call": "pinned host buffers copied in on the stream, the config-4 chain of C-ABI calls, results "
-                              "copied back, stream synchronised"}
+                      "call": "ppo_lmhead_step_host (pinned host buffers in: the real rows of H, both unembeddings, the "
+                              "[B,T] inputs; losses and the [B,T] results out)"}
     if full and D.rank == 0 and world == 1 and not args.no_cpu_baseline:
         res["cpu_baseline"] = _lmhead_oracle_baseline(cfg, b)
     del b, ws

@@ -469,6 +469,41 @@ int ppo_step(const ppo_step_io *io /* host */, int dtype, int32_t B, int32_t T, 
 int ppo_step_host(const ppo_step_io *host /* host */, const ppo_step_io *dev /* host */, int dtype,
                   int32_t B, int32_t T, int64_t V, const ppo_params *p /* host */, void *stream);
 
+/*
+ * The config with the fused LM head as one call: the logits are never materialised, so the path is
+ * steps 2 (EOS trick), 1 through ppo_lmhead_logprob_entropy for the policy unembedding W and for the frozen
+ * SFT reference's W_ref (both with the mask of step 2: padding rows are taken out of the GEMMs), 3, 4, 5 and
+ * step 6 at log-prob level (ppo_loss_from_logprob).  Same citations as the individual calls.
+ *   inputs   H [B*T, K] bf16 hidden states of the response positions; W, W_ref [K, V] bf16;
+ *            responses [B,T] i32; scores [B]; values, values_new [B,T];
+ *            old_logprob [B,T] or NULL (= the log-probs this call computes: first PPO epoch, ratio 1)
+ *   outputs  responses_out, eos_index, seq_len, mask, scores_out; logprob, entropy, lse, ref_logprob (0 at
+ *            padding positions); kl, rewards; advantages, returns; advantages_whitened, whiten_stats[3];
+ *            losses[8], dlogprob, dvalues; workspace (device only) of at least
+ *            max(ppo_lmhead_workspace_bytes(B*T, K, V), ppo_workspace_bytes(B, T, V)) bytes
+ * ppo_lmhead_step: `io` is a host struct of DEVICE pointers; everything is enqueued on `stream`, nothing
+ * synchronises.  K a multiple of 64, V a multiple of 8 (PPO_ERR_UNSUPPORTED otherwise).
+ * ppo_lmhead_step_host: `host` holds HOST pointers (pinned memory makes the copies asynchronous), `dev` the
+ * device staging and output buffers.  Copies the inputs host -> device (of H only the rows the GEMMs read:
+ * each response's positions up to its first EOS, found from host->responses), runs ppo_lmhead_step on `dev`,
+ * copies back each output whose pointer in `host` is not NULL and waits for the stream.
+ */
+typedef struct ppo_lmhead_step_io {
+    const void *H, *W, *W_ref;
+    const int32_t *responses;
+    const float *scores, *values, *values_new, *old_logprob;
+    int32_t *responses_out, *eos_index, *seq_len;
+    uint8_t *mask;
+    float *scores_out, *logprob, *entropy, *lse, *ref_logprob, *kl, *rewards, *advantages, *returns,
+        *advantages_whitened, *whiten_stats, *losses, *dlogprob, *dvalues;
+    void *workspace;
+} ppo_lmhead_step_io;
+
+int ppo_lmhead_step(const ppo_lmhead_step_io *io /* host */, int32_t B, int32_t T, int64_t K, int64_t V,
+                    const ppo_params *p /* host */, void *stream);
+int ppo_lmhead_step_host(const ppo_lmhead_step_io *host /* host */, const ppo_lmhead_step_io *dev /* host */,
+                         int32_t B, int32_t T, int64_t K, int64_t V, const ppo_params *p /* host */, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

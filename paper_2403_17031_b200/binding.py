@@ -60,6 +60,16 @@ class PPOStepIO(C.Structure):
         return io
 
 
+class LMHeadStepIO(C.Structure):
+    """Mirror of ppo_lmhead_step_io (all pointers in one memory space)."""
+    _in = ("H", "W", "W_ref", "responses", "scores", "values", "values_new", "old_logprob")
+    _out = ("responses_out", "eos_index", "seq_len", "mask", "scores_out", "logprob", "entropy", "lse", "ref_logprob",
+            "kl", "rewards", "advantages", "returns", "advantages_whitened", "whiten_stats", "losses", "dlogprob",
+            "dvalues", "workspace")
+    _fields_ = [(n, C.c_void_p) for n in _in + _out]
+    from_tensors = classmethod(PPOStepIO.from_tensors.__func__)
+
+
 _lib = None
 
 _SIGS = {
@@ -95,6 +105,10 @@ _SIGS = {
                            C.c_void_p]),
     "ppo_step_host": (C.c_int, [C.POINTER(PPOStepIO), C.POINTER(PPOStepIO), C.c_int, C.c_int32, C.c_int32, C.c_int64,
                                 C.POINTER(PPOParams), C.c_void_p]),
+    "ppo_lmhead_step": (C.c_int, [C.POINTER(LMHeadStepIO), C.c_int32, C.c_int32, C.c_int64, C.c_int64,
+                                  C.POINTER(PPOParams), C.c_void_p]),
+    "ppo_lmhead_step_host": (C.c_int, [C.POINTER(LMHeadStepIO), C.POINTER(LMHeadStepIO), C.c_int32, C.c_int32,
+                                       C.c_int64, C.c_int64, C.POINTER(PPOParams), C.c_void_p]),
     "ppo_logprob_entropy_pair": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p,
                                            C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p]),
@@ -365,6 +379,17 @@ def step_host(host: PPOStepIO, dev: PPOStepIO, dtype: torch.dtype, B: int, T: in
     """Host buffers in, host buffers out: copies, the whole path, copies back, stream synchronised."""
     code = PPO_F32 if dtype == torch.float32 else PPO_BF16
     _check("ppo_step_host", lib().ppo_step_host(C.byref(host), C.byref(dev), code, B, T, V, C.byref(params), _stream()))
+
+
+def lmhead_step(io: LMHeadStepIO, B: int, T: int, K: int, V: int, params: PPOParams) -> None:
+    """The fused-LM-head config in one C call on device buffers (asynchronous on the current stream)."""
+    _check("ppo_lmhead_step", lib().ppo_lmhead_step(C.byref(io), B, T, K, V, C.byref(params), _stream()))
+
+
+def lmhead_step_host(host: LMHeadStepIO, dev: LMHeadStepIO, B: int, T: int, K: int, V: int, params: PPOParams) -> None:
+    """Host buffers in, host buffers out: copies, the fused-LM-head path, copies back, stream synchronised."""
+    _check("ppo_lmhead_step_host", lib().ppo_lmhead_step_host(C.byref(host), C.byref(dev), B, T, K, V, C.byref(params),
+                                                               _stream()))
 
 
 STATIC_MAX_TOKENS = 32768

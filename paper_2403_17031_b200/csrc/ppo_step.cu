@@ -204,3 +204,78 @@ extern "C" int ppo_step_host(const ppo_step_io *host, const ppo_step_io *dev, in
     PPO_RETURN_IF_CUDA(cudaStreamSynchronize(s));
     return PPO_OK;
 }
+
+
+// ---------------------------------------------------------------- the fused-LM-head config as one call
+extern "C" int ppo_lmhead_step(const ppo_lmhead_step_io *io, int32_t B, int32_t T, int64_t K, int64_t V,
+                               const ppo_params *p, void *stream)
+{
+    if (!io || !p) return PPO_ERR_NULL;
+    if (B <= 0 || T <= 0 || K <= 0 || V <= 0) return PPO_ERR_SHAPE;
+    if (!io->H || !io->W || !io->W_ref || !io->responses || !io->scores || !io->values || !io->values_new)
+        return PPO_ERR_NULL;
+    if (!io->responses_out || !io->eos_index || !io->seq_len || !io->mask || !io->scores_out || !io->logprob ||
+        !io->entropy || !io->ref_logprob || !io->kl || !io->rewards || !io->advantages || !io->returns ||
+        !io->advantages_whitened || !io->losses || !io->dvalues || !io->workspace)
+        return PPO_ERR_NULL;
+    const int64_t M = (int64_t)B * T;
+    PPO_TRY(ppo_truncate_and_score(io->responses, B, T, p->eos_id, p->pad_id, io->scores, p->no_eos_score,
+                                   io->responses_out, io->eos_index, io->seq_len, io->mask, io->scores_out, stream));
+    PPO_TRY(ppo_lmhead_logprob_entropy(io->H, io->W, M, K, V, io->responses, io->mask, p->temperature, io->logprob,
+                                       io->entropy, io->lse, io->workspace, stream));
+    PPO_TRY(ppo_lmhead_logprob_entropy(io->H, io->W_ref, M, K, V, io->responses, io->mask, p->temperature,
+                                       io->ref_logprob, nullptr, nullptr, io->workspace, stream));
+    PPO_TRY(ppo_kl_rewards(io->logprob, io->ref_logprob, io->mask, io->seq_len, io->scores_out, B, T, p->kl_coef,
+                           io->kl, io->rewards, stream));
+    if (p->whiten_rewards)   // optional reward whitening: mean kept, in place, before GAE
+        PPO_TRY(ppo_whiten(io->rewards, io->mask, M, 0, p->whiten_eps, io->rewards, nullptr, io->workspace, stream));
+    PPO_TRY(ppo_gae(io->rewards, io->values, io->seq_len, B, T, p->gamma, p->lam, io->advantages, io->returns, stream));
+    PPO_TRY(ppo_whiten(io->advantages, io->mask, M, 1, p->whiten_eps, io->advantages_whitened, io->whiten_stats,
+                       io->workspace, stream));
+    return ppo_loss_from_logprob(io->logprob, io->entropy, B, T, io->mask, io->old_logprob ? io->old_logprob : io->logprob,
+                                 io->advantages_whitened, io->values_new, io->values, io->returns, p, io->losses,
+                                 io->dlogprob, io->dvalues, io->workspace, stream);
+}
+
+extern "C" int ppo_lmhead_step_host(const ppo_lmhead_step_io *host, const ppo_lmhead_step_io *dev, int32_t B, int32_t T,
+                                    int64_t K, int64_t V, const ppo_params *p, void *stream)
+{
+    if (!host || !dev || !p) return PPO_ERR_NULL;
+    if (B <= 0 || T <= 0 || K <= 0 || V <= 0) return PPO_ERR_SHAPE;
+    if (!host->H || !host->W || !host->W_ref || !host->responses || !host->scores || !host->values || !host->values_new)
+        return PPO_ERR_NULL;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const size_t bt = (size_t)B * (size_t)T, w_bytes = (size_t)K * (size_t)V * 2;
+    // (the rows of H behind a response's first EOS are never multiplied: they are not copied either)
+    PPO_TRY(copy_in_real_rows(const_cast<void *>(dev->H), host->H, host->responses, B, T, (size_t)K * 2, p->eos_id, s));
+    PPO_TRY(copy_in(const_cast<void *>(dev->W), host->W, w_bytes, s));
+    PPO_TRY(copy_in(const_cast<void *>(dev->W_ref), host->W_ref, w_bytes, s));
+    PPO_TRY(copy_in(const_cast<int32_t *>(dev->responses), host->responses, bt * 4, s));
+    PPO_TRY(copy_in(const_cast<float *>(dev->scores), host->scores, (size_t)B * 4, s));
+    PPO_TRY(copy_in(const_cast<float *>(dev->values), host->values, bt * 4, s));
+    PPO_TRY(copy_in(const_cast<float *>(dev->values_new), host->values_new, bt * 4, s));
+    PPO_TRY(copy_in(const_cast<float *>(dev->old_logprob), host->old_logprob, bt * 4, s));
+    ppo_lmhead_step_io run = *dev;
+    if (!host->old_logprob) run.old_logprob = nullptr;
+    PPO_TRY(ppo_lmhead_step(&run, B, T, K, V, p, stream));
+    PPO_TRY(copy_out(host->responses_out, dev->responses_out, bt * 4, s));
+    PPO_TRY(copy_out(host->eos_index, dev->eos_index, (size_t)B * 4, s));
+    PPO_TRY(copy_out(host->seq_len, dev->seq_len, (size_t)B * 4, s));
+    PPO_TRY(copy_out(host->mask, dev->mask, bt, s));
+    PPO_TRY(copy_out(host->scores_out, dev->scores_out, (size_t)B * 4, s));
+    PPO_TRY(copy_out(host->logprob, dev->logprob, bt * 4, s));
+    PPO_TRY(copy_out(host->entropy, dev->entropy, bt * 4, s));
+    PPO_TRY(copy_out(host->lse, dev->lse, bt * 4, s));
+    PPO_TRY(copy_out(host->ref_logprob, dev->ref_logprob, bt * 4, s));
+    PPO_TRY(copy_out(host->kl, dev->kl, bt * 4, s));
+    PPO_TRY(copy_out(host->rewards, dev->rewards, bt * 4, s));
+    PPO_TRY(copy_out(host->advantages, dev->advantages, bt * 4, s));
+    PPO_TRY(copy_out(host->returns, dev->returns, bt * 4, s));
+    PPO_TRY(copy_out(host->advantages_whitened, dev->advantages_whitened, bt * 4, s));
+    PPO_TRY(copy_out(host->whiten_stats, dev->whiten_stats, 3 * 4, s));
+    PPO_TRY(copy_out(host->losses, dev->losses, 8 * 4, s));
+    PPO_TRY(copy_out(host->dlogprob, dev->dlogprob, bt * 4, s));
+    PPO_TRY(copy_out(host->dvalues, dev->dvalues, bt * 4, s));
+    PPO_RETURN_IF_CUDA(cudaStreamSynchronize(s));
+    return PPO_OK;
+}

@@ -249,3 +249,60 @@ def test_config4_chained_path_against_the_oracle(P, oracle):
     assert 0 < ref["losses"][4] < 1 and 0 < ref["losses"][5] < 1
     assert_abs(n * npy(out["dvalues"]), n * ref["dvalues"], 1e-4, "n*dvalues")
     assert_abs((n * npy(out["dlogprob"]).astype(np.float64))[~kink], (n * ref["dlogprob"])[~kink], 1e-4, "n*dlogprob")
+
+
+def test_lmhead_step_and_host_step_match_the_separate_calls(P):
+    """ppo_lmhead_step / ppo_lmhead_step_host only sequence the entry points of the fused-LM-head config: same bits as
+    calling them one by one (the chained test above checks those against the oracle); the host variant copies in only the
+    rows of H that the GEMMs read."""
+    from paper_2403_17031_b200 import binding
+    from paper_2403_17031_b200.synthetic import CONFIGS, make_lmhead_batch
+    cfg = CONFIGS[4]
+    h = cfg.hyper
+    p = binding.params_from(h)
+    B, T, K, V = 24, 53, 256, 2048
+    b = make_lmhead_batch(cfg, "cuda", M=B * T, K=K, V=V)
+    ws = P.new_workspace(max(P.lmhead_workspace_bytes(B * T, K, V), P.workspace_bytes(B, T, V)))
+    tok = b["responses"].reshape(-1)
+    ro, ei, sl, mask, so = P.truncate_and_score(b["responses"], b["scores"], h.eos_id, h.pad_id, h.no_eos_score)
+    lp, ent, lse = P.lmhead_logprob_entropy(b["H"], b["W"], tok, h.temperature, ws, mask=mask.view(-1))
+    rlp, _, _ = P.lmhead_logprob_entropy(b["H"], b["W_ref"], tok, h.temperature, ws, mask=mask.view(-1))
+    lp, ent, lse, rlp = (t.view(B, T).clone() for t in (lp, ent, lse, rlp))
+    kl, rew = P.kl_rewards(lp, rlp, mask, sl, so, h.kl_coef)
+    adv, ret = P.gae(rew, b["values"], sl, h.gamma, h.lam)
+    aw, st = P.whiten(adv, mask, True, h.whiten_eps, workspace=ws)
+    old = (lp + b["old_logprob_noise"]).contiguous()
+    want_loss = P.loss_from_logprob(lp, ent, mask, old, aw, b["values_new"], b["values"], ret, p, ws)
+    want = {"responses_out": ro, "eos_index": ei, "seq_len": sl, "mask": mask, "scores_out": so, "logprob": lp, "entropy": ent,
+            "lse": lse, "ref_logprob": rlp, "kl": kl, "rewards": rew, "advantages": adv, "returns": ret,
+            "advantages_whitened": aw, "whiten_stats": st, "losses": want_loss["losses"], "dlogprob": want_loss["dlogprob"],
+            "dvalues": want_loss["dvalues"]}
+    torch.cuda.synchronize()
+    inputs = {"H": b["H"], "W": b["W"], "W_ref": b["W_ref"], "responses": b["responses"], "scores": b["scores"],
+              "values": b["values"], "values_new": b["values_new"], "old_logprob": old}
+    out = {k: torch.full_like(v, 7) for k, v in want.items()}
+    ws2 = P.new_workspace(max(P.lmhead_workspace_bytes(B * T, K, V), P.workspace_bytes(B, T, V)))
+    io = binding.LMHeadStepIO.from_tensors({**inputs, **out, "workspace": ws2}, cuda=True)
+    binding.lmhead_step(io, B, T, K, V, p)
+    torch.cuda.synchronize()
+    assert P.last_device_status(ws2) == 0
+    for k in want:
+        assert torch.equal(out[k], want[k]), k
+    # host buffers in, host buffers out; the staging copy of H starts out as garbage behind the first EOS
+    host_in = {k: v.cpu().pin_memory() for k, v in inputs.items()}
+    host_out = {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in want.items()}
+    stage = {k: torch.empty_like(v) for k, v in inputs.items()}
+    stage["H"].fill_(float("nan"))
+    dev_out = {k: torch.full_like(v, 7) for k, v in want.items()}
+    binding.lmhead_step_host(binding.LMHeadStepIO.from_tensors({**host_in, **host_out}, cuda=False),
+                             binding.LMHeadStepIO.from_tensors({**stage, **dev_out, "workspace": ws2}, cuda=True),
+                             B, T, K, V, p)
+    for k in want:
+        assert torch.equal(host_out[k], want[k].cpu()), k
+    assert torch.isnan(stage["H"].view(B, T, K)[mask == 0]).all()       # padding rows of H were never copied
+    # first-epoch default: no stored old log-probs -> ratio 1 -> nothing clipped
+    io2 = binding.LMHeadStepIO.from_tensors({**{k: v for k, v in inputs.items() if k != "old_logprob"}, **out,
+                                             "workspace": ws2}, cuda=True)
+    binding.lmhead_step(io2, B, T, K, V, p)
+    torch.cuda.synchronize()
+    assert float(out["losses"][3]) == 0.0 and float(out["losses"][4]) == 0.0
