@@ -49,10 +49,15 @@ _LOSS_KERNEL_SOURCES = ("ppo_rows_bulk.cu", "ppo_rows.cuh", "ppo_common.cuh")
 
 
 def _loss_kernel_hash():
+    """Hash of the loss kernel's sources with comments and white space taken out (a comment edit changes no kernel)."""
+    import re
     h = hashlib.sha256()
     for name in _LOSS_KERNEL_SOURCES:
-        with open(os.path.join(ROOT, "paper_2403_17031_b200", "csrc", name), "rb") as f:
-            h.update(f.read())
+        with open(os.path.join(ROOT, "paper_2403_17031_b200", "csrc", name), "r") as f:
+            text = f.read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        text = re.sub(r"//[^\n]*", "", text)
+        h.update("".join(text.split()).encode())
     return h.hexdigest()
 
 
