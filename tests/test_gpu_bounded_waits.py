@@ -12,13 +12,12 @@ import torch
 pytestmark = pytest.mark.gpu
 
 DEV_TIMEOUT = 4
-_SOURCES = ["ppo_rows.cu", "ppo_rows_bulk.cu", "ppo_tokens.cu", "ppo_step.cu"]
 
 
 def _load_variant(tmp, withhold):
     from paper_2403_17031_b200 import binding, build
     path = build.build_variant(os.path.join(str(tmp), "libppo_withhold%d.so" % withhold),
-                               ["PPO_TEST_WITHHOLD_FLAGS=%d" % withhold, "PPO_WAIT_TRIES=512"], only=_SOURCES)
+                               ["PPO_TEST_WITHHOLD_FLAGS=%d" % withhold, "PPO_WAIT_TRIES=512"])
     L = C.CDLL(path)
     for name in ("ppo_loss_fwd_bwd", "ppo_last_device_status", "ppo_step"):
         res, args = binding._SIGS[name]
