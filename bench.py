@@ -567,6 +567,12 @@ def measure_lmhead(cfg, args, D, K, warmup, target_s, full: bool):
         blocks, total_ms = _timed_blocks(lambda: step(old), K, est, D, target_s)
         lm_ms = _back_to_back_ms(lm_policy, n=10)
         bwd_ms = _back_to_back_ms(backward, n=5) if bwd_out is not None else None
+        if bwd_out is None and full:
+            # the step after the loss (gradient on the log-probs back to dlogits, dH, dW), timed on its own
+            bwd_out = {"dlogits": torch.empty((M, V), dtype=torch.bfloat16, device=dev),
+                       "dH": torch.empty_like(b["H"]), "dW": torch.empty_like(b["W"])}
+            bwd_ms = _back_to_back_ms(backward, n=3)
+            bwd_out = None
     ms_per_step = D.max_float(statistics.median(blocks) / K)
     status = binding.last_device_status(ws)
     n_real = int(o["mask"].sum().item())
@@ -644,10 +650,74 @@ def _summary_of(res):
            "roofline": {k: res["roofline"].get(k) for k in keep if k in res["roofline"]},
            "clocks": res["clocks"], "device_status": c.get("device_status")}
     for k in ("path_hbm_frac_of_8tbs", "logprob_entropy_ms", "logprob_entropy_frac_of_8tbs", "loss_fwd_bwd_next_epoch_ms",
-              "lmhead_ms"):
+              "lmhead_ms", "lmhead_bwd_ms", "lmhead_bwd_tflops"):
         if k in c:
             out[k] = c[k]
     return out
+
+
+def _extra_dpo(args, D, K, target_s):
+    """The DPO step on preference pairs (the paper's (B, 638) layout, 8 pairs per GPU), short form for config.others."""
+    from paper_2403_17031_b200 import binding
+    from paper_2403_17031_b200.pipeline import DPOStep
+    from paper_2403_17031_b200.synthetic import PREF_CONFIGS, make_pref_batch
+    cfg = PREF_CONFIGS["dpo"]
+    b = make_pref_batch(cfg, D.dev, seed=cfg.seed + 1000 * D.rank)
+    P, T, V = cfg.P, cfg.T, cfg.V
+    st = DPOStep(P, T, V, cfg.torch_dtype, cfg.beta, device=D.dev)
+    run = lambda: st.step(b["policy_logits"], b["ref_logits"], b["tokens"], b["mask"])
+    for _ in range(3):
+        run()
+    torch.cuda.synchronize()
+    n_real, rows, es = int(b["mask"].sum().item()), 2 * P * T, 2 if cfg.dtype == "bf16" else 4
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record(); run(); t1.record(); torch.cuda.synchronize()
+    with ClockSampler(D.local) as clk:
+        blocks, total_ms = _timed_blocks(run, K, t0.elapsed_time(t1), D, target_s)
+        bwd_ms = _back_to_back_ms(lambda: binding.logprob_bwd(b["policy_logits"], b["tokens"], b["mask"], st.out["dlogprob"],
+                                                              1.0, st.workspace, dlogits=st.out["dlogits"]))
+    ms = D.max_float(statistics.median(blocks) / K)
+    peak, _ = _peaks("hbm_gbs", 6650.0)
+    bwd_bytes = (n_real + rows) * V * es
+    gbs = bwd_bytes / (bwd_ms * 1e-3) / 1e9
+    return {"workload": "config5 %s (DPO step, %d pairs x (2, %d) positions, V=%d, %s)" % (cfg.name, P, T, V, cfg.dtype),
+            "ms_per_step": ms, "tokens_per_s": n_real * D.world / (ms * 1e-3), "real_tokens": n_real,
+            "response_positions": rows, "blocks": len(blocks), "steps_timed": len(blocks) * K, "timed_region_ms": total_ms,
+            "roofline": {"kernel": "row_engine_kernel (ppo_logprob_bwd)", "achieved": gbs, "peak": peak, "unit": "GB/s",
+                         "frac": gbs / peak, "frac_of_8tbs": gbs / 8000.0, "algorithmic_bytes": bwd_bytes},
+            "clocks": clk.summary(), "device_status": st.device_status()}
+
+
+def _extra_sample(args, D, K, target_s):
+    """Temperature sampling fused with the log-prob pass on config-1 logits, short form for config.others."""
+    from paper_2403_17031_b200 import binding
+    from paper_2403_17031_b200.synthetic import CONFIGS, make_batch
+    cfg = CONFIGS[1]
+    x = make_batch(cfg, D.dev, seed=cfg.seed + 1000 * D.rank, with_ref=False)["policy_logits"]
+    B, T, V = x.shape
+    ws = binding.new_workspace(binding.workspace_bytes(B, T, V), D.dev)
+    out = binding.sample_logprob_entropy(x, cfg.hyper.temperature, 20240317, 0, workspace=ws)
+    ctr = [0]
+
+    def run():
+        ctr[0] += 1
+        binding.sample_logprob_entropy(x, cfg.hyper.temperature, 20240317, ctr[0], workspace=ws, out=out)
+    for _ in range(3):
+        run()
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record(); run(); t1.record(); torch.cuda.synchronize()
+    with ClockSampler(D.local) as clk:
+        blocks, total_ms = _timed_blocks(run, K, t0.elapsed_time(t1), D, target_s)
+    ms = D.max_float(statistics.median(blocks) / K)
+    peak, _ = _peaks("hbm_gbs", 6650.0)
+    gbs = B * T * V * 2 / (ms * 1e-3) / 1e9
+    return {"workload": "config6 fused sampling + log-prob on config1 logits (%d rows x %d, bf16)" % (B * T, V),
+            "ms_per_step": ms, "tokens_per_s": B * T * D.world / (ms * 1e-3), "response_positions": B * T,
+            "blocks": len(blocks), "steps_timed": len(blocks) * K, "timed_region_ms": total_ms,
+            "roofline": {"kernel": "sample_kernel (ppo_sample_logprob_entropy)", "achieved": gbs, "peak": peak, "unit": "GB/s",
+                         "frac": gbs / peak, "frac_of_8tbs": gbs / 8000.0, "algorithmic_bytes": B * T * V * 2},
+            "clocks": clk.summary(), "device_status": binding.last_device_status(ws)}
 
 
 def run_ours(args, cfgs):
@@ -691,6 +761,11 @@ def run_ours(args, cfgs):
             if idx == 4:
                 summary["e2e"], summary["cpu_baseline"] = res["e2e"], res["cpu_baseline"]
             others.append(summary)
+        # the widened workloads, so that they too are measured by whoever runs the default command
+        others.append(_extra_dpo(args, D, min(K, 20), min(0.2, args.target_seconds)))
+        torch.cuda.empty_cache()
+        others.append(_extra_sample(args, D, min(K, 20), min(0.2, args.target_seconds)))
+        torch.cuda.empty_cache()
     if rank == 0:
         line = {
             "metric": "response tokens/s", "value": head["value"], "unit": "tokens/s", "n_gpus": world, "steps": K,
